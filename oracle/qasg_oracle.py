@@ -1,0 +1,332 @@
+"""Oracle for one synchronisation + update step of QCMD adagrad / QRDA adagrad.
+
+TEST INFRASTRUCTURE ONLY (see the package docstring).  Every function restates one
+passage of the paper in numpy.  Floating point is fp64 except where a comparison
+decides an integer code: there the operands are fp32, like the data they come from.
+
+Conventions the paper leaves open (each is this library's documented reading):
+
+* 2-bit code per coordinate: 0 -> 0, 1 -> +1, 2 -> -1, 3 is never produced and decodes
+  to 0.  Coordinate i sits in 32-bit word i // 16 at bits [2*(i%16), 2*(i%16)+1].
+* The sums over a worker's gradient ("canonical sum") are taken in one fixed order so
+  that the fp64 result, and the fp32 threshold / scale rounded from it, do not depend
+  on who computes them.  See `canonical_sum`.
+* The stochastic ternary quantizer (the unbiased comparison quantizer the paper's
+  theorems assume) draws from Philox4x32-10 keyed by (seed, t, m, i).
+* Scalars lambda, eta, delta and the threshold coefficient are fp32 at the library
+  boundary; they are promoted exactly to fp64 here.
+"""
+import numpy as np
+
+F32 = np.float32
+F64 = np.float64
+
+# Geometry of the canonical sum: a tile is TILE_ROWS rows of TILE_COLS consecutive
+# coordinates (row-major), i.e. 4096 consecutive coordinates.
+TILE_ROWS = 4
+TILE_COLS = 1024
+TILE = TILE_ROWS * TILE_COLS
+
+
+# ----------------------------------------------------------------------------------
+# Canonical summation
+# ----------------------------------------------------------------------------------
+def _adjacent_pairs(a):
+    """Pairwise (recursive halving) sum along the last axis, whose length is 2**k:
+    level by level, element 2j is added to element 2j+1."""
+    while a.shape[-1] > 1:
+        a = a[..., 0::2] + a[..., 1::2]
+    return a[..., 0]
+
+
+def pairwise_sum(a):
+    """Pairwise sum of a 1-D fp64 vector, zero-padded (+0.0) to the next power of two."""
+    a = np.asarray(a, dtype=F64).ravel()
+    n = max(1, a.size)
+    p = 1 << (n - 1).bit_length()
+    buf = np.zeros(p, dtype=F64)
+    buf[: a.size] = a
+    return F64(_adjacent_pairs(buf))
+
+
+def canonical_sum(a):
+    """Sum of a non-negative fp32 vector in the library's fixed order.
+
+    The vector is cut into tiles of 4096 consecutive coordinates (the last one padded
+    with +0.0).  A tile is read as 4 rows x 1024 columns; each column is summed down
+    its 4 rows, in row order, in fp64; the 1024 column sums are combined by pairwise
+    summation; the tile sums are combined by pairwise summation over the tile index
+    (padded with +0.0 to a power of two).  All additions are fp64.
+    """
+    a = np.asarray(a, dtype=F32).ravel()
+    d = a.size
+    n_tiles = max(1, -(-d // TILE))
+    buf = np.zeros(n_tiles * TILE, dtype=F32)
+    buf[:d] = a
+    buf = buf.reshape(n_tiles, TILE_ROWS, TILE_COLS)
+    col = buf[:, 0, :].astype(F64)
+    for r in range(1, TILE_ROWS):
+        col = col + buf[:, r, :].astype(F64)
+    tile_sums = _adjacent_pairs(col)
+    return pairwise_sum(tile_sums)
+
+
+# ----------------------------------------------------------------------------------
+# Threshold quantization (Section 3.4, Q_Delta; threshold from Section 3.5)
+# ----------------------------------------------------------------------------------
+def threshold_quantize(v, coef=0.75):
+    """Q_Delta(v) = s * tern with the approximate threshold of Section 3.5.
+
+    Delta = coef/d * sum_i |v_i|                      (Section 3.5, coef = 0.75)
+    tern_i = +1 if v_i > Delta, -1 if v_i < -Delta, 0 if |v_i| <= Delta   (Section 3.4)
+    s = mean of |v_i| over I_Delta = {i : |v_i| > Delta}                   (s*_Delta)
+
+    Returns (tern int8[d], s fp32, Delta fp32, |I_Delta| int).  An empty I_Delta gives
+    s = 0.  The comparisons are fp32 against the fp32 Delta.
+    """
+    v = np.asarray(v, dtype=F32).ravel()
+    d = v.size
+    absv = np.abs(v)
+    with np.errstate(invalid="ignore", over="ignore"):
+        total = canonical_sum(absv)
+        delta = F32((F64(F32(coef)) * total) / F64(d))
+        pos = v > delta
+        neg = v < -delta
+    tern = pos.astype(np.int8) - neg.astype(np.int8)
+    selected = pos | neg
+    n = int(np.count_nonzero(selected))
+    if n == 0:
+        return tern, F32(0.0), delta, 0
+    picked = canonical_sum(np.where(selected, absv, F32(0.0)))
+    scale = F32(picked / F64(n))
+    return tern, scale, delta, n
+
+
+# ----------------------------------------------------------------------------------
+# Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
+# 1, 2, 3", SC'11) and the stochastic ternary quantizer
+# ----------------------------------------------------------------------------------
+_PHILOX_M0 = np.uint64(0xD2511F53)
+_PHILOX_M1 = np.uint64(0xCD9E8D57)
+_PHILOX_W0 = 0x9E3779B9
+_PHILOX_W1 = 0xBB67AE85
+_MASK32 = np.uint64(0xFFFFFFFF)
+_SH32 = np.uint64(32)
+
+
+def philox4x32_10(c0, c1, c2, c3, k0, k1):
+    """Ten rounds of Philox-4x32.  Counter words are arrays (broadcast together), key
+    words are Python ints.  Returns four uint32 arrays."""
+    c0, c1, c2, c3 = np.broadcast_arrays(
+        *(np.asarray(c, dtype=np.uint64) & _MASK32 for c in (c0, c1, c2, c3)))
+    k0 = int(k0) & 0xFFFFFFFF
+    k1 = int(k1) & 0xFFFFFFFF
+    for _ in range(10):
+        p0 = _PHILOX_M0 * c0          # 32x32 -> 64-bit products
+        p1 = _PHILOX_M1 * c2
+        hi0, lo0 = p0 >> _SH32, p0 & _MASK32
+        hi1, lo1 = p1 >> _SH32, p1 & _MASK32
+        c0, c1, c2, c3 = (hi1 ^ c1 ^ np.uint64(k0), lo1,
+                          hi0 ^ c3 ^ np.uint64(k1), lo0)
+        k0 = (k0 + _PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + _PHILOX_W1) & 0xFFFFFFFF
+    return tuple(c.astype(np.uint32) for c in (c0, c1, c2, c3))
+
+
+def philox_draws(seed, t, m, idx, domain=0):
+    """The random word and uniform drawn for (seed, step t, worker m, coordinate idx).
+
+    key     = (seed[31:0], seed[63:32])
+    counter = (idx >> 2, m | domain << 16, t[31:0], t[63:32]); coordinate idx takes
+              output word idx & 3.
+    u       = (word >> 8) * 2**-24, exactly representable in fp32, in [0, 1).
+    `t` and `idx` may be arrays (broadcast).  Returns (word uint32, u fp32).
+    """
+    idx = np.asarray(idx, dtype=np.uint64)
+    t = np.asarray(t, dtype=np.uint64)
+    seed = int(seed)
+    words = philox4x32_10(idx >> np.uint64(2),
+                          np.uint64((int(m) & 0xFFFF) | (int(domain) << 16)),
+                          t & _MASK32, t >> _SH32,
+                          seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    lane = np.broadcast_to(idx & np.uint64(3), words[0].shape)
+    word = np.choose(lane.astype(np.intp), words)
+    u = (word >> np.uint32(8)).astype(F32) * F32(2.0 ** -24)
+    return word, u
+
+
+def ternary_stochastic_quantize(v, u):
+    """Unbiased ternary quantizer with the max-norm scaler (the comparison quantizer
+    of Section 3.4 / related work: levels {-1, 0, 1} times a scaler).
+
+    s = max_i |v_i|;  tern_i = sign(v_i) with probability |v_i| / s, else 0, realised
+    as  u_i < |v_i| / s  with the fp32 division and the given uniforms u in [0, 1).
+    Returns (tern int8[d], s fp32).  s = 0 gives all zeros.
+    """
+    v = np.asarray(v, dtype=F32).ravel()
+    u = np.asarray(u, dtype=F32).ravel()
+    absv = np.abs(v)
+    s = F32(absv.max()) if v.size else F32(0.0)
+    if not s > 0:
+        return np.zeros(v.size, dtype=np.int8), F32(0.0)
+    prob = absv / s
+    keep = u < prob
+    tern = (np.sign(v).astype(np.int8)) * keep.astype(np.int8)
+    return tern, s
+
+
+# ----------------------------------------------------------------------------------
+# Encoding (Section 3.5, "Encode": 2 bits per coordinate + one fp32 scale)
+# ----------------------------------------------------------------------------------
+def code_words(d):
+    return -(-int(d) // 16)
+
+
+def pack_codes(tern):
+    """Ternary vector -> little-endian array of 32-bit words, 16 codes per word, the
+    tail padded with code 0."""
+    tern = np.asarray(tern).ravel()
+    d = tern.size
+    w = code_words(d)
+    two_bit = np.zeros(w * 16, dtype=np.uint32)
+    two_bit[:d] = np.where(tern > 0, 1, np.where(tern < 0, 2, 0))
+    shifts = (2 * np.arange(16)).astype(np.uint32)
+    return np.bitwise_or.reduce(two_bit.reshape(w, 16) << shifts, axis=1).astype(np.uint32)
+
+
+def unpack_codes(words, d):
+    """Inverse of `pack_codes` for the first d coordinates; code 3 decodes to 0."""
+    words = np.asarray(words, dtype=np.uint32).ravel()
+    shifts = (2 * np.arange(16)).astype(np.uint32)
+    two_bit = ((words[:, None] >> shifts) & np.uint32(3)).ravel()[: int(d)]
+    return (two_bit == 1).astype(np.int8) - (two_bit == 2).astype(np.int8)
+
+
+def wire_bits(d):
+    """Bits one worker sends for a dense model: 32 + 2d (Section 3.5, "Encode")."""
+    return 32 + 2 * int(d)
+
+
+# ----------------------------------------------------------------------------------
+# Server side: decode and average (SynQ_t)
+# ----------------------------------------------------------------------------------
+def decode_average(terns, scales):
+    """SynQ_t = (1/M) sum_m s_m * tern_m, in fp64."""
+    terns = np.asarray(terns)
+    scales = np.asarray(scales, dtype=F32)
+    m_workers = terns.shape[0]
+    acc = np.zeros(terns.shape[1], dtype=F64)
+    for m in range(m_workers):
+        acc = acc + F64(scales[m]) * terns[m].astype(F64)
+    return acc / F64(m_workers)
+
+
+# ----------------------------------------------------------------------------------
+# Worker side: accumulator H_t and the two closed-form updates
+# ----------------------------------------------------------------------------------
+def _scalars(lam, eta, delta):
+    return F64(F32(lam)), F64(F32(eta)), F64(F32(delta))
+
+
+def cmd_step(q, x, h, lam, eta, delta):
+    """QCMD adagrad update (closed form of the composite-mirror-descent argmin).
+
+    h <- h + q^2 (h holds c_t^2 = sum of squared quantized gradients, current one
+    included);  H = delta + sqrt(h);  u = x - (eta/H) q;
+    x <- sign(u) * [|u| - lambda*eta/H]_+ .
+    Returns (x_new, h_new, a) with a = |u| * H / eta, the quantity the closed form
+    compares with lambda (x_new == 0 exactly when a <= lambda).
+    """
+    lam, eta, delta = _scalars(lam, eta, delta)
+    q = np.asarray(q, dtype=F64)
+    x = np.asarray(x, dtype=F64)
+    h = np.asarray(h, dtype=F64)
+    h_new = h + q * q
+    big_h = delta + np.sqrt(h_new)
+    u = x - (eta / big_h) * q
+    x_new = np.sign(u) * np.maximum(np.abs(u) - lam * eta / big_h, 0.0)
+    x_new = x_new + 0.0                       # -0.0 -> +0.0
+    return x_new, h_new, np.abs(u) * big_h / eta
+
+
+def rda_step(q, h, z, t, lam, eta, delta):
+    """QRDA adagrad update (closed form of the dual-averaging argmin).
+
+    h <- h + q^2;  z <- z + q (z = sum of quantized gradients up to t);
+    H = delta + sqrt(h);  x <- -sign(z) * (t*eta/H) * [|z|/t - lambda]_+ .
+    Returns (x_new, h_new, z_new, a) with a = |z|/t, compared with lambda.
+    """
+    lam, eta, delta = _scalars(lam, eta, delta)
+    q = np.asarray(q, dtype=F64)
+    h = np.asarray(h, dtype=F64)
+    z = np.asarray(z, dtype=F64)
+    tt = F64(int(t))
+    h_new = h + q * q
+    z_new = z + q
+    big_h = delta + np.sqrt(h_new)
+    a = np.abs(z_new) / tt
+    x_new = -np.sign(z_new) * (tt * eta / big_h) * np.maximum(a - lam, 0.0)
+    x_new = x_new + 0.0
+    return x_new, h_new, z_new, a
+
+
+# ----------------------------------------------------------------------------------
+# The whole step (one-way quantization: local gradients quantized, the average not)
+# ----------------------------------------------------------------------------------
+QUANT_THRESHOLD = 0
+QUANT_TERNARY_STOCH = 1
+QUANT_NONE = 2
+RULE_CMD = 0
+RULE_RDA = 1
+
+
+def quantize_workers(g, quantizer, t=1, seed=0, coef=0.75):
+    """Quantize each worker's gradient row of g (M x d, fp32).
+
+    Returns dict(terns int8[M,d], scales fp32[M], thresholds fp32[M], counts int64[M],
+    codes uint32[M, W]).  For the stochastic quantizer thresholds are 0 and counts are
+    the numbers of non-zero codes.
+    """
+    g = np.asarray(g, dtype=F32)
+    m_workers, d = g.shape
+    terns = np.zeros((m_workers, d), dtype=np.int8)
+    scales = np.zeros(m_workers, dtype=F32)
+    thresholds = np.zeros(m_workers, dtype=F32)
+    counts = np.zeros(m_workers, dtype=np.int64)
+    for m in range(m_workers):
+        if quantizer == QUANT_THRESHOLD:
+            terns[m], scales[m], thresholds[m], counts[m] = threshold_quantize(g[m], coef)
+        elif quantizer == QUANT_TERNARY_STOCH:
+            _, u = philox_draws(seed, t, m, np.arange(d, dtype=np.uint64))
+            terns[m], scales[m] = ternary_stochastic_quantize(g[m], u)
+            counts[m] = np.count_nonzero(terns[m])
+        else:
+            raise ValueError("quantizer")
+    codes = np.stack([pack_codes(terns[m]) for m in range(m_workers)])
+    return dict(terns=terns, scales=scales, thresholds=thresholds, counts=counts, codes=codes)
+
+
+def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0, coef=0.75):
+    """One iteration: quantize every worker's gradient, decode and average, update the
+    accumulator and apply the rule's closed-form update.  State in, state out (fp64).
+
+    quantizer == QUANT_NONE skips quantization: q is the fp64 mean of the rows of g
+    (the 32-bit CMD / RDA adagrad baseline).
+    Returns dict(x, h, z, a, q, quant) where `a` is the quantity compared with lambda
+    and `quant` the output of `quantize_workers` (None without quantization).
+    """
+    g = np.asarray(g, dtype=F32)
+    if quantizer == QUANT_NONE:
+        quant = None
+        q = g.astype(F64).sum(axis=0) / F64(g.shape[0])
+    else:
+        quant = quantize_workers(g, quantizer, t=t, seed=seed, coef=coef)
+        q = decode_average(quant["terns"], quant["scales"])
+    if rule == RULE_CMD:
+        x_new, h_new, a = cmd_step(q, x, h, lam, eta, delta)
+        z_new = None if z is None else np.asarray(z, dtype=F64)
+    elif rule == RULE_RDA:
+        x_new, h_new, z_new, a = rda_step(q, h, z, t, lam, eta, delta)
+    else:
+        raise ValueError("rule")
+    return dict(x=x_new, h=h_new, z=z_new, a=a, q=q, quant=quant)

@@ -1,0 +1,365 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these compares the oracle with itself or with the CUDA path: each one checks a
+function against a closed form, a brute-force search, an invariant the paper states,
+a library routine it must reduce to, or published known-answer values.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import qasg_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ canonical sum
+def test_canonical_sum_matches_exact_sum_to_fp64_accuracy():
+    rng = np.random.default_rng(11)
+    for d in (1, 5, 1023, 1024, 4095, 4096, 4097, 3 * 4096 + 17, 100_003):
+        a = np.abs(rng.standard_normal(d)).astype(np.float32) * np.float32(10.0 ** rng.integers(-6, 6))
+        exact = math.fsum(float(v) for v in a)
+        got = float(O.canonical_sum(a))
+        levels = 3 + 10 + max(1, math.ceil(math.log2(max(2, d / 4096))))
+        assert abs(got - exact) <= levels * 2.0 ** -53 * exact
+
+
+def test_canonical_sum_exact_when_every_partial_sum_is_representable():
+    rng = np.random.default_rng(12)
+    a = rng.integers(0, 1 << 20, size=50_001).astype(np.float32)   # integers < 2^20
+    assert float(O.canonical_sum(a)) == float(int(a.astype(np.int64).sum()))
+
+
+def test_canonical_sum_is_not_an_fp32_sum():
+    # 2^24 followed by ones: an fp32 accumulator would drop every 1.
+    a = np.ones(5000, dtype=np.float32)
+    a[0] = 2.0 ** 24
+    assert float(O.canonical_sum(a)) == 2.0 ** 24 + 4999
+
+
+def test_pairwise_sum_tree_shape():
+    # With fp64 values chosen so that rounding depends on the pairing, the adjacent-pair
+    # tree (a0+a1)+(a2+a3) differs from the left-to-right sum; check the tree is used.
+    big, one = 2.0 ** 53, 1.0
+    a = [big, one, one, one]                      # ((big+1)+(1+1)) = big+2 ; sequential = big
+    assert float(O.pairwise_sum(a)) == big + 2.0
+    assert float(O.pairwise_sum([one, one, one])) == 3.0        # padding with +0.0
+
+
+def test_threshold_equals_exact_definition_on_seeded_cases():
+    # Delta from the canonical sum equals Delta from the exactly rounded sum.
+    rng = np.random.default_rng(13)
+    for d in (7, 4096, 10_000, 65_537):
+        v = rng.standard_normal(d).astype(np.float32)
+        _, _, delta, _ = O.threshold_quantize(v)
+        exact = math.fsum(abs(float(t)) for t in v)
+        assert delta == np.float32(0.75 * exact / d)
+
+
+# ------------------------------------------------------------------ threshold quantizer
+def _q_error(v, tern, s):
+    return float(((v.astype(np.float64) - float(s) * tern) ** 2).sum())
+
+
+def test_scale_minimises_the_quadratic_for_fixed_threshold():
+    # Section 3.4: for a given Delta the optimal s is the mean of |v| over I_Delta.
+    rng = np.random.default_rng(1)
+    for d in (3, 8, 33):
+        v = rng.standard_normal(d).astype(np.float32)
+        tern, s, delta, n = O.threshold_quantize(v)
+        assert n == int((np.abs(v) > delta).sum()) and n > 0
+        grid = np.linspace(0.0, 2.0 * float(np.abs(v).max()), 200_001)
+        absv = np.abs(v).astype(np.float64)
+        sel = absv > float(delta)
+        obj = n * grid ** 2 - 2.0 * grid * absv[sel].sum() + (absv ** 2).sum()
+        assert abs(grid[obj.argmin()] - float(s)) <= grid[1] - grid[0]
+
+
+def test_error_identity_and_bound():
+    # ||v - Q(v)||^2 = ||v||^2 - |I| s^2 at the optimal s, hence <= ||v||^2.
+    rng = np.random.default_rng(2)
+    v = rng.standard_normal(5000).astype(np.float32)
+    tern, s, delta, n = O.threshold_quantize(v)
+    err = _q_error(v, tern, s)
+    v2 = float((v.astype(np.float64) ** 2).sum())
+    assert err == pytest.approx(v2 - n * float(s) ** 2, rel=1e-6)
+    assert err <= v2
+
+
+def _optimal_threshold_objective(v):
+    """Section 3.4: rank |v|, try every component as the threshold, maximise
+    (sum_{I}|v|)^2 / |I|."""
+    a = np.sort(np.abs(v).astype(np.float64))[::-1]
+    pref = np.cumsum(a)
+    obj = pref ** 2 / np.arange(1, a.size + 1)
+    return obj.max()
+
+
+def test_approximate_threshold_close_to_optimal_for_gaussian():
+    rng = np.random.default_rng(3)
+    for d in (16, 64):
+        for _ in range(20):
+            v = rng.standard_normal(d).astype(np.float32)
+            tern, s, delta, n = O.threshold_quantize(v)
+            if n == 0:
+                continue
+            got = (np.abs(v.astype(np.float64))[tern != 0].sum()) ** 2 / n
+            assert got <= _optimal_threshold_objective(v) * (1 + 1e-12)
+    v = rng.standard_normal(200_000).astype(np.float32) * np.float32(3.0)
+    tern, s, delta, n = O.threshold_quantize(v)
+    got = (np.abs(v.astype(np.float64))[tern != 0].sum()) ** 2 / n
+    assert got >= 0.99 * _optimal_threshold_objective(v)
+    # 0.75 * E|v| = 0.75 * sigma * sqrt(2/pi) ~ 0.6 sigma  (Section 3.5)
+    assert float(delta) == pytest.approx(0.75 * 3.0 * math.sqrt(2 / math.pi), rel=0.01)
+    # fraction of non-zero codes = P(|Z| > 0.598)
+    assert n / v.size == pytest.approx(math.erfc(0.75 * math.sqrt(2 / math.pi) / math.sqrt(2)), abs=0.005)
+
+
+def test_boundary_is_strict_and_worked_example():
+    # |v| = (3, 3, 6, 4): Delta = 0.75 * 16 / 4 = 3; components equal to Delta code 0.
+    v = np.array([3.0, -3.0, 6.0, -4.0], dtype=np.float32)
+    tern, s, delta, n = O.threshold_quantize(v)
+    assert delta == np.float32(3.0)
+    assert tern.tolist() == [0, 0, 1, -1]
+    assert n == 2 and s == np.float32(5.0)
+
+
+def test_zero_gradient_and_nonfinite():
+    tern, s, delta, n = O.threshold_quantize(np.zeros(100, dtype=np.float32))
+    assert not tern.any() and s == 0 and delta == 0 and n == 0
+    v = np.ones(10, dtype=np.float32)
+    v[3] = np.nan
+    tern, s, _, n = O.threshold_quantize(v)
+    assert not tern.any() and s == 0 and n == 0
+    v[3] = np.inf
+    tern, s, _, n = O.threshold_quantize(v)
+    assert not tern.any() and s == 0 and n == 0
+
+
+def test_power_of_two_equivariance():
+    rng = np.random.default_rng(4)
+    v = rng.standard_normal(9001).astype(np.float32)
+    t0, s0, d0, n0 = O.threshold_quantize(v)
+    for k in (-20, 7):
+        t1, s1, d1, n1 = O.threshold_quantize(v * np.float32(2.0 ** k))
+        assert np.array_equal(t0, t1) and n0 == n1
+        assert s1 == s0 * np.float32(2.0 ** k) and d1 == d0 * np.float32(2.0 ** k)
+
+
+# ------------------------------------------------------------------ encoding
+def test_pack_layout_and_bit_budget():
+    assert int(O.pack_codes(np.array([1, -1, 0, 1]))[0]) == (1 | (2 << 2) | (1 << 6))
+    tern = np.zeros(17, dtype=np.int8)
+    tern[16] = -1
+    words = O.pack_codes(tern)
+    assert words.tolist() == [0, 2]
+    rng = np.random.default_rng(5)
+    for d in (1, 15, 16, 17, 1000):
+        tern = rng.integers(-1, 2, size=d).astype(np.int8)
+        words = O.pack_codes(tern)
+        assert words.dtype == np.uint32 and words.size == O.code_words(d)
+        assert np.array_equal(O.unpack_codes(words, d), tern)
+        # Section 3.5: (32 + 2d) bits per worker, up to padding of the last word
+        assert O.wire_bits(d) == 32 + 2 * d <= 32 + 32 * words.size < O.wire_bits(d) + 32
+    assert O.unpack_codes(np.array([3], dtype=np.uint32), 1).tolist() == [0]
+
+
+# ------------------------------------------------------------------ Philox / stochastic mode
+def test_philox_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        v = [int(x, 16) for x in r]
+        out = O.philox4x32_10(v[0], v[1], v[2], v[3], v[4], v[5])
+        assert [int(o) for o in out] == v[6:]
+
+
+def test_philox_draws_keying():
+    idx = np.arange(64, dtype=np.uint64)
+    w, u = O.philox_draws(seed=0x1234567890ABCDEF, t=5, m=3, idx=idx)
+    # coordinate i takes word i&3 of the block with counter (i>>2, m, t_lo, t_hi)
+    for i in (0, 1, 6, 63):
+        blk = O.philox4x32_10(i >> 2, 3, 5, 0, 0x90ABCDEF, 0x12345678)
+        assert int(w[i]) == int(blk[i & 3])
+    assert u.dtype == np.float32 and (u >= 0).all() and (u < 1).all()
+    assert np.array_equal(u.astype(np.float64) * 2 ** 24, (w >> 8).astype(np.float64))
+    # every argument of the key changes the stream
+    base = O.philox_draws(1, 1, 0, idx)[0]
+    for other in (O.philox_draws(2, 1, 0, idx), O.philox_draws(1, 2, 0, idx),
+                  O.philox_draws(1, 1, 1, idx), O.philox_draws(1, 1, 0, idx, domain=1),
+                  O.philox_draws(1, 1 + (1 << 32), 0, idx)):
+        assert not np.array_equal(base, other[0])
+    big = O.philox_draws(7, 3, 2, np.arange(1 << 16, dtype=np.uint64))[1]
+    assert abs(float(big.mean()) - 0.5) < 0.01
+
+
+def test_stochastic_quantizer_unbiased_and_variance_identity():
+    # E[Q(g)] = g and E||Q(g) - g||^2 = E||Q(g)||^2 - ||g||^2 <= E||Q(g)||^2  (Section 3.3 remark)
+    g = np.array([0.9, -0.05, 0.3, 0.0, -1.2, 0.61, 0.007, -0.33], dtype=np.float32)
+    trials = 400_000
+    t = np.arange(1, trials + 1, dtype=np.uint64)[:, None]
+    idx = np.arange(g.size, dtype=np.uint64)[None, :]
+    _, u = O.philox_draws(seed=99, t=t, m=2, idx=idx)
+    s = np.float32(np.abs(g).max())
+    total = np.zeros(g.size)
+    sq = 0.0
+    err = 0.0
+    for lo in range(0, trials, 50_000):
+        for row in u[lo:lo + 50_000]:
+            tern, s_row = O.ternary_stochastic_quantize(g, row)
+            qv = float(s_row) * tern
+            total += qv
+            sq += float((qv ** 2).sum())
+            err += float(((qv - g) ** 2).sum())
+    mean = total / trials
+    p = np.abs(g.astype(np.float64)) / float(s)
+    sigma = float(s) * np.sqrt(p * (1 - p) / trials)
+    assert (np.abs(mean - g) <= 5 * sigma + 1e-12).all()
+    g2 = float((g.astype(np.float64) ** 2).sum())
+    assert err / trials == pytest.approx(sq / trials - g2, rel=0.02)
+    assert err / trials <= sq / trials
+    # expected squared norm is s * ||g||_1
+    assert sq / trials == pytest.approx(float(s) * float(np.abs(g).sum()), rel=0.01)
+
+
+def test_stochastic_quantizer_edges():
+    tern, s = O.ternary_stochastic_quantize(np.zeros(5, dtype=np.float32), np.zeros(5, dtype=np.float32))
+    assert not tern.any() and s == 0
+    g = np.array([2.0, -2.0, 1.0], dtype=np.float32)
+    u = np.array([0.999, 0.0, 0.5], dtype=np.float32)        # p = 1, 1, 0.5 ; u < p strict
+    tern, s = O.ternary_stochastic_quantize(g, u)
+    assert s == 2 and tern.tolist() == [1, -1, 0]
+
+
+# ------------------------------------------------------------------ averaging
+def test_average_of_identical_workers_and_single_worker():
+    rng = np.random.default_rng(6)
+    v = rng.standard_normal(300).astype(np.float32)
+    tern, s, _, _ = O.threshold_quantize(v)
+    one = O.decode_average(tern[None], np.array([s]))
+    assert np.array_equal(one, float(s) * tern)
+    many = O.decode_average(np.stack([tern] * 5), np.array([s] * 5, dtype=np.float32))
+    assert np.allclose(many, one, rtol=1e-15, atol=0)
+    # two different workers: plain mean of the two decoded vectors
+    v2 = rng.standard_normal(300).astype(np.float32) * 3
+    tern2, s2, _, _ = O.threshold_quantize(v2)
+    both = O.decode_average(np.stack([tern, tern2]), np.array([s, s2]))
+    assert np.allclose(both, (float(s) * tern + float(s2) * tern2) / 2, rtol=1e-15, atol=0)
+
+
+# ------------------------------------------------------------------ closed-form updates
+def _argmin_convex(fun, lo, hi, iters=200):
+    for _ in range(iters):
+        a = lo + (hi - lo) / 3
+        b = hi - (hi - lo) / 3
+        if fun(a) < fun(b):
+            hi = b
+        else:
+            lo = a
+    return 0.5 * (lo + hi)
+
+
+def test_cmd_closed_form_is_the_argmin():
+    # minimise eta*q*x + eta*lambda*|x| + H/2 (x - x_t)^2 coordinate-wise (QCMD objective)
+    rng = np.random.default_rng(7)
+    lam, eta, delta = np.float32(0.05), np.float32(0.3), np.float32(1e-3)
+    for _ in range(60):
+        q, xt, h = rng.standard_normal() * 0.3, rng.standard_normal() * 0.2, rng.random()
+        x_new, h_new, a = O.cmd_step(np.array([q]), np.array([xt]), np.array([h]), lam, eta, delta)
+        H = float(delta) + math.sqrt(h + q * q)
+        assert h_new[0] == pytest.approx(h + q * q, rel=1e-15)
+        f = lambda x: float(eta) * q * x + float(eta) * float(lam) * abs(x) + 0.5 * H * (x - xt) ** 2
+        best = _argmin_convex(f, -5.0, 5.0)
+        assert x_new[0] == pytest.approx(best, abs=1e-7)
+        assert f(x_new[0]) <= f(best) + 1e-15
+        assert (x_new[0] == 0.0) == (a[0] <= float(lam))
+
+
+def test_rda_closed_form_is_the_argmin():
+    # minimise eta*(z/t)*x + eta*lambda*|x| + H x^2 / (2t)  (QRDA objective)
+    rng = np.random.default_rng(8)
+    lam, eta, delta = np.float32(0.05), np.float32(0.3), np.float32(1e-3)
+    for _ in range(60):
+        t = int(rng.integers(1, 50))
+        q, z0, h = rng.standard_normal() * 0.3, rng.standard_normal() * t * 0.05, rng.random()
+        x_new, h_new, z_new, a = O.rda_step(np.array([q]), np.array([h]), np.array([z0]), t, lam, eta, delta)
+        z = z0 + q
+        H = float(delta) + math.sqrt(h + q * q)
+        assert z_new[0] == pytest.approx(z, rel=1e-15)
+        f = lambda x: float(eta) * (z / t) * x + float(eta) * float(lam) * abs(x) + H * x * x / (2 * t)
+        best = _argmin_convex(f, -50.0, 50.0)
+        assert x_new[0] == pytest.approx(best, abs=1e-6)
+        assert f(x_new[0]) <= f(best) + 1e-15
+        assert (x_new[0] == 0.0) == (abs(z) / t <= float(lam))
+
+
+def test_exact_sparsity_rules():
+    lam, eta, delta = np.float32(0.01), np.float32(0.1), np.float32(1e-8)
+    q = np.array([0.0099, -0.0099, 0.0101, -0.0101, 0.0])
+    # QCMD from x_t = 0, h = 0: zero iff |q| <= lambda
+    x_new, _, _ = O.cmd_step(q, np.zeros(5), np.zeros(5), lam, eta, delta)
+    assert (x_new == 0).tolist() == [True, True, False, False, True]
+    assert np.sign(x_new[2]) == -1 and np.sign(x_new[3]) == 1
+    assert not np.signbit(x_new).any() or (x_new[np.signbit(x_new)] != 0).all()   # zeros are +0.0
+    # QRDA: zero iff |z|/t <= lambda
+    x_new, _, z_new, _ = O.rda_step(q, np.zeros(5), np.zeros(5), 1, lam, eta, delta)
+    assert (x_new == 0).tolist() == [True, True, False, False, True]
+    x_new, _, _, _ = O.rda_step(np.zeros(5), np.ones(5), np.array([0.5, -0.5, 0.0499, -0.0499, 0.0501]), 5, lam, eta, delta)
+    assert (x_new == 0).tolist() == [False, False, True, True, False]
+
+
+def test_reduces_to_diagonal_adagrad():
+    # Q = identity, lambda = 0, M = 1: QCMD is torch.optim.Adagrad(lr=eta, eps=delta).
+    rng = np.random.default_rng(9)
+    d, steps, eta, delta = 50, 25, 0.1, 1e-3
+    p = torch.zeros(d, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adagrad([p], lr=eta, eps=delta, lr_decay=0.0, initial_accumulator_value=0.0)
+    x = np.zeros(d)
+    h = np.zeros(d)
+    for t in range(1, steps + 1):
+        g = rng.standard_normal((1, d)).astype(np.float32)
+        out = O.step(O.RULE_CMD, g, x, h, None, t, 0.0, eta, delta, quantizer=O.QUANT_NONE)
+        x, h = out["x"], out["h"]
+        p.grad = torch.from_numpy(g[0].astype(np.float64))
+        opt.step()
+        # eta and delta are fp32 at the boundary, so agreement is to fp32 rounding of the scalars
+        assert np.allclose(x, p.detach().numpy(), rtol=1e-6, atol=1e-12)
+
+
+def test_accumulator_satisfies_lemma_1():
+    # (1/2) sum_t ||q_t||^2_{psi*_t} <= sum_i ||q_{1:T,i}||_2 with H_t including q_t.
+    rng = np.random.default_rng(10)
+    d, M, T = 200, 3, 40
+    x = np.zeros(d)
+    h = np.zeros(d)
+    lhs = 0.0
+    delta = np.float32(1e-8)
+    for t in range(1, T + 1):
+        g = rng.standard_normal((M, d)).astype(np.float32)
+        out = O.step(O.RULE_CMD, g, x, h, None, t, 1e-3, 0.1, delta)
+        x, h, q = out["x"], out["h"], out["q"]
+        lhs += float((q * q / (float(delta) + np.sqrt(h))).sum())
+    assert 0.5 * lhs <= float(np.sqrt(h).sum()) * (1 + 1e-12)
+
+
+def test_fused_step_composes_its_parts():
+    # a planted dropped 1/M, wrong sign or missing h update would break these relations
+    rng = np.random.default_rng(14)
+    d, M = 500, 4
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    x0 = rng.standard_normal(d) * 0.1
+    h0 = rng.random(d)
+    z0 = rng.standard_normal(d) * 0.1
+    out = O.step(O.RULE_RDA, g, x0, h0, z0, 16, 1e-3, 0.1, 1e-8)
+    quant = out["quant"]
+    manual_q = sum(float(quant["scales"][m]) * O.unpack_codes(quant["codes"][m], d) for m in range(M)) / M
+    assert np.allclose(out["q"], manual_q, rtol=1e-14, atol=0)
+    assert np.allclose(out["z"], z0 + manual_q, rtol=1e-14)
+    assert np.allclose(out["h"], h0 + manual_q ** 2, rtol=1e-14)
+    assert np.mean(out["x"] == 0) > 0.0                      # some exact zeros
+    nzmask = out["x"] != 0
+    assert (np.sign(out["x"][nzmask]) == -np.sign(out["z"][nzmask])).all()
