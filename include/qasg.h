@@ -1,0 +1,194 @@
+/* libqasg - the per-iteration hot path of QCMD adagrad / QRDA adagrad on one GPU.
+ *
+ * Paper: "Quantized Adaptive Subgradient Algorithms and Their Applications"
+ * (arXiv 2208.05631).  One iteration of its Algorithm 1, with the M workers simulated on
+ * one device: every worker's fp32 gradient is quantized to ternary codes and a scale,
+ * the codes are decoded and averaged (Eq. SynQ_t), the diagonal AdaGrad accumulator
+ * H_t = delta*I + diag(c_t) is updated from the quantized gradient, and the closed-form
+ * L1-proximal update is applied (Eq. QCMD or Eq. QRDA).  The averaged gradient is not
+ * re-quantized (the one-way variant marked with a dagger in Section 5).
+ *
+ * Conventions for every entry point
+ *   - "device pointer": memory of the context's device, owned by the caller, at least
+ *     16-byte aligned unless stated, not overlapping any other argument.  "host
+ *     pointer": ordinary or pinned host memory.
+ *   - Calls validate their arguments on the host, enqueue their kernels on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream) and return without
+ *     waiting.  An argument error returns a status other than QASG_OK and enqueues
+ *     nothing.  Conditions found on the device (a non-finite gradient, an invalid
+ *     code) are reported later by qasg_last_async_status.
+ *   - One context must not be used from two streams at the same time: its workspace
+ *     (per-worker statistics, partial sums, code scratch) is shared by all calls.
+ *   - Step index t is 1-based.  1 <= M <= 64.  1 <= d <= 2^34.
+ *   - There is no CPU implementation behind this interface.
+ */
+#ifndef QASG_H_
+#define QASG_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qasg_ctx qasg_ctx; /* opaque; owns only its workspace */
+
+typedef enum {
+  QASG_OK = 0,
+  QASG_ERR_INVALID_ARG = 1, /* NULL pointer, size or parameter out of range           */
+  QASG_ERR_ALIGNMENT = 2,   /* pointer or leading dimension not aligned as required   */
+  QASG_ERR_WORKSPACE = 3,   /* d or M beyond what the context was created for         */
+  QASG_ERR_CUDA = 4,        /* a CUDA runtime call failed                             */
+  QASG_ERR_TIMEOUT = 5,     /* reserved: a bounded device-side wait ran out           */
+  QASG_ERR_NONFINITE = 6,   /* (async) a gradient held NaN or Inf                     */
+  QASG_ERR_BAD_CODE = 7     /* (async) a packed code word held the unused value 3     */
+} qasg_status;
+
+/* The quantization function Q(.) applied to each worker's gradient. */
+typedef enum {
+  /* Q_Delta of Section 3.4 with the threshold of Section 3.5:
+   * Delta = thr_coef/d * sum|v_i|; code +1 if v > Delta, -1 if v < -Delta, 0 if
+   * |v| <= Delta; scale s = mean of |v_i| over the non-zero codes.  Deterministic. */
+  QASG_Q_THRESHOLD = 0,
+  /* The unbiased ternary quantizer the paper compares with (Section 3.4, first
+   * paragraph): scale s = max|v_i|; code sign(v_i) with probability |v_i|/s, else 0.
+   * Randomness: Philox4x32-10 (Salmon et al., SC'11), key (seed lo, seed hi), counter
+   * (i>>2, m, t lo, t hi), coordinate i uses output word i&3, u = (word>>8) * 2^-24,
+   * non-zero iff u < |v_i|/s in fp32. */
+  QASG_Q_TERNARY_STOCH = 1
+} qasg_quantizer;
+
+typedef enum {
+  QASG_RULE_CMD = 0, /* Eq. QCMD: soft-threshold composite mirror descent           */
+  QASG_RULE_RDA = 1  /* Eq. QRDA: dual averaging with closed-form truncation        */
+} qasg_rule;
+
+typedef struct {
+  uint32_t struct_size; /* sizeof(qasg_params), checked                              */
+  uint32_t quantizer;   /* qasg_quantizer                                            */
+  float thr_coef;       /* 0.75 in Section 3.5; > 0                                  */
+  float lambda;         /* L1 coefficient, >= 0                                      */
+  float eta;            /* learning rate, > 0                                        */
+  float delta;          /* the delta of H_t = delta*I + diag(c_t), > 0               */
+  uint64_t seed;        /* Philox key (stochastic quantizer only)                    */
+} qasg_params;
+
+/* Flags of qasg_create. */
+#define QASG_CREATE_NO_CODE_SCRATCH 1u /* qasg_step will always be given codes_out   */
+
+/* Creates a context on CUDA device `device` able to serve calls with d <= d_max and
+ * M <= M_max.  Allocates the whole workspace here (a few hundred KB of statistics, and,
+ * unless QASG_CREATE_NO_CODE_SCRATCH, M_max * qasg_code_words(d_max) * 4 bytes of code
+ * scratch); no other call allocates device memory.  On error *out is NULL. */
+qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_max,
+                        uint32_t flags);
+/* Frees the workspace.  The caller must have synchronized the streams it used. */
+qasg_status qasg_destroy(qasg_ctx* ctx);
+
+/* Number of 32-bit code words one worker's d codes occupy: ceil(d/16)
+ * (Section 3.5 "Encode": 2 bits per coordinate). */
+uint64_t qasg_code_words(uint64_t d);
+
+/* Workers' side of Algorithm 1 ("Quantize ... the gradients", with the selection S
+ * keeping every coordinate): quantizes each of the M gradients and packs the codes.
+ *   g          device, fp32 [M][ld_g] row-major, row m = gradient of worker m; ld_g >= d,
+ *              ld_g a multiple of 4 (so every row is 16-byte aligned).
+ *   codes      device, uint32 [M][qasg_code_words(d)]; coordinate i of worker m is in
+ *              word i>>4 at bits 2*(i&15), 2*(i&15)+1: 0 -> 0, 1 -> +1, 2 -> -1; unused
+ *              tail bits are written as 0.
+ *   scales     device, fp32 [M]: s_m.
+ *   thresholds device, fp32 [M] or NULL: Delta_m (0 for the stochastic quantizer).
+ *   counts     device, uint64 [M] or NULL: number of non-zero codes of worker m.
+ * Delta_m and s_m come from sums taken in a fixed order (4096-coordinate tiles, fp64,
+ * pairwise), so they do not depend on the launch shape. */
+qasg_status qasg_quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g,
+                               uint32_t M, uint64_t t, const qasg_params* params,
+                               uint32_t* codes, float* scales, float* thresholds,
+                               uint64_t* counts, void* stream);
+
+/* Server's side of Algorithm 1 ("Decode", "Average the quantized gradients",
+ * Eq. SynQ_t): gbar_i = (1/M) * sum_m scales[m] * code_{m,i}.
+ *   codes, scales  device, as written by qasg_quantize_pack.
+ *   gbar           device, fp32 [d]. */
+qasg_status qasg_decode_average(qasg_ctx* ctx, const uint32_t* codes, const float* scales,
+                                uint64_t d, uint32_t M, float* gbar, void* stream);
+
+/* Workers' update of Algorithm 1 for QCMD adagrad (Eq. H_t, Eq. QCMD), from a dense
+ * quantized gradient q (device, fp32 [d]):
+ *   h_i += q_i^2;  H = delta + sqrt(h_i);  u = x_i - (eta/H) q_i;
+ *   x_i = sign(u) * max(|u| - lambda*eta/H, 0), zeros written as +0.0.
+ *   x, h  device, fp32 [d], updated in place (h holds the sum of squares, not its root). */
+qasg_status qasg_cmd_step(qasg_ctx* ctx, const float* q, float* x, float* h, uint64_t d,
+                          uint64_t t, const qasg_params* params, void* stream);
+
+/* Same for QRDA adagrad (Eq. H_t, Eq. QRDA):
+ *   h_i += q_i^2;  z_i += q_i;  H = delta + sqrt(h_i);
+ *   x_i = -sign(z_i) * (t*eta/H) * max(|z_i|/t - lambda, 0), zeros written as +0.0.
+ *   x is written only (its old value is not read); h, z updated in place. */
+qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, float* z,
+                          uint64_t d, uint64_t t, const qasg_params* params, void* stream);
+
+/* The whole iteration, fused: quantize_pack, then decode + average + accumulator +
+ * update in one pass that keeps the averaged gradient in registers, so that per
+ * coordinate the M gradients are read twice (threshold statistics, then codes), the
+ * M/4 code bytes are written and read once, and h, x (z) cross memory once.
+ *   rule        QASG_RULE_CMD (z may be NULL) or QASG_RULE_RDA (z required).
+ *   codes_out   device uint32 [M][code_words(d)] or NULL to use the context's scratch.
+ *   scales_out  device fp32 [M] or NULL. */
+qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
+                      uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h,
+                      float* z, uint32_t* codes_out, float* scales_out, void* stream);
+
+/* qasg_step for callers whose data lives in host memory.  Copies g (M rows of d floats,
+ * row stride ld_g) and the state from the host buffers into the caller's device staging
+ * buffers, runs qasg_step there, and copies the new state back, all on `stream`; returns
+ * without waiting (synchronize the stream before reading the host buffers).
+ *   g_host, x_host, h_host, z_host   host pointers (pinned memory for asynchronous
+ *                                    copies); z_host NULL for QASG_RULE_CMD.  For
+ *                                    QASG_RULE_RDA x_host is output only.
+ *   g_dev [M][ld_g], x_dev, h_dev, z_dev [d]   device staging, as for qasg_step. */
+qasg_status qasg_step_host(qasg_ctx* ctx, qasg_rule rule, const float* g_host, uint64_t d,
+                           uint64_t ld_g, uint32_t M, uint64_t t, const qasg_params* params,
+                           float* x_host, float* h_host, float* z_host, float* g_dev,
+                           float* x_dev, float* h_dev, float* z_dev, void* stream);
+
+/* Per-worker minibatch gradient of logistic regression, the linear-model workload of
+ * Section 5.1 (Eq. of Section 3.1: the minibatch average of per-sample gradients):
+ *   g_m = (1/B) sum_{j in batch m} -y_j * sigmoid(-y_j <a_j, x>) * a_j ,  y_j in {-1,+1}.
+ * The L1 term is left to the proximal update.
+ *   X          device, fp32 [n_rows][d] row-major, d a multiple of 4.
+ *   y          device, fp32 [n_rows].
+ *   shard_row0 host, uint64 [M+1]: worker m owns rows [shard_row0[m], shard_row0[m+1]).
+ *   batch_rows device, uint32 [M][B] global row ids, or NULL for the default minibatch:
+ *              B consecutive rows of the shard starting at ((t-1)*B) mod shard size,
+ *              wrapping inside the shard.
+ *   x          device, fp32 [d].
+ *   g          device, fp32 [M][ld_g], rows fully overwritten (first d entries). */
+qasg_status qasg_logreg_grad_dense(qasg_ctx* ctx, const float* X, const float* y,
+                                   uint64_t n_rows, uint64_t d, uint32_t M,
+                                   const uint64_t* shard_row0, const uint32_t* batch_rows,
+                                   uint32_t B, uint64_t t, const float* x, float* g,
+                                   uint64_t ld_g, void* stream);
+
+/* Same for a CSR matrix: rowptr device int64 [n_rows+1], colidx device int32 [nnz]
+ * (0 <= colidx < d), vals device fp32 [nnz].  g rows are zeroed, then accumulated with
+ * atomic adds (the summation order inside one coordinate is not fixed). */
+qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
+                                 const float* vals, const float* y, uint64_t n_rows,
+                                 uint64_t d, uint32_t M, const uint64_t* shard_row0,
+                                 const uint32_t* batch_rows, uint32_t B, uint64_t t,
+                                 const float* x, float* g, uint64_t ld_g, void* stream);
+
+/* Waits for `stream`, then returns and clears the conditions kernels recorded since
+ * the last call: QASG_ERR_NONFINITE, QASG_ERR_BAD_CODE, QASG_ERR_CUDA, else QASG_OK. */
+qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched since it was created. */
+uint64_t qasg_launch_count(const qasg_ctx* ctx);
+
+const char* qasg_status_string(qasg_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QASG_H_ */

@@ -1,0 +1,332 @@
+// C-ABI layer of libqasg: context, argument validation, sequencing of the passes.
+#include "../../include/qasg.h"
+
+#include <new>
+
+#include "qasg_internal.h"
+
+using namespace qasg;
+
+struct qasg_ctx {
+  int device;
+  uint64_t d_max;
+  uint32_t M_max;
+  LaunchShape shape;
+  Workspace ws;
+  uint32_t* code_scratch;   // [M_max][code_words(d_max)] or NULL
+  float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
+  uint64_t launches;
+};
+
+namespace {
+
+constexpr uint64_t kMaxD = 1ull << 34;
+constexpr uint64_t kLogregEntries = 1ull << 20;  // M * B of one gradient call
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+qasg_status check_params(const qasg_params* p, bool need_update) {
+  if (!p || p->struct_size != sizeof(qasg_params)) return QASG_ERR_INVALID_ARG;
+  if (p->quantizer != QASG_Q_THRESHOLD && p->quantizer != QASG_Q_TERNARY_STOCH) return QASG_ERR_INVALID_ARG;
+  if (!(p->thr_coef > 0.f) || !isfinite(p->thr_coef)) return QASG_ERR_INVALID_ARG;
+  if (need_update) {
+    if (!(p->lambda >= 0.f) || !isfinite(p->lambda)) return QASG_ERR_INVALID_ARG;
+    if (!(p->eta > 0.f) || !isfinite(p->eta)) return QASG_ERR_INVALID_ARG;
+    if (!(p->delta > 0.f) || !isfinite(p->delta)) return QASG_ERR_INVALID_ARG;
+  }
+  return QASG_OK;
+}
+
+qasg_status check_shape(const qasg_ctx* ctx, uint64_t d, uint32_t M) {
+  if (!ctx) return QASG_ERR_INVALID_ARG;
+  if (d < 1 || d > kMaxD || M < 1 || M > static_cast<uint32_t>(kMaxWorkers)) return QASG_ERR_INVALID_ARG;
+  if (d > ctx->d_max || M > ctx->M_max) return QASG_ERR_WORKSPACE;
+  return QASG_OK;
+}
+
+qasg_status enter(const qasg_ctx* ctx) {
+  return cudaSetDevice(ctx->device) == cudaSuccess ? QASG_OK : QASG_ERR_CUDA;
+}
+
+qasg_status leave() { return cudaGetLastError() == cudaSuccess ? QASG_OK : QASG_ERR_CUDA; }
+
+StepScalars scalars(const qasg_params* p, uint64_t t) {
+  StepScalars sc;
+  sc.lambda = p->lambda;
+  sc.eta = p->eta;
+  sc.delta = p->delta;
+  sc.t = static_cast<float>(t);
+  return sc;
+}
+
+// Passes A and B on validated arguments.
+void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint64_t t,
+                   const qasg_params* p, uint32_t* codes, float* scales, float* thresholds,
+                   uint64_t* counts, cudaStream_t stream) {
+  const Geometry geo = make_geometry(d, ld_g, M);
+  unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
+  if (p->quantizer == QASG_Q_THRESHOLD) {
+    ctx->launches += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream);
+    ctx->launches += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream);
+  } else {
+    ctx->launches += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream);
+    ctx->launches += launch_stochastic_codes(g, geo, p->seed, t, ctx->ws, codes, scales, counts_out,
+                                             ctx->shape, stream);
+    if (thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
+  }
+}
+
+qasg_status check_gradient(const float* g, uint64_t d, uint64_t ld_g) {
+  if (!g) return QASG_ERR_INVALID_ARG;
+  if (ld_g < d) return QASG_ERR_INVALID_ARG;
+  if ((ld_g & 3u) || !aligned16(g)) return QASG_ERR_ALIGNMENT;
+  return QASG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_max, uint32_t flags) {
+  if (!out) return QASG_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (d_max < 1 || d_max > kMaxD || M_max < 1 || M_max > static_cast<uint32_t>(kMaxWorkers))
+    return QASG_ERR_INVALID_ARG;
+  if (cudaSetDevice(device) != cudaSuccess) return QASG_ERR_CUDA;
+  qasg_ctx* ctx = new (std::nothrow) qasg_ctx();
+  if (!ctx) return QASG_ERR_CUDA;
+  ctx->device = device;
+  ctx->d_max = d_max;
+  ctx->M_max = M_max;
+  ctx->launches = 0;
+  query_launch_shape(&ctx->shape);
+  const size_t slots = static_cast<size_t>(M_max) * kMaxChunks;
+  bool ok = true;
+  ok &= cudaMalloc(&ctx->ws.part_sum, slots * sizeof(double)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.part_max, slots * sizeof(uint32_t)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.part_cnt, slots * sizeof(unsigned long long)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.thresholds, kMaxWorkers * sizeof(float)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.scales, kMaxWorkers * sizeof(float)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.counts, kMaxWorkers * sizeof(unsigned long long)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.ticket, 64) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.status, 64) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->logreg_ws, kLogregEntries * 2 * sizeof(float)) == cudaSuccess;
+  if (ok && !(flags & QASG_CREATE_NO_CODE_SCRATCH))
+    ok &= cudaMalloc(&ctx->code_scratch, static_cast<size_t>(M_max) * qasg_code_words(d_max) * 4) == cudaSuccess;
+  if (ok) {
+    ok &= cudaMemset(ctx->ws.ticket, 0, 64) == cudaSuccess;
+    ok &= cudaMemset(ctx->ws.status, 0, 64) == cudaSuccess;
+    ok &= cudaMemset(ctx->ws.thresholds, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
+    ok &= cudaMemset(ctx->ws.scales, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    qasg_destroy(ctx);
+    return QASG_ERR_CUDA;
+  }
+  *out = ctx;
+  return QASG_OK;
+}
+
+qasg_status qasg_destroy(qasg_ctx* ctx) {
+  if (!ctx) return QASG_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaFree(ctx->ws.part_sum);
+  cudaFree(ctx->ws.part_max);
+  cudaFree(ctx->ws.part_cnt);
+  cudaFree(ctx->ws.thresholds);
+  cudaFree(ctx->ws.scales);
+  cudaFree(ctx->ws.counts);
+  cudaFree(ctx->ws.ticket);
+  cudaFree(ctx->ws.status);
+  cudaFree(ctx->logreg_ws);
+  cudaFree(ctx->code_scratch);
+  delete ctx;
+  return QASG_OK;
+}
+
+uint64_t qasg_code_words(uint64_t d) { return (d + 15) >> 4; }
+
+qasg_status qasg_quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                               uint64_t t, const qasg_params* params, uint32_t* codes, float* scales,
+                               float* thresholds, uint64_t* counts, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, false);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (!codes || !scales || t < 1) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(codes)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales, thresholds, counts,
+                static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_decode_average(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d,
+                                uint32_t M, float* gbar, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st != QASG_OK) return st;
+  if (!codes || !scales || !gbar) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(codes) || !aligned16(gbar)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  ctx->launches += launch_decode_average(codes, scales, d, M, gbar, ctx->ws.status, ctx->shape,
+                                         static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_cmd_step(qasg_ctx* ctx, const float* q, float* x, float* h, uint64_t d, uint64_t t,
+                          const qasg_params* params, void* stream) {
+  qasg_status st = check_shape(ctx, d, 1);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st != QASG_OK) return st;
+  if (!q || !x || !h || t < 1) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(x) || !aligned16(h)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  ctx->launches += launch_dense_update(QASG_RULE_CMD, q, d, x, h, nullptr, scalars(params, t), ctx->shape,
+                                       static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, float* z, uint64_t d,
+                          uint64_t t, const qasg_params* params, void* stream) {
+  qasg_status st = check_shape(ctx, d, 1);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st != QASG_OK) return st;
+  if (!q || !x || !h || !z || t < 1) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(x) || !aligned16(h) || !aligned16(z)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  ctx->launches += launch_dense_update(QASG_RULE_RDA, q, d, x, h, z, scalars(params, t), ctx->shape,
+                                       static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                      uint64_t t, const qasg_params* params, float* x, float* h, float* z,
+                      uint32_t* codes_out, float* scales_out, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
+  if (!x || !h || t < 1 || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(h) || (z && !aligned16(z)) || (codes_out && !aligned16(codes_out)))
+    return QASG_ERR_ALIGNMENT;
+  uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
+  if (!codes) return QASG_ERR_WORKSPACE;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
+  ctx->launches += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
+                                        ctx->ws.status, ctx->shape, s);
+  return leave();
+}
+
+qasg_status qasg_step_host(qasg_ctx* ctx, qasg_rule rule, const float* g_host, uint64_t d, uint64_t ld_g,
+                           uint32_t M, uint64_t t, const qasg_params* params, float* x_host, float* h_host,
+                           float* z_host, float* g_dev, float* x_dev, float* h_dev, float* z_dev,
+                           void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st != QASG_OK) return st;
+  if (!g_host || !x_host || !h_host || !g_dev || !x_dev || !h_dev) return QASG_ERR_INVALID_ARG;
+  if (rule == QASG_RULE_RDA && (!z_host || !z_dev)) return QASG_ERR_INVALID_ARG;
+  if (ld_g < d) return QASG_ERR_INVALID_ARG;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t vec = d * sizeof(float);
+  bool ok = true;
+  ok &= cudaMemcpy2DAsync(g_dev, ld_g * sizeof(float), g_host, ld_g * sizeof(float), vec, M,
+                          cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (rule == QASG_RULE_CMD) ok &= cudaMemcpyAsync(x_dev, x_host, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(h_dev, h_host, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (rule == QASG_RULE_RDA) ok &= cudaMemcpyAsync(z_dev, z_host, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return QASG_ERR_CUDA;
+  }
+  st = qasg_step(ctx, rule, g_dev, d, ld_g, M, t, params, x_dev, h_dev, z_dev, nullptr, nullptr, stream);
+  if (st != QASG_OK) return st;
+  ok &= cudaMemcpyAsync(x_host, x_dev, vec, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(h_host, h_dev, vec, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (rule == QASG_RULE_RDA) ok &= cudaMemcpyAsync(z_host, z_dev, vec, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return QASG_ERR_CUDA;
+  }
+  return QASG_OK;
+}
+
+static qasg_status check_logreg(qasg_ctx* ctx, const float* y, uint64_t n_rows, uint64_t d, uint32_t M,
+                                const uint64_t* shard_row0, uint32_t B, uint64_t t, const float* x,
+                                const float* g, uint64_t ld_g) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st != QASG_OK) return st;
+  if (!y || !shard_row0 || !x || !g || B < 1 || t < 1 || n_rows < 1) return QASG_ERR_INVALID_ARG;
+  if (ld_g < d) return QASG_ERR_INVALID_ARG;
+  if ((ld_g & 3u) || !aligned16(g) || !aligned16(x)) return QASG_ERR_ALIGNMENT;
+  if (static_cast<uint64_t>(M) * B > kLogregEntries) return QASG_ERR_WORKSPACE;
+  for (uint32_t m = 0; m < M; ++m)
+    if (shard_row0[m + 1] <= shard_row0[m] || shard_row0[m + 1] > n_rows) return QASG_ERR_INVALID_ARG;
+  if (n_rows > 0xffffffffull) return QASG_ERR_INVALID_ARG;
+  return QASG_OK;
+}
+
+qasg_status qasg_logreg_grad_dense(qasg_ctx* ctx, const float* X, const float* y, uint64_t n_rows, uint64_t d,
+                                   uint32_t M, const uint64_t* shard_row0, const uint32_t* batch_rows,
+                                   uint32_t B, uint64_t t, const float* x, float* g, uint64_t ld_g,
+                                   void* stream) {
+  qasg_status st = check_logreg(ctx, y, n_rows, d, M, shard_row0, B, t, x, g, ld_g);
+  if (st != QASG_OK) return st;
+  if (!X) return QASG_ERR_INVALID_ARG;
+  if ((d & 3u) || !aligned16(X)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  ctx->launches += launch_logreg_dense(X, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->logreg_ws,
+                                       ctx->shape, static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
+                                 const float* vals, const float* y, uint64_t n_rows, uint64_t d, uint32_t M,
+                                 const uint64_t* shard_row0, const uint32_t* batch_rows, uint32_t B,
+                                 uint64_t t, const float* x, float* g, uint64_t ld_g, void* stream) {
+  qasg_status st = check_logreg(ctx, y, n_rows, d, M, shard_row0, B, t, x, g, ld_g);
+  if (st != QASG_OK) return st;
+  if (!rowptr || !colidx || !vals) return QASG_ERR_INVALID_ARG;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  ctx->launches += launch_logreg_csr(rowptr, colidx, vals, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
+                                     ctx->shape, static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream) {
+  if (!ctx) return QASG_ERR_INVALID_ARG;
+  if (enter(ctx) != QASG_OK) return QASG_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned int flags = 0;
+  if (cudaMemcpyAsync(&flags, ctx->ws.status, sizeof(flags), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaMemsetAsync(ctx->ws.status, 0, sizeof(flags), s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) {
+    cudaGetLastError();
+    return QASG_ERR_CUDA;
+  }
+  if (flags & kFlagNonFinite) return QASG_ERR_NONFINITE;
+  if (flags & kFlagBadCode) return QASG_ERR_BAD_CODE;
+  return QASG_OK;
+}
+
+uint64_t qasg_launch_count(const qasg_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* qasg_status_string(qasg_status s) {
+  switch (s) {
+    case QASG_OK: return "ok";
+    case QASG_ERR_INVALID_ARG: return "invalid argument";
+    case QASG_ERR_ALIGNMENT: return "pointer or leading dimension not aligned";
+    case QASG_ERR_WORKSPACE: return "size beyond the context's workspace";
+    case QASG_ERR_CUDA: return "CUDA runtime error";
+    case QASG_ERR_TIMEOUT: return "device-side wait timed out";
+    case QASG_ERR_NONFINITE: return "non-finite gradient";
+    case QASG_ERR_BAD_CODE: return "invalid code value in packed words";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

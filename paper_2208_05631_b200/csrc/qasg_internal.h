@@ -1,0 +1,91 @@
+// Internal interface between the C-ABI layer and the kernel launchers of libqasg.
+#ifndef QASG_INTERNAL_H_
+#define QASG_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace qasg {
+
+// Geometry of the fixed-order sums.  A tile is 4 rows x 1024 columns = 4096 consecutive
+// coordinates; 256 threads own 4 adjacent columns each.
+constexpr int kThreads = 256;
+constexpr int kTileRows = 4;
+constexpr int kTileCols = 1024;
+constexpr int kTile = kTileRows * kTileCols;
+// A worker's tiles are cut into at most kMaxChunks aligned groups of `group` tiles
+// (group a power of two).  One CTA reduces one group to one partial; the partials of a
+// worker are combined by one warp.
+constexpr int kMaxChunks = 1024;
+constexpr int kMaxWorkers = 64;
+
+enum : unsigned { kFlagNonFinite = 1u, kFlagBadCode = 2u };
+
+struct Geometry {
+  uint64_t d;       // coordinates per worker
+  uint64_t ld;      // row stride of g in floats
+  uint32_t M;       // workers
+  uint32_t tiles;   // ceil(d / 4096)
+  uint32_t group;   // tiles per chunk, power of two
+  uint32_t log2_group;
+  uint32_t chunks;  // ceil(tiles / group) <= kMaxChunks
+};
+
+Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M);
+
+struct Workspace {
+  double* part_sum;              // [M_max][kMaxChunks] chunk partials of a canonical sum
+  uint32_t* part_max;            // [M_max][kMaxChunks] chunk maxima of |g| (bit patterns)
+  unsigned long long* part_cnt;  // [M_max][kMaxChunks] chunk counts of non-zero codes
+  float* thresholds;             // [M_max] Delta_m
+  float* scales;                 // [M_max] s_m
+  unsigned long long* counts;    // [M_max] non-zero codes
+  unsigned int* ticket;          // grid-completion counter, zero between launches
+  unsigned int* status;          // OR of kFlag*
+};
+
+struct LaunchShape {
+  int sm_count;
+  int reduce_ctas_per_sm;  // resident CTAs per SM for the reduction kernels
+  int update_ctas_per_sm;  // same for the coordinate-wise kernels
+};
+
+struct StepScalars {
+  float lambda, eta, delta, t;
+};
+
+// Each launcher enqueues on `stream` and returns the number of kernels it launched.
+int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
+                   float* thresholds_out, const LaunchShape& shape, cudaStream_t stream);
+int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
+                   const LaunchShape& shape, cudaStream_t stream);
+int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
+                           uint32_t* codes, float* scales_out, unsigned long long* counts_out,
+                           const LaunchShape& shape, cudaStream_t stream);
+int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
+                            const Workspace& ws, uint32_t* codes, float* scales_out,
+                            unsigned long long* counts_out, const LaunchShape& shape,
+                            cudaStream_t stream);
+int launch_decode_update(int rule, const uint32_t* codes, const float* scales, uint64_t d,
+                         uint32_t M, float* x, float* h, float* z, const StepScalars& sc,
+                         unsigned int* status, const LaunchShape& shape, cudaStream_t stream);
+int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
+                          float* gbar, unsigned int* status, const LaunchShape& shape,
+                          cudaStream_t stream);
+int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h, float* z,
+                        const StepScalars& sc, const LaunchShape& shape, cudaStream_t stream);
+
+// margins_ws: device fp32 [M*B] scratch for the per-row coefficients.
+int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
+                        const uint64_t* shard_row0_host, const uint32_t* batch_rows, uint32_t B,
+                        uint64_t t, const float* x, float* g, uint64_t ld_g, float* coef_ws,
+                        const LaunchShape& shape, cudaStream_t stream);
+int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float* vals,
+                      const float* y, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
+                      const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
+                      uint64_t ld_g, const LaunchShape& shape, cudaStream_t stream);
+
+void query_launch_shape(LaunchShape* shape);
+
+}  // namespace qasg
+#endif  // QASG_INTERNAL_H_

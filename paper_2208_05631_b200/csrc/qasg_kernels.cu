@@ -1,0 +1,692 @@
+// Kernels of the quantized adaptive-subgradient step for sm_100a.
+//
+//   pass A  abs_sum_kernel / abs_max_kernel     per-worker sum|g| -> Delta_m, or max|g| -> s_m
+//   pass B  threshold_codes_kernel              ternary codes, packed; s_m = mean of kept |g|
+//           stochastic_codes_kernel             unbiased ternary codes from Philox draws
+//   pass C  decode_update_kernel                decode + average + accumulator + QCMD/QRDA
+//           decode_average_kernel, dense_update_kernel   the same in two unfused halves
+//
+// All three passes are HBM streams.  Passes A and B walk each worker's gradient in
+// 4096-coordinate tiles with 128-bit loads (thread j owns columns 4j..4j+3 of each of
+// the tile's 4 rows) and keep one tile of loads in flight ahead of the arithmetic.  The
+// sums that decide Delta_m and s_m are taken in a fixed order that does not depend on
+// the grid: column sums down the rows, a pairwise tree over the 1024 columns (in-thread,
+// warp butterfly, across warps), a pairwise tree over tiles.  The CTA that finishes last
+// combines the per-chunk partials, so no extra launch or host round trip is needed.
+#include "qasg_internal.h"
+
+namespace qasg {
+
+// ------------------------------------------------------------------ geometry
+Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M) {
+  Geometry geo;
+  geo.d = d;
+  geo.ld = ld;
+  geo.M = M;
+  geo.tiles = static_cast<uint32_t>((d + kTile - 1) / kTile);
+  uint32_t group = 1, lg = 0;
+  while ((geo.tiles + group - 1) / group > static_cast<uint32_t>(kMaxChunks)) {
+    group <<= 1;
+    ++lg;
+  }
+  geo.group = group;
+  geo.log2_group = lg;
+  geo.chunks = (geo.tiles + group - 1) / group;
+  return geo;
+}
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ float4 load_f4(const float* p) {
+  return __ldg(reinterpret_cast<const float4*>(p));
+}
+
+// The four float4 a thread owns in the tile starting at coordinate tile_base.
+// Coordinates >= d read as +0.0 (they neither count nor code).
+__device__ __forceinline__ void load_tile(const float* __restrict__ row, uint64_t tile_base,
+                                          uint64_t d, int j, float4 (&v)[kTileRows]) {
+  if (tile_base + kTile <= d) {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) v[r] = load_f4(row + tile_base + r * kTileCols + 4 * j);
+  } else {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) {
+      const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
+      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i0 < d) {
+        t = load_f4(row + i0);  // stays inside the row: ld is a multiple of 4 and >= d
+        if (i0 + 1 >= d) t.y = 0.f;
+        if (i0 + 2 >= d) t.z = 0.f;
+        if (i0 + 3 >= d) t.w = 0.f;
+      }
+      v[r] = t;
+    }
+  }
+}
+
+// Pairwise tree over the 32 lanes (adjacent pairs first).  Addition commutes bit for bit,
+// so both partners of every exchange hold the same value.
+__device__ __forceinline__ double warp_pair_tree(double v) {
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+  return v;
+}
+
+// Pairwise tree over the 1024 column sums of a tile: v is the thread's sum of its 4
+// columns.  The result is valid in thread 0.  `slot` alternates between calls so that
+// one barrier per tile is enough.
+__device__ __forceinline__ double block_pair_tree(double v, double (*sm)[kThreads / 32], int slot) {
+  v = warp_pair_tree(v);
+  if ((threadIdx.x & 31) == 0) sm[slot][threadIdx.x >> 5] = v;
+  __syncthreads();
+  double r = 0.0;
+  if (threadIdx.x == 0) {
+    const double* a = sm[slot];
+    r = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+  }
+  return r;
+}
+
+// Streaming pairwise summation over the tiles of a chunk (thread 0 only): stack[l] holds
+// the sum of a complete aligned subtree of 2^l tiles.
+__device__ __forceinline__ void tile_push(double* stack, uint32_t k_local, double v) {
+  int lvl = 0;
+  while (k_local & 1u) {
+    v = stack[lvl] + v;
+    k_local >>= 1;
+    ++lvl;
+  }
+  stack[lvl] = v;
+}
+// Completes the chunk's tree after n <= 2^log2_group tiles (missing tiles are +0.0).
+__device__ __forceinline__ double tile_fold(const double* stack, uint32_t n, uint32_t log2_group) {
+  double carry = 0.0;
+  for (uint32_t lvl = 0; lvl <= log2_group; ++lvl)
+    if ((n >> lvl) & 1u) carry = stack[lvl] + carry;
+  return carry;
+}
+
+// Pairwise tree over a worker's kMaxChunks partial slots (slots >= chunks are +0.0),
+// computed by one warp: 32 adjacent slots per lane, then the lane butterfly.
+__device__ __forceinline__ double warp_chunk_tree(const double* part, uint32_t chunks, int lane) {
+  double top[4];
+#pragma unroll 1
+  for (int q = 0; q < 4; ++q) {  // 8 adjacent slots at a time keeps the register count low
+    double v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const uint32_t idx = lane * 32 + q * 8 + k;
+      v[k] = idx < chunks ? __ldcg(part + idx) : 0.0;
+    }
+    top[q] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+  }
+  return warp_pair_tree((top[0] + top[1]) + (top[2] + top[3]));
+}
+
+// True in every thread of the CTA that finishes last.  All global writes this CTA made
+// before the call (by thread 0) are visible to that CTA.
+__device__ __forceinline__ bool grid_last_cta(unsigned int* ticket, bool* sm_flag) {
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int prev = atomicAdd(ticket, 1u);
+    *sm_flag = (prev == gridDim.x - 1);
+  }
+  __syncthreads();
+  const bool last = *sm_flag;
+  if (last) __threadfence();
+  return last;
+}
+
+// ------------------------------------------------------------------ pass A: sum |g|
+__global__ void __launch_bounds__(kThreads)
+abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
+               float* __restrict__ thresholds_out) {
+  __shared__ double sm_warp[2][kThreads / 32];
+  __shared__ double sm_stack[32];
+  __shared__ bool sm_last;
+  const int j = threadIdx.x;
+  const uint32_t n_items = geo.M * geo.chunks;
+  int slot = 0;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
+    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    float4 cur[kTileRows], nxt[kTileRows];
+    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
+    for (uint32_t k = k0; k < k1; ++k) {
+      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
+      double cx = fabsf(cur[0].x), cy = fabsf(cur[0].y), cz = fabsf(cur[0].z), cw = fabsf(cur[0].w);
+#pragma unroll
+      for (int r = 1; r < kTileRows; ++r) {
+        cx += static_cast<double>(fabsf(cur[r].x));
+        cy += static_cast<double>(fabsf(cur[r].y));
+        cz += static_cast<double>(fabsf(cur[r].z));
+        cw += static_cast<double>(fabsf(cur[r].w));
+      }
+      const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
+      slot ^= 1;
+      if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) cur[r] = nxt[r];
+    }
+    if (j == 0)
+      ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = tile_fold(sm_stack, k1 - k0, geo.log2_group);
+  }
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  const int warp = j >> 5, lane = j & 31;
+  for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
+    const double total = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+    if (lane == 0) {
+      const float delta = static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(geo.d));
+      ws.thresholds[m] = delta;
+      if (thresholds_out) thresholds_out[m] = delta;
+      if (!isfinite(total)) atomicOr(ws.status, kFlagNonFinite);
+    }
+  }
+  if (j == 0) *ws.ticket = 0u;
+}
+
+// ------------------------------------------------------------------ pass A': max |g|
+__global__ void __launch_bounds__(kThreads)
+abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
+  __shared__ uint32_t sm_warp[kThreads / 32];
+  __shared__ bool sm_last;
+  const int j = threadIdx.x;
+  const uint32_t n_items = geo.M * geo.chunks;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
+    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    float4 cur[kTileRows], nxt[kTileRows];
+    uint32_t best = 0u;  // bit patterns of non-negative floats order like their values
+    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
+    for (uint32_t k = k0; k < k1; ++k) {
+      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) {
+        best = max(best, __float_as_uint(fabsf(cur[r].x)));
+        best = max(best, __float_as_uint(fabsf(cur[r].y)));
+        best = max(best, __float_as_uint(fabsf(cur[r].z)));
+        best = max(best, __float_as_uint(fabsf(cur[r].w)));
+        cur[r] = nxt[r];
+      }
+    }
+    best = __reduce_max_sync(0xffffffffu, best);
+    __syncthreads();  // the previous item's readers are done with sm_warp
+    if ((j & 31) == 0) sm_warp[j >> 5] = best;
+    __syncthreads();
+    if (j == 0) {
+      uint32_t b = sm_warp[0];
+#pragma unroll
+      for (int w = 1; w < kThreads / 32; ++w) b = max(b, sm_warp[w]);
+      ws.part_max[static_cast<uint64_t>(m) * kMaxChunks + c] = b;
+    }
+  }
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  const int warp = j >> 5, lane = j & 31;
+  for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
+    uint32_t b = 0u;
+    for (uint32_t idx = lane; idx < geo.chunks; idx += 32)
+      b = max(b, __ldcg(ws.part_max + static_cast<uint64_t>(m) * kMaxChunks + idx));
+    b = __reduce_max_sync(0xffffffffu, b);
+    if (lane == 0) {
+      ws.scales[m] = __uint_as_float(b);
+      ws.thresholds[m] = 0.f;
+      if (b >= 0x7f800000u) atomicOr(ws.status, kFlagNonFinite);
+    }
+  }
+  if (j == 0) *ws.ticket = 0u;
+}
+
+// ------------------------------------------------------------------ pass B helpers
+// One code: 1 for +1, 2 for -1, 0 for 0.
+__device__ __forceinline__ uint32_t ternary_code(float v, bool keep) {
+  return keep ? ((__float_as_uint(v) >> 31) + 1u) : 0u;
+}
+
+// Writes the byte holding the codes of coordinates i0..i0+3 of worker row `codes8`.
+__device__ __forceinline__ void store_code_byte(uint8_t* __restrict__ codes8, uint64_t i0,
+                                                uint64_t row_bytes, uint32_t byte) {
+  const uint64_t b = i0 >> 2;
+  if (b < row_bytes) codes8[b] = static_cast<uint8_t>(byte);
+}
+
+// Sums per-thread counts over the CTA; the result is valid in thread 0.
+__device__ __forceinline__ unsigned long long block_count(uint32_t cnt, uint32_t* sm_cnt) {
+  cnt = __reduce_add_sync(0xffffffffu, cnt);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sm_cnt[threadIdx.x >> 5] = cnt;
+  __syncthreads();
+  unsigned long long total = 0;
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) total += sm_cnt[w];
+  }
+  return total;
+}
+
+// Last-CTA epilogue shared by both code kernels: per-worker totals of the counts, and for
+// the threshold quantizer the scale s_m = P_m / n_m.
+template <bool kThreshold>
+__device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspace& ws,
+                                             float* scales_out, unsigned long long* counts_out) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
+    unsigned long long n = 0;
+    for (uint32_t idx = lane; idx < geo.chunks; idx += 32)
+      n += __ldcg(ws.part_cnt + static_cast<uint64_t>(m) * kMaxChunks + idx);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
+    float scale;
+    if (kThreshold) {
+      const double picked = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+      scale = n ? static_cast<float>(picked / static_cast<double>(n)) : 0.f;
+    } else {
+      scale = ws.scales[m];
+    }
+    if (lane == 0) {
+      ws.counts[m] = n;
+      if (kThreshold) ws.scales[m] = scale;
+      if (scales_out) scales_out[m] = scale;
+      if (counts_out) counts_out[m] = n;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ pass B: Q_Delta codes
+__global__ void __launch_bounds__(kThreads)
+threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
+                       uint32_t* __restrict__ codes, float* __restrict__ scales_out,
+                       unsigned long long* __restrict__ counts_out) {
+  __shared__ double sm_warp[2][kThreads / 32];
+  __shared__ double sm_stack[32];
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ bool sm_last;
+  const int j = threadIdx.x;
+  const uint32_t n_items = geo.M * geo.chunks;
+  const uint64_t row_words = (geo.d + 15) >> 4;
+  int slot = 0;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
+    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+    uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
+    const float delta = ws.thresholds[m];
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    uint32_t cnt = 0;
+    float4 cur[kTileRows], nxt[kTileRows];
+    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
+    for (uint32_t k = k0; k < k1; ++k) {
+      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
+      const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) {
+        const float4 t = cur[r];
+        const float ax = fabsf(t.x), ay = fabsf(t.y), az = fabsf(t.z), aw = fabsf(t.w);
+        const bool kx = ax > delta, ky = ay > delta, kz = az > delta, kw = aw > delta;
+        if (kx) cx += static_cast<double>(ax);
+        if (ky) cy += static_cast<double>(ay);
+        if (kz) cz += static_cast<double>(az);
+        if (kw) cw += static_cast<double>(aw);
+        cnt += static_cast<uint32_t>(kx) + static_cast<uint32_t>(ky) + static_cast<uint32_t>(kz) +
+               static_cast<uint32_t>(kw);
+        const uint32_t byte = ternary_code(t.x, kx) | (ternary_code(t.y, ky) << 2) |
+                              (ternary_code(t.z, kz) << 4) | (ternary_code(t.w, kw) << 6);
+        store_code_byte(codes8, tile_base + r * kTileCols + 4 * j, row_words * 4, byte);
+        cur[r] = nxt[r];
+      }
+      const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
+      slot ^= 1;
+      if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
+    }
+    const unsigned long long total = block_count(cnt, sm_cnt);
+    if (j == 0) {
+      const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
+      ws.part_sum[p] = tile_fold(sm_stack, k1 - k0, geo.log2_group);
+      ws.part_cnt[p] = total;
+    }
+  }
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  finish_codes<true>(geo, ws, scales_out, counts_out);
+  if (j == 0) *ws.ticket = 0u;
+}
+
+// ------------------------------------------------------------------ Philox4x32-10
+// Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3" (SC'11):
+// ten rounds of  (c0,c1,c2,c3) <- (hi(M1*c2)^c1^k0, lo(M1*c2), hi(M0*c0)^c3^k1, lo(M0*c0)),
+// the key advancing by the Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+  constexpr uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u;
+  constexpr uint32_t kW0 = 0x9E3779B9u, kW1 = 0xBB67AE85u;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(kM0, c.x), lo0 = kM0 * c.x;
+    const uint32_t hi1 = __umulhi(kM1, c.z), lo1 = kM1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += kW0;
+    k1 += kW1;
+  }
+  return c;
+}
+
+__device__ __forceinline__ float philox_uniform(uint32_t word) {
+  return static_cast<float>(word >> 8) * 5.9604644775390625e-08f;  // 2^-24, exact
+}
+
+// ------------------------------------------------------------------ pass B': stochastic codes
+__global__ void __launch_bounds__(kThreads)
+stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
+                        Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
+                        unsigned long long* __restrict__ counts_out) {
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ bool sm_last;
+  const int j = threadIdx.x;
+  const uint32_t n_items = geo.M * geo.chunks;
+  const uint64_t row_words = (geo.d + 15) >> 4;
+  const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
+  const uint32_t t_lo = static_cast<uint32_t>(t), t_hi = static_cast<uint32_t>(t >> 32);
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
+    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+    uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
+    const float scale = ws.scales[m];
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    uint32_t cnt = 0;
+    float4 cur[kTileRows], nxt[kTileRows];
+    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
+    for (uint32_t k = k0; k < k1; ++k) {
+      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
+      const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) {
+        const float4 v = cur[r];
+        const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
+        const uint4 w = philox4x32_10(make_uint4(static_cast<uint32_t>(i0 >> 2), m, t_lo, t_hi), key0, key1);
+        // |v|/s with IEEE division; s = 0 gives NaN and the comparison is false.
+        const bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
+        const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
+        const bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
+        const bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
+        cnt += static_cast<uint32_t>(kx) + static_cast<uint32_t>(ky) + static_cast<uint32_t>(kz) +
+               static_cast<uint32_t>(kw);
+        const uint32_t byte = ternary_code(v.x, kx) | (ternary_code(v.y, ky) << 2) |
+                              (ternary_code(v.z, kz) << 4) | (ternary_code(v.w, kw) << 6);
+        store_code_byte(codes8, i0, row_words * 4, byte);
+        cur[r] = nxt[r];
+      }
+    }
+    const unsigned long long total = block_count(cnt, sm_cnt);
+    if (j == 0) ws.part_cnt[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
+  }
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  finish_codes<false>(geo, ws, scales_out, counts_out);
+  if (j == 0) *ws.ticket = 0u;
+}
+
+// ------------------------------------------------------------------ pass C helpers
+// Eq. H_t and Eq. QCMD for one coordinate.
+__device__ __forceinline__ void cmd_update(float q, float& x, float& h, const StepScalars& sc) {
+  const float hn = fmaf(q, q, h);
+  const float big_h = sc.delta + sqrtf(hn);
+  const float rate = sc.eta / big_h;
+  const float u = fmaf(-rate, q, x);
+  const float mag = fabsf(u) - sc.lambda * rate;
+  x = mag > 0.f ? copysignf(mag, u) : 0.f;
+  h = hn;
+}
+
+// Eq. H_t and Eq. QRDA for one coordinate.
+__device__ __forceinline__ void rda_update(float q, float& x, float& h, float& z, const StepScalars& sc) {
+  const float hn = fmaf(q, q, h);
+  const float zn = z + q;
+  const float big_h = sc.delta + sqrtf(hn);
+  const float a = fabsf(zn) / sc.t - sc.lambda;
+  const float coef = (sc.t * sc.eta) / big_h;
+  x = a > 0.f ? -copysignf(coef * a, zn) : 0.f;
+  h = hn;
+  z = zn;
+}
+
+// Adds scale * code for the four codes of one byte.
+__device__ __forceinline__ void decode_byte(uint32_t byte, float scale, float4& acc) {
+  const uint32_t s_bits = __float_as_uint(scale);
+  // code 1 -> +scale, code 2 -> -scale, code 0 or 3 -> 0
+  uint32_t c;
+  c = byte & 3u;
+  acc.x += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
+  c = (byte >> 2) & 3u;
+  acc.y += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
+  c = (byte >> 4) & 3u;
+  acc.z += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
+  c = (byte >> 6) & 3u;
+  acc.w += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
+}
+
+// Averaged decoded gradient of the four coordinates of group `grp` (Eq. SynQ_t).
+__device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes8, uint64_t row_bytes,
+                                               const float* sm_scale, uint32_t M, float inv_m,
+                                               uint64_t grp, uint32_t& bad) {
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (uint32_t m = 0; m < M; ++m) {
+    const uint32_t byte = __ldg(codes8 + m * row_bytes + grp);
+    bad |= byte & (byte >> 1) & 0x55u;
+    decode_byte(byte, sm_scale[m], acc);
+  }
+  acc.x *= inv_m;
+  acc.y *= inv_m;
+  acc.z *= inv_m;
+  acc.w *= inv_m;
+  return acc;
+}
+
+// ------------------------------------------------------------------ pass C: fused
+template <int kRule>
+__global__ void __launch_bounds__(kThreads)
+decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
+                     uint32_t M, float inv_m, float* __restrict__ x, float* __restrict__ h,
+                     float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
+  __shared__ float sm_scale[kMaxWorkers];
+  if (threadIdx.x < M) sm_scale[threadIdx.x] = scales[threadIdx.x];
+  __syncthreads();
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  const uint64_t row_bytes = ((d + 15) >> 4) * 4;
+  const uint64_t groups = (d + 3) >> 2, full = d >> 2;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+  uint32_t bad = 0;
+  for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
+    const float4 q = decode_group(codes8, row_bytes, sm_scale, M, inv_m, grp, bad);
+    if (grp < full) {
+      float4 hv = *reinterpret_cast<const float4*>(h + 4 * grp);
+      float4 xv, zv;
+      if (kRule == 0) {
+        xv = *reinterpret_cast<const float4*>(x + 4 * grp);
+        cmd_update(q.x, xv.x, hv.x, sc);
+        cmd_update(q.y, xv.y, hv.y, sc);
+        cmd_update(q.z, xv.z, hv.z, sc);
+        cmd_update(q.w, xv.w, hv.w, sc);
+      } else {
+        zv = *reinterpret_cast<const float4*>(z + 4 * grp);
+        rda_update(q.x, xv.x, hv.x, zv.x, sc);
+        rda_update(q.y, xv.y, hv.y, zv.y, sc);
+        rda_update(q.z, xv.z, hv.z, zv.z, sc);
+        rda_update(q.w, xv.w, hv.w, zv.w, sc);
+        *reinterpret_cast<float4*>(z + 4 * grp) = zv;
+      }
+      *reinterpret_cast<float4*>(h + 4 * grp) = hv;
+      *reinterpret_cast<float4*>(x + 4 * grp) = xv;
+    } else {  // ragged tail: d % 4 coordinates
+      const float qs[4] = {q.x, q.y, q.z, q.w};
+      for (uint64_t i = 4 * grp; i < d; ++i) {
+        float xi = (kRule == 0) ? x[i] : 0.f, hi = h[i];
+        if (kRule == 0) {
+          cmd_update(qs[i - 4 * grp], xi, hi, sc);
+        } else {
+          float zi = z[i];
+          rda_update(qs[i - 4 * grp], xi, hi, zi, sc);
+          z[i] = zi;
+        }
+        x[i] = xi;
+        h[i] = hi;
+      }
+    }
+  }
+  if (bad) atomicOr(status, kFlagBadCode);
+}
+
+// ------------------------------------------------------------------ pass C, unfused halves
+__global__ void __launch_bounds__(kThreads)
+decode_average_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
+                      uint32_t M, float inv_m, float* __restrict__ gbar, unsigned int* __restrict__ status) {
+  __shared__ float sm_scale[kMaxWorkers];
+  if (threadIdx.x < M) sm_scale[threadIdx.x] = scales[threadIdx.x];
+  __syncthreads();
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  const uint64_t row_bytes = ((d + 15) >> 4) * 4;
+  const uint64_t groups = (d + 3) >> 2, full = d >> 2;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+  uint32_t bad = 0;
+  for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
+    const float4 q = decode_group(codes8, row_bytes, sm_scale, M, inv_m, grp, bad);
+    if (grp < full) {
+      *reinterpret_cast<float4*>(gbar + 4 * grp) = q;
+    } else {
+      const float qs[4] = {q.x, q.y, q.z, q.w};
+      for (uint64_t i = 4 * grp; i < d; ++i) gbar[i] = qs[i - 4 * grp];
+    }
+  }
+  if (bad) atomicOr(status, kFlagBadCode);
+}
+
+template <int kRule>
+__global__ void __launch_bounds__(kThreads)
+dense_update_kernel(const float* __restrict__ q, uint64_t d, float* __restrict__ x,
+                    float* __restrict__ h, float* __restrict__ z, StepScalars sc) {
+  const uint64_t full = d >> 2;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+  const uint64_t first = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  for (uint64_t grp = first; grp < full; grp += stride) {
+    const float4 qv = __ldg(reinterpret_cast<const float4*>(q) + grp);
+    float4 hv = *reinterpret_cast<const float4*>(h + 4 * grp);
+    float4 xv, zv;
+    if (kRule == 0) {
+      xv = *reinterpret_cast<const float4*>(x + 4 * grp);
+      cmd_update(qv.x, xv.x, hv.x, sc);
+      cmd_update(qv.y, xv.y, hv.y, sc);
+      cmd_update(qv.z, xv.z, hv.z, sc);
+      cmd_update(qv.w, xv.w, hv.w, sc);
+    } else {
+      zv = *reinterpret_cast<const float4*>(z + 4 * grp);
+      rda_update(qv.x, xv.x, hv.x, zv.x, sc);
+      rda_update(qv.y, xv.y, hv.y, zv.y, sc);
+      rda_update(qv.z, xv.z, hv.z, zv.z, sc);
+      rda_update(qv.w, xv.w, hv.w, zv.w, sc);
+      *reinterpret_cast<float4*>(z + 4 * grp) = zv;
+    }
+    *reinterpret_cast<float4*>(h + 4 * grp) = hv;
+    *reinterpret_cast<float4*>(x + 4 * grp) = xv;
+  }
+  if (first == 0) {
+    for (uint64_t i = 4 * full; i < d; ++i) {
+      float xi = (kRule == 0) ? x[i] : 0.f, hi = h[i];
+      if (kRule == 0) {
+        cmd_update(q[i], xi, hi, sc);
+      } else {
+        float zi = z[i];
+        rda_update(q[i], xi, hi, zi, sc);
+        z[i] = zi;
+      }
+      x[i] = xi;
+      h[i] = hi;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ launchers
+void query_launch_shape(LaunchShape* shape) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&shape->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  int a = 0, b = 0;
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel, kThreads, 0);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_update_kernel<1>, kThreads, 0);
+  shape->reduce_ctas_per_sm = a > 0 ? a : 1;
+  shape->update_ctas_per_sm = b > 0 ? b : 1;
+}
+
+static unsigned reduce_grid(const Geometry& geo, const LaunchShape& shape) {
+  const uint64_t items = static_cast<uint64_t>(geo.M) * geo.chunks;
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * shape.reduce_ctas_per_sm;
+  return static_cast<unsigned>(items < resident ? items : resident);
+}
+
+static unsigned update_grid(uint64_t d, const LaunchShape& shape) {
+  const uint64_t groups = (d + 3) >> 2;
+  const uint64_t ctas = (groups + kThreads - 1) / kThreads;
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * shape.update_ctas_per_sm;
+  return static_cast<unsigned>(ctas < resident ? (ctas ? ctas : 1) : resident);
+}
+
+int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
+                   float* thresholds_out, const LaunchShape& shape, cudaStream_t stream) {
+  abs_sum_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out);
+  return 1;
+}
+
+int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
+                   const LaunchShape& shape, cudaStream_t stream) {
+  abs_max_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws);
+  return 1;
+}
+
+int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
+                           uint32_t* codes, float* scales_out, unsigned long long* counts_out,
+                           const LaunchShape& shape, cudaStream_t stream) {
+  threshold_codes_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                          counts_out);
+  return 1;
+}
+
+int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
+                            const Workspace& ws, uint32_t* codes, float* scales_out,
+                            unsigned long long* counts_out, const LaunchShape& shape,
+                            cudaStream_t stream) {
+  stochastic_codes_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, seed, t, ws, codes,
+                                                                           scales_out, counts_out);
+  return 1;
+}
+
+int launch_decode_update(int rule, const uint32_t* codes, const float* scales, uint64_t d,
+                         uint32_t M, float* x, float* h, float* z, const StepScalars& sc,
+                         unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
+  const float inv_m = 1.0f / static_cast<float>(M);
+  const unsigned grid = update_grid(d, shape);
+  if (rule == 0)
+    decode_update_kernel<0><<<grid, kThreads, 0, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
+  else
+    decode_update_kernel<1><<<grid, kThreads, 0, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
+  return 1;
+}
+
+int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
+                          float* gbar, unsigned int* status, const LaunchShape& shape,
+                          cudaStream_t stream) {
+  const float inv_m = 1.0f / static_cast<float>(M);
+  decode_average_kernel<<<update_grid(d, shape), kThreads, 0, stream>>>(codes, scales, d, M, inv_m, gbar,
+                                                                       status);
+  return 1;
+}
+
+int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h, float* z,
+                        const StepScalars& sc, const LaunchShape& shape, cudaStream_t stream) {
+  const unsigned grid = update_grid(d, shape);
+  if (rule == 0)
+    dense_update_kernel<0><<<grid, kThreads, 0, stream>>>(q, d, x, h, z, sc);
+  else
+    dense_update_kernel<1><<<grid, kThreads, 0, stream>>>(q, d, x, h, z, sc);
+  return 1;
+}
+
+}  // namespace qasg

@@ -1,0 +1,147 @@
+// Per-worker minibatch gradient of logistic regression (the linear-model workload):
+//   g_m = (1/B) sum_j -y_j * sigmoid(-y_j <a_j, x>) * a_j
+// Dense: GEMV-shaped and memory-bound.  Kernel 1 computes one coefficient per minibatch
+// row (a warp per row, 128-bit loads); kernel 2 forms the coefficient-weighted column sums
+// with a fixed summation order, reading the rows a second time out of L2.
+// CSR: one warp per minibatch row computes the margin and scatters with atomic adds.
+#include "qasg_internal.h"
+
+namespace qasg {
+
+struct Shards {
+  uint64_t row0[kMaxWorkers + 1];
+};
+
+// Global row id of minibatch entry b of worker m.
+__device__ __forceinline__ uint64_t batch_row(const Shards& sh, const uint32_t* __restrict__ batch_rows,
+                                              uint32_t m, uint32_t b, uint32_t B, uint64_t t) {
+  if (batch_rows) return batch_rows[static_cast<uint64_t>(m) * B + b];
+  const uint64_t lo = sh.row0[m], n = sh.row0[m + 1] - lo;
+  return lo + ((t - 1) % n * (B % n) + b) % n;
+}
+
+// -y * sigmoid(-y * s) / B, evaluated without overflow.
+__device__ __forceinline__ float logistic_coef(float y, float s, float inv_b) {
+  const float v = -y * s;
+  float sig;
+  if (v >= 0.f) {
+    sig = 1.f / (1.f + expf(-v));
+  } else {
+    const float e = expf(v);
+    sig = e / (1.f + e);
+  }
+  return -y * sig * inv_b;
+}
+
+__global__ void __launch_bounds__(kThreads)
+logreg_dense_coef_kernel(const float* __restrict__ X, const float* __restrict__ y, uint64_t d, uint32_t M,
+                         Shards sh, const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t,
+                         const float* __restrict__ x, float* __restrict__ coef, uint32_t* __restrict__ rows) {
+  const uint32_t warp = (blockIdx.x * kThreads + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= M * B) return;
+  const uint32_t m = warp / B, b = warp - m * B;
+  const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
+  const float4* a = reinterpret_cast<const float4*>(X + r * d);
+  const float4* xv = reinterpret_cast<const float4*>(x);
+  float acc = 0.f;
+  for (uint64_t k = lane; k < (d >> 2); k += 32) {
+    const float4 u = __ldg(a + k), w = __ldg(xv + k);
+    acc = fmaf(u.x, w.x, acc);
+    acc = fmaf(u.y, w.y, acc);
+    acc = fmaf(u.z, w.z, acc);
+    acc = fmaf(u.w, w.w, acc);
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+  if (lane == 0) {
+    coef[warp] = logistic_coef(y[r], acc, 1.f / static_cast<float>(B));
+    rows[warp] = static_cast<uint32_t>(r);
+  }
+}
+
+// grid (d/128, M); thread (cq = tid & 31 -> 4 columns, rl = tid >> 5 -> rows rl, rl+8, ...).
+__global__ void __launch_bounds__(kThreads)
+logreg_dense_colsum_kernel(const float* __restrict__ X, uint64_t d, uint32_t B, const float* __restrict__ coef,
+                           const uint32_t* __restrict__ rows, float* __restrict__ g, uint64_t ld_g) {
+  __shared__ float4 sm[kThreads / 32][32];
+  const uint32_t m = blockIdx.y, cq = threadIdx.x & 31, rl = threadIdx.x >> 5;
+  const uint64_t col = (static_cast<uint64_t>(blockIdx.x) * 32 + cq) * 4;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (col < d) {
+    for (uint32_t b = rl; b < B; b += kThreads / 32) {
+      const float c = coef[static_cast<uint64_t>(m) * B + b];
+      const uint64_t r = rows[static_cast<uint64_t>(m) * B + b];
+      const float4 a = __ldg(reinterpret_cast<const float4*>(X + r * d + col));
+      acc.x = fmaf(c, a.x, acc.x);
+      acc.y = fmaf(c, a.y, acc.y);
+      acc.z = fmaf(c, a.z, acc.z);
+      acc.w = fmaf(c, a.w, acc.w);
+    }
+  }
+  sm[rl][cq] = acc;
+  __syncthreads();
+  if (rl == 0 && col < d) {
+#pragma unroll
+    for (int k = 1; k < kThreads / 32; ++k) {
+      const float4 o = sm[k][cq];
+      acc.x += o.x;
+      acc.y += o.y;
+      acc.z += o.z;
+      acc.w += o.w;
+    }
+    *reinterpret_cast<float4*>(g + static_cast<uint64_t>(m) * ld_g + col) = acc;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ colidx,
+                  const float* __restrict__ vals, const float* __restrict__ y, uint32_t M, Shards sh,
+                  const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t, const float* __restrict__ x,
+                  float* __restrict__ g, uint64_t ld_g) {
+  const uint32_t warp = (blockIdx.x * kThreads + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= M * B) return;
+  const uint32_t m = warp / B, b = warp - m * B;
+  const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
+  const int64_t lo = rowptr[r], hi = rowptr[r + 1];
+  float acc = 0.f;
+  for (int64_t k = lo + lane; k < hi; k += 32) acc = fmaf(__ldg(vals + k), __ldg(x + __ldg(colidx + k)), acc);
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+  const float c = logistic_coef(y[r], acc, 1.f / static_cast<float>(B));
+  float* row = g + static_cast<uint64_t>(m) * ld_g;
+  for (int64_t k = lo + lane; k < hi; k += 32) atomicAdd(row + __ldg(colidx + k), c * __ldg(vals + k));
+}
+
+static Shards make_shards(const uint64_t* shard_row0_host, uint32_t M) {
+  Shards sh;
+  for (uint32_t m = 0; m <= M; ++m) sh.row0[m] = shard_row0_host[m];
+  return sh;
+}
+
+int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
+                        const uint64_t* shard_row0_host, const uint32_t* batch_rows, uint32_t B,
+                        uint64_t t, const float* x, float* g, uint64_t ld_g, float* coef_ws,
+                        const LaunchShape&, cudaStream_t stream) {
+  const Shards sh = make_shards(shard_row0_host, M);
+  uint32_t* rows_ws = reinterpret_cast<uint32_t*>(coef_ws + static_cast<uint64_t>(M) * B);
+  const uint64_t warps = static_cast<uint64_t>(M) * B;
+  const unsigned grid1 = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
+  logreg_dense_coef_kernel<<<grid1, kThreads, 0, stream>>>(X, y, d, M, sh, batch_rows, B, t, x, coef_ws, rows_ws);
+  const dim3 grid2(static_cast<unsigned>((d + 127) / 128), M);
+  logreg_dense_colsum_kernel<<<grid2, kThreads, 0, stream>>>(X, d, B, coef_ws, rows_ws, g, ld_g);
+  return 2;
+}
+
+int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float* vals,
+                      const float* y, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
+                      const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
+                      uint64_t ld_g, const LaunchShape&, cudaStream_t stream) {
+  const Shards sh = make_shards(shard_row0_host, M);
+  cudaMemset2DAsync(g, ld_g * sizeof(float), 0, d * sizeof(float), M, stream);
+  const uint64_t warps = static_cast<uint64_t>(M) * B;
+  const unsigned grid = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
+  logreg_csr_kernel<<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, M, sh, batch_rows, B, t, x, g, ld_g);
+  return 1;
+}
+
+}  // namespace qasg
