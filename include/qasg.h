@@ -186,6 +186,17 @@ qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream);
 /* Number of kernels this context has launched since it was created. */
 uint64_t qasg_launch_count(const qasg_ctx* ctx);
 
+/* Per-kernel device timing, for benchmarks.  Between qasg_profile_begin and
+ * qasg_profile_end every kernel the context launches is bracketed by a pair of CUDA events
+ * recorded on the stream it is launched on.  qasg_profile_end waits for those events and
+ * adds up, per kernel id (0 <= id < QASG_KERNEL_COUNT, names from qasg_kernel_name), the
+ * elapsed milliseconds into ms[id] and the number of launches into launches[id] (both host
+ * arrays of QASG_KERNEL_COUNT entries), then stops recording. */
+#define QASG_KERNEL_COUNT 12
+qasg_status qasg_profile_begin(qasg_ctx* ctx);
+qasg_status qasg_profile_end(qasg_ctx* ctx, double* ms, uint64_t* launches);
+const char* qasg_kernel_name(int id);
+
 const char* qasg_status_string(qasg_status s);
 
 #ifdef __cplusplus

@@ -2,6 +2,7 @@
 #include "../../include/qasg.h"
 
 #include <new>
+#include <vector>
 
 #include "qasg_internal.h"
 
@@ -16,9 +17,44 @@ struct qasg_ctx {
   uint32_t* code_scratch;   // [M_max][code_words(d_max)] or NULL
   float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
   uint64_t launches;
+  bool profiling;
+  std::vector<cudaEvent_t> events;  // pairs (start, stop), reused between profiles
+  std::vector<int> event_kernel;    // kernel id of each recorded pair
 };
 
 namespace {
+
+enum KernelId {
+  kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
+  kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kKernelIdCount
+};
+static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
+
+// Counts the launches of one launcher call and, while profiling, brackets them with events.
+struct Launch {
+  qasg_ctx* ctx;
+  cudaStream_t stream;
+  bool timed;
+  size_t slot;
+  Launch(qasg_ctx* c, int kernel, cudaStream_t s) : ctx(c), stream(s), timed(c->profiling), slot(0) {
+    if (!timed) return;
+    slot = ctx->event_kernel.size();
+    while (ctx->events.size() < 2 * (slot + 1)) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreate(&e) != cudaSuccess) {
+        timed = false;
+        return;
+      }
+      ctx->events.push_back(e);
+    }
+    ctx->event_kernel.push_back(kernel);
+    cudaEventRecord(ctx->events[2 * slot], stream);
+  }
+  void operator+=(int n) { ctx->launches += n; }
+  ~Launch() {
+    if (timed) cudaEventRecord(ctx->events[2 * slot + 1], stream);
+  }
+};
 
 constexpr uint64_t kMaxD = 1ull << 34;
 constexpr uint64_t kLogregEntries = 1ull << 20;  // M * B of one gradient call
@@ -66,12 +102,12 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
   const Geometry geo = make_geometry(d, ld_g, M);
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
   if (p->quantizer == QASG_Q_THRESHOLD) {
-    ctx->launches += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream);
-    ctx->launches += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream);
+    { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream); }
+    { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream); }
   } else {
-    ctx->launches += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream);
-    ctx->launches += launch_stochastic_codes(g, geo, p->seed, t, ctx->ws, codes, scales, counts_out,
-                                             ctx->shape, stream);
+    { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream); }
+    { Launch l(ctx, kStochasticCodes, stream); l += launch_stochastic_codes(g, geo, p->seed, t, ctx->ws, codes, scales, counts_out,
+                                             ctx->shape, stream); }
     if (thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
   }
 }
@@ -99,6 +135,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ctx->d_max = d_max;
   ctx->M_max = M_max;
   ctx->launches = 0;
+  ctx->profiling = false;
   query_launch_shape(&ctx->shape);
   const size_t slots = static_cast<size_t>(M_max) * kMaxChunks;
   bool ok = true;
@@ -141,6 +178,7 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->ws.status);
   cudaFree(ctx->logreg_ws);
   cudaFree(ctx->code_scratch);
+  for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   delete ctx;
   return QASG_OK;
 }
@@ -169,8 +207,8 @@ qasg_status qasg_decode_average(qasg_ctx* ctx, const uint32_t* codes, const floa
   if (!codes || !scales || !gbar) return QASG_ERR_INVALID_ARG;
   if (!aligned16(codes) || !aligned16(gbar)) return QASG_ERR_ALIGNMENT;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  ctx->launches += launch_decode_average(codes, scales, d, M, gbar, ctx->ws.status, ctx->shape,
-                                         static_cast<cudaStream_t>(stream));
+  { Launch l(ctx, kDecodeAverage, static_cast<cudaStream_t>(stream)); l += launch_decode_average(codes, scales, d, M, gbar, ctx->ws.status, ctx->shape,
+                                         static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -182,8 +220,8 @@ qasg_status qasg_cmd_step(qasg_ctx* ctx, const float* q, float* x, float* h, uin
   if (!q || !x || !h || t < 1) return QASG_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(x) || !aligned16(h)) return QASG_ERR_ALIGNMENT;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  ctx->launches += launch_dense_update(QASG_RULE_CMD, q, d, x, h, nullptr, scalars(params, t), ctx->shape,
-                                       static_cast<cudaStream_t>(stream));
+  { Launch l(ctx, kDenseUpdateCmd, static_cast<cudaStream_t>(stream)); l += launch_dense_update(QASG_RULE_CMD, q, d, x, h, nullptr, scalars(params, t), ctx->shape,
+                                       static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -195,8 +233,8 @@ qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, flo
   if (!q || !x || !h || !z || t < 1) return QASG_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(x) || !aligned16(h) || !aligned16(z)) return QASG_ERR_ALIGNMENT;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  ctx->launches += launch_dense_update(QASG_RULE_RDA, q, d, x, h, z, scalars(params, t), ctx->shape,
-                                       static_cast<cudaStream_t>(stream));
+  { Launch l(ctx, kDenseUpdateRda, static_cast<cudaStream_t>(stream)); l += launch_dense_update(QASG_RULE_RDA, q, d, x, h, z, scalars(params, t), ctx->shape,
+                                       static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -216,8 +254,8 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
   if ((st = enter(ctx)) != QASG_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
-  ctx->launches += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
-                                        ctx->ws.status, ctx->shape, s);
+  { Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s); l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
+                                        ctx->ws.status, ctx->shape, s); }
   return leave();
 }
 
@@ -279,8 +317,8 @@ qasg_status qasg_logreg_grad_dense(qasg_ctx* ctx, const float* X, const float* y
   if (!X) return QASG_ERR_INVALID_ARG;
   if ((d & 3u) || !aligned16(X)) return QASG_ERR_ALIGNMENT;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  ctx->launches += launch_logreg_dense(X, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->logreg_ws,
-                                       ctx->shape, static_cast<cudaStream_t>(stream));
+  { Launch l(ctx, kLogregDense, static_cast<cudaStream_t>(stream)); l += launch_logreg_dense(X, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->logreg_ws,
+                                       ctx->shape, static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -292,8 +330,8 @@ qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int
   if (st != QASG_OK) return st;
   if (!rowptr || !colidx || !vals) return QASG_ERR_INVALID_ARG;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  ctx->launches += launch_logreg_csr(rowptr, colidx, vals, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
-                                     ctx->shape, static_cast<cudaStream_t>(stream));
+  { Launch l(ctx, kLogregCsr, static_cast<cudaStream_t>(stream)); l += launch_logreg_csr(rowptr, colidx, vals, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
+                                     ctx->shape, static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -314,6 +352,42 @@ qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream) {
 }
 
 uint64_t qasg_launch_count(const qasg_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+qasg_status qasg_profile_begin(qasg_ctx* ctx) {
+  if (!ctx) return QASG_ERR_INVALID_ARG;
+  ctx->event_kernel.clear();
+  ctx->profiling = true;
+  return QASG_OK;
+}
+
+qasg_status qasg_profile_end(qasg_ctx* ctx, double* ms, uint64_t* launches) {
+  if (!ctx || !ms || !launches) return QASG_ERR_INVALID_ARG;
+  ctx->profiling = false;
+  for (int k = 0; k < QASG_KERNEL_COUNT; ++k) {
+    ms[k] = 0.0;
+    launches[k] = 0;
+  }
+  if (enter(ctx) != QASG_OK) return QASG_ERR_CUDA;
+  for (size_t i = 0; i < ctx->event_kernel.size(); ++i) {
+    float elapsed = 0.f;
+    if (cudaEventSynchronize(ctx->events[2 * i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&elapsed, ctx->events[2 * i], ctx->events[2 * i + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      return QASG_ERR_CUDA;
+    }
+    ms[ctx->event_kernel[i]] += elapsed;
+    launches[ctx->event_kernel[i]] += 1;
+  }
+  ctx->event_kernel.clear();
+  return QASG_OK;
+}
+
+const char* qasg_kernel_name(int id) {
+  static const char* const names[kKernelIdCount] = {
+      "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
+      "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr"};
+  return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
+}
 
 const char* qasg_status_string(qasg_status s) {
   switch (s) {

@@ -450,46 +450,40 @@ __device__ __forceinline__ void rda_update(float q, float& x, float& h, float& z
   z = zn;
 }
 
-// Adds scale * code for the four codes of one byte.
-__device__ __forceinline__ void decode_byte(uint32_t byte, float scale, float4& acc) {
-  const uint32_t s_bits = __float_as_uint(scale);
-  // code 1 -> +scale, code 2 -> -scale, code 0 or 3 -> 0
-  uint32_t c;
-  c = byte & 3u;
-  acc.x += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
-  c = (byte >> 2) & 3u;
-  acc.y += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
-  c = (byte >> 4) & 3u;
-  acc.z += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
-  c = (byte >> 6) & 3u;
-  acc.w += (c == 1u) ? scale : ((c == 2u) ? __uint_as_float(s_bits ^ 0x80000000u) : 0.f);
+// Adds scale * code for the four codes of one byte (code 1 -> +scale, 2 -> -scale, 0 or 3 -> 0).
+// The sum over workers is kept in fp64: terms of opposite sign cancel, and the update divides
+// by H = delta + sqrt(h), which can be as small as |q| itself, so q must carry no more than
+// its own fp32 rounding error.
+__device__ __forceinline__ void decode_byte(uint32_t byte, double scale, double (&acc)[4]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t c = (byte >> (2 * k)) & 3u;
+    acc[k] += (c == 1u) ? scale : ((c == 2u) ? -scale : 0.0);
+  }
 }
 
 // Averaged decoded gradient of the four coordinates of group `grp` (Eq. SynQ_t).
 __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes8, uint64_t row_bytes,
-                                               const float* sm_scale, uint32_t M, float inv_m,
+                                               const double* sm_scale, uint32_t M, double inv_m,
                                                uint64_t grp, uint32_t& bad) {
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
   for (uint32_t m = 0; m < M; ++m) {
     const uint32_t byte = __ldg(codes8 + m * row_bytes + grp);
     bad |= byte & (byte >> 1) & 0x55u;
     decode_byte(byte, sm_scale[m], acc);
   }
-  acc.x *= inv_m;
-  acc.y *= inv_m;
-  acc.z *= inv_m;
-  acc.w *= inv_m;
-  return acc;
+  return make_float4(static_cast<float>(acc[0] * inv_m), static_cast<float>(acc[1] * inv_m),
+                     static_cast<float>(acc[2] * inv_m), static_cast<float>(acc[3] * inv_m));
 }
 
 // ------------------------------------------------------------------ pass C: fused
 template <int kRule>
 __global__ void __launch_bounds__(kThreads)
 decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
-                     uint32_t M, float inv_m, float* __restrict__ x, float* __restrict__ h,
+                     uint32_t M, double inv_m, float* __restrict__ x, float* __restrict__ h,
                      float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
-  __shared__ float sm_scale[kMaxWorkers];
-  if (threadIdx.x < M) sm_scale[threadIdx.x] = scales[threadIdx.x];
+  __shared__ double sm_scale[kMaxWorkers];
+  if (threadIdx.x < M) sm_scale[threadIdx.x] = static_cast<double>(scales[threadIdx.x]);
   __syncthreads();
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
@@ -539,9 +533,9 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
 // ------------------------------------------------------------------ pass C, unfused halves
 __global__ void __launch_bounds__(kThreads)
 decode_average_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
-                      uint32_t M, float inv_m, float* __restrict__ gbar, unsigned int* __restrict__ status) {
-  __shared__ float sm_scale[kMaxWorkers];
-  if (threadIdx.x < M) sm_scale[threadIdx.x] = scales[threadIdx.x];
+                      uint32_t M, double inv_m, float* __restrict__ gbar, unsigned int* __restrict__ status) {
+  __shared__ double sm_scale[kMaxWorkers];
+  if (threadIdx.x < M) sm_scale[threadIdx.x] = static_cast<double>(scales[threadIdx.x]);
   __syncthreads();
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
@@ -661,7 +655,7 @@ int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, 
 int launch_decode_update(int rule, const uint32_t* codes, const float* scales, uint64_t d,
                          uint32_t M, float* x, float* h, float* z, const StepScalars& sc,
                          unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
-  const float inv_m = 1.0f / static_cast<float>(M);
+  const double inv_m = 1.0 / static_cast<double>(M);
   const unsigned grid = update_grid(d, shape);
   if (rule == 0)
     decode_update_kernel<0><<<grid, kThreads, 0, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
@@ -673,7 +667,7 @@ int launch_decode_update(int rule, const uint32_t* codes, const float* scales, u
 int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                           float* gbar, unsigned int* status, const LaunchShape& shape,
                           cudaStream_t stream) {
-  const float inv_m = 1.0f / static_cast<float>(M);
+  const double inv_m = 1.0 / static_cast<double>(M);
   decode_average_kernel<<<update_grid(d, shape), kThreads, 0, stream>>>(codes, scales, d, M, inv_m, gbar,
                                                                        status);
   return 1;

@@ -25,7 +25,9 @@ EXPORTS = [
     "qasg_create", "qasg_destroy", "qasg_code_words", "qasg_quantize_pack", "qasg_decode_average",
     "qasg_cmd_step", "qasg_rda_step", "qasg_step", "qasg_step_host", "qasg_logreg_grad_dense",
     "qasg_logreg_grad_csr", "qasg_last_async_status", "qasg_launch_count", "qasg_status_string",
+    "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name",
 ]
+KERNEL_COUNT = 12
 
 
 class QasgError(RuntimeError):
@@ -75,6 +77,10 @@ def load():
     lib.qasg_last_async_status.argtypes = [vp, vp]
     lib.qasg_launch_count.argtypes = [vp]
     lib.qasg_launch_count.restype = u64
+    lib.qasg_profile_begin.argtypes = [vp]
+    lib.qasg_profile_end.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(u64)]
+    lib.qasg_kernel_name.argtypes = [i32]
+    lib.qasg_kernel_name.restype = ctypes.c_char_p
     lib.qasg_status_string.argtypes = [i32]
     lib.qasg_status_string.restype = ctypes.c_char_p
     _lib = lib
@@ -171,6 +177,17 @@ class Context:
 
     def last_async_status(self, stream=None):
         return int(load().qasg_last_async_status(self._h, _stream(stream)))
+
+    def profile_begin(self):
+        _check(load().qasg_profile_begin(self._h), "qasg_profile_begin")
+
+    def profile_end(self):
+        """Returns {kernel name: (total ms, launches)} for the kernels launched since profile_begin."""
+        ms = (ctypes.c_double * KERNEL_COUNT)()
+        n = (ctypes.c_uint64 * KERNEL_COUNT)()
+        _check(load().qasg_profile_end(self._h, ms, n), "qasg_profile_end")
+        return {load().qasg_kernel_name(k).decode(): (float(ms[k]), int(n[k]))
+                for k in range(KERNEL_COUNT) if n[k]}
 
     def launch_count(self):
         return int(load().qasg_launch_count(self._h))

@@ -27,11 +27,11 @@ def grad_to_dev(g, pad_value=float("nan")):
     return to_dev(buf), ld
 
 
-def assert_close(got, want, what=""):
+def assert_close(got, want, what="", atol=ATOL):
     got = got.detach().cpu().numpy().astype(np.float64) if isinstance(got, torch.Tensor) else np.asarray(got, np.float64)
     want = np.asarray(want, dtype=np.float64)
     err = np.abs(got - want)
-    bound = ATOL + RTOL * np.abs(want)
+    bound = atol + RTOL * np.abs(want)
     bad = np.nonzero(err > bound)[0]
     assert bad.size == 0, "%s: %d of %d outside tolerance; worst at %d: got %r want %r" % (
         what, bad.size, want.size, bad[0], got[bad[0]], want[bad[0]])
