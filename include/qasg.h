@@ -179,6 +179,41 @@ qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int
                                  const uint32_t* batch_rows, uint32_t B, uint64_t t,
                                  const float* x, float* g, uint64_t ld_g, void* stream);
 
+/* The threshold quantizer of qasg_quantize_pack for callers that cannot allocate device
+ * memory.  (The paper has no counterpart: this entry point exists for the sake of its
+ * callers, not of the method.)
+ *
+ * Some code that wants to quantize gradients runs where cudaMalloc is off limits: inside a
+ * framework that has already handed all device memory to its own pool, so that a raw
+ * allocation fails or fragments it; or inside a latency-critical loop that cannot accept the
+ * device-wide synchronisation an allocation implies.  Such callers cannot create a qasg_ctx,
+ * whose workspace is allocated in qasg_create.  This call needs no context and allocates
+ * nothing, on the host or on the device: its scratch (per-chunk partial sums and counts,
+ * per-worker statistics, a completion counter) is a fixed array of
+ * QASG_STATIC_SCRATCH_BYTES bytes built into the library, which every GPU that loads the
+ * library holds until the process exits.
+ *
+ *   device      CUDA device ordinal (0 <= device < 64); made current by the call.
+ *   g, d, ld_g, codes, scales, thresholds, counts, stream   as for qasg_quantize_pack;
+ *               the quantizer is QASG_Q_THRESHOLD with coefficient thr_coef (0.75 in
+ *               Section 3.5).  Results are bit-identical to qasg_quantize_pack's.
+ *   M           1 <= M <= QASG_STATIC_MAX_WORKERS; more workers than the scratch holds is
+ *               refused with QASG_ERR_WORKSPACE and nothing is enqueued.  d may be as large
+ *               as for any other call (1 <= d <= 2^34): the scratch does not grow with d.
+ *
+ * The first call on a device looks up the device address of the built-in array; make that
+ * first call before any stream capture begins.  All calls on a device share the one array
+ * and it keeps the previous call's contents: each call clears the counter it needs at zero
+ * on `stream` before its kernels, so calls issued one after another on one stream are safe,
+ * but two calls that may overlap on the GPU (different streams, no dependency between them)
+ * race on the array and give undefined results.  A non-finite gradient gives all-zero codes
+ * and a zero scale for that worker, as in qasg_quantize_pack, but is not reported. */
+#define QASG_STATIC_MAX_WORKERS 16u
+#define QASG_STATIC_SCRATCH_BYTES (336u * 1024u)
+qasg_status qasg_quantize_pack_static(int device, const float* g, uint64_t d, uint64_t ld_g,
+                                      uint32_t M, float thr_coef, uint32_t* codes, float* scales,
+                                      float* thresholds, uint64_t* counts, void* stream);
+
 /* Waits for `stream`, then returns and clears the conditions kernels recorded since
  * the last call: QASG_ERR_NONFINITE, QASG_ERR_BAD_CODE, QASG_ERR_CUDA, else QASG_OK. */
 qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream);

@@ -25,8 +25,9 @@ EXPORTS = [
     "qasg_create", "qasg_destroy", "qasg_code_words", "qasg_quantize_pack", "qasg_decode_average",
     "qasg_cmd_step", "qasg_rda_step", "qasg_step", "qasg_step_host", "qasg_logreg_grad_dense",
     "qasg_logreg_grad_csr", "qasg_last_async_status", "qasg_launch_count", "qasg_status_string",
-    "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name",
+    "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static",
 ]
+STATIC_MAX_WORKERS = 16
 KERNEL_COUNT = 12
 
 
@@ -81,6 +82,7 @@ def load():
     lib.qasg_profile_end.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(u64)]
     lib.qasg_kernel_name.argtypes = [i32]
     lib.qasg_kernel_name.restype = ctypes.c_char_p
+    lib.qasg_quantize_pack_static.argtypes = [i32, vp, u64, u64, u32, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.qasg_status_string.argtypes = [i32]
     lib.qasg_status_string.restype = ctypes.c_char_p
     _lib = lib
@@ -191,6 +193,16 @@ class Context:
 
     def launch_count(self):
         return int(load().qasg_launch_count(self._h))
+
+
+def quantize_pack_static(device, g, d, ld_g, M, thr_coef, codes, scales, thresholds=None, counts=None,
+                          stream=None):
+    """qasg_quantize_pack_static: the threshold quantizer without a context and without any
+    allocation (the scratch is a fixed array inside the library; at most STATIC_MAX_WORKERS
+    workers; calls that overlap on the GPU race on it)."""
+    _check(load().qasg_quantize_pack_static(int(device), _ptr(g), d, ld_g, M, float(thr_coef), _ptr(codes),
+                                            _ptr(scales), _ptr(thresholds), _ptr(counts), _stream(stream)),
+           "qasg_quantize_pack_static")
 
 
 def code_words(d):
