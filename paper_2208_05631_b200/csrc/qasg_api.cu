@@ -92,6 +92,7 @@ StepScalars scalars(const qasg_params* p, uint64_t t) {
   sc.eta = p->eta;
   sc.delta = p->delta;
   sc.t = static_cast<float>(t);
+  sc.inv_t = 1.0f / sc.t;
   return sc;
 }
 

@@ -51,7 +51,7 @@ struct LaunchShape {
 };
 
 struct StepScalars {
-  float lambda, eta, delta, t;
+  float lambda, eta, delta, t, inv_t;
 };
 
 // Each launcher enqueues on `stream` and returns the number of kernels it launched.

@@ -136,6 +136,24 @@ __device__ __forceinline__ bool grid_last_cta(unsigned int* ticket, bool* sm_fla
   return last;
 }
 
+// Calls body(tile_values, k) for the tiles k0 <= k < k1 of one worker row, keeping the loads
+// of tile k+1 in flight while tile k is processed (two register buffers, no copies).
+template <class Body>
+__device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64_t d, uint32_t k0,
+                                           uint32_t k1, int j, Body&& body) {
+  float4 a[kTileRows], b[kTileRows];
+  load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
+  uint32_t k = k0;
+  while (true) {
+    if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, b);
+    body(a, k);
+    if (++k >= k1) break;
+    if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, a);
+    body(b, k);
+    if (++k >= k1) break;
+  }
+}
+
 // ------------------------------------------------------------------ pass A: sum |g|
 __global__ void __launch_bounds__(kThreads)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
@@ -151,24 +169,19 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    float4 cur[kTileRows], nxt[kTileRows];
-    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
-    for (uint32_t k = k0; k < k1; ++k) {
-      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
-      double cx = fabsf(cur[0].x), cy = fabsf(cur[0].y), cz = fabsf(cur[0].z), cw = fabsf(cur[0].w);
+    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t k) {
+      double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
 #pragma unroll
       for (int r = 1; r < kTileRows; ++r) {
-        cx += static_cast<double>(fabsf(cur[r].x));
-        cy += static_cast<double>(fabsf(cur[r].y));
-        cz += static_cast<double>(fabsf(cur[r].z));
-        cw += static_cast<double>(fabsf(cur[r].w));
+        cx += static_cast<double>(fabsf(v[r].x));
+        cy += static_cast<double>(fabsf(v[r].y));
+        cz += static_cast<double>(fabsf(v[r].z));
+        cw += static_cast<double>(fabsf(v[r].w));
       }
       const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
       slot ^= 1;
       if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
-#pragma unroll
-      for (int r = 0; r < kTileRows; ++r) cur[r] = nxt[r];
-    }
+    });
     if (j == 0)
       ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = tile_fold(sm_stack, k1 - k0, geo.log2_group);
   }
@@ -198,42 +211,38 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    float4 cur[kTileRows], nxt[kTileRows];
     uint32_t best = 0u;  // bit patterns of non-negative floats order like their values
-    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
-    for (uint32_t k = k0; k < k1; ++k) {
-      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
+    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t) {
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
-        best = max(best, __float_as_uint(fabsf(cur[r].x)));
-        best = max(best, __float_as_uint(fabsf(cur[r].y)));
-        best = max(best, __float_as_uint(fabsf(cur[r].z)));
-        best = max(best, __float_as_uint(fabsf(cur[r].w)));
-        cur[r] = nxt[r];
+        best = max(best, __float_as_uint(fabsf(v[r].x)));
+        best = max(best, __float_as_uint(fabsf(v[r].y)));
+        best = max(best, __float_as_uint(fabsf(v[r].z)));
+        best = max(best, __float_as_uint(fabsf(v[r].w)));
       }
-    }
+    });
     best = __reduce_max_sync(0xffffffffu, best);
     __syncthreads();  // the previous item's readers are done with sm_warp
     if ((j & 31) == 0) sm_warp[j >> 5] = best;
     __syncthreads();
     if (j == 0) {
-      uint32_t b = sm_warp[0];
+      uint32_t bmax = sm_warp[0];
 #pragma unroll
-      for (int w = 1; w < kThreads / 32; ++w) b = max(b, sm_warp[w]);
-      ws.part_max[static_cast<uint64_t>(m) * kMaxChunks + c] = b;
+      for (int w = 1; w < kThreads / 32; ++w) bmax = max(bmax, sm_warp[w]);
+      ws.part_max[static_cast<uint64_t>(m) * kMaxChunks + c] = bmax;
     }
   }
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   const int warp = j >> 5, lane = j & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
-    uint32_t b = 0u;
+    uint32_t bmax = 0u;
     for (uint32_t idx = lane; idx < geo.chunks; idx += 32)
-      b = max(b, __ldcg(ws.part_max + static_cast<uint64_t>(m) * kMaxChunks + idx));
-    b = __reduce_max_sync(0xffffffffu, b);
+      bmax = max(bmax, __ldcg(ws.part_max + static_cast<uint64_t>(m) * kMaxChunks + idx));
+    bmax = __reduce_max_sync(0xffffffffu, bmax);
     if (lane == 0) {
-      ws.scales[m] = __uint_as_float(b);
+      ws.scales[m] = __uint_as_float(bmax);
       ws.thresholds[m] = 0.f;
-      if (b >= 0x7f800000u) atomicOr(ws.status, kFlagNonFinite);
+      if (bmax >= 0x7f800000u) atomicOr(ws.status, kFlagNonFinite);
     }
   }
   if (j == 0) *ws.ticket = 0u;
@@ -245,11 +254,29 @@ __device__ __forceinline__ uint32_t ternary_code(float v, bool keep) {
   return keep ? ((__float_as_uint(v) >> 31) + 1u) : 0u;
 }
 
-// Writes the byte holding the codes of coordinates i0..i0+3 of worker row `codes8`.
-__device__ __forceinline__ void store_code_byte(uint8_t* __restrict__ codes8, uint64_t i0,
-                                                uint64_t row_bytes, uint32_t byte) {
-  const uint64_t b = i0 >> 2;
-  if (b < row_bytes) codes8[b] = static_cast<uint8_t>(byte);
+__device__ __forceinline__ uint32_t pack4(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3) {
+  return c0 + (c1 << 2) + (c2 << 4) + (c3 << 6);
+}
+
+// Number of non-zero 2-bit codes in a byte.
+__device__ __forceinline__ uint32_t nonzero_codes(uint32_t byte) {
+  return __popc((byte | (byte >> 1)) & 0x55u);
+}
+
+// Writes the code bytes of the thread's four rows of tile k.  codes8 is the worker's code
+// row; only the last tile can reach past the row's last byte.
+__device__ __forceinline__ void store_code_bytes(uint8_t* __restrict__ codes8, uint32_t k, int j,
+                                                 bool full, uint64_t row_bytes,
+                                                 const uint32_t (&bytes)[kTileRows]) {
+  const uint64_t b0 = static_cast<uint64_t>(k) * (kTile / 4) + j;
+  if (full) {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) codes8[b0 + r * (kTileCols / 4)] = static_cast<uint8_t>(bytes[r]);
+  } else {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r)
+      if (b0 + r * (kTileCols / 4) < row_bytes) codes8[b0 + r * (kTileCols / 4)] = static_cast<uint8_t>(bytes[r]);
+  }
 }
 
 // Sums per-thread counts over the CTA; the result is valid in thread 0.
@@ -306,6 +333,7 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
   const int j = threadIdx.x;
   const uint32_t n_items = geo.M * geo.chunks;
   const uint64_t row_words = (geo.d + 15) >> 4;
+  const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
   int slot = 0;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
@@ -315,32 +343,27 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
-    float4 cur[kTileRows], nxt[kTileRows];
-    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
-    for (uint32_t k = k0; k < k1; ++k) {
-      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
-      const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t k) {
       double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+      uint32_t bytes[kTileRows];
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
-        const float4 t = cur[r];
+        const float4 t = v[r];
         const float ax = fabsf(t.x), ay = fabsf(t.y), az = fabsf(t.z), aw = fabsf(t.w);
         const bool kx = ax > delta, ky = ay > delta, kz = az > delta, kw = aw > delta;
         if (kx) cx += static_cast<double>(ax);
         if (ky) cy += static_cast<double>(ay);
         if (kz) cz += static_cast<double>(az);
         if (kw) cw += static_cast<double>(aw);
-        cnt += static_cast<uint32_t>(kx) + static_cast<uint32_t>(ky) + static_cast<uint32_t>(kz) +
-               static_cast<uint32_t>(kw);
-        const uint32_t byte = ternary_code(t.x, kx) | (ternary_code(t.y, ky) << 2) |
-                              (ternary_code(t.z, kz) << 4) | (ternary_code(t.w, kw) << 6);
-        store_code_byte(codes8, tile_base + r * kTileCols + 4 * j, row_words * 4, byte);
-        cur[r] = nxt[r];
+        bytes[r] = pack4(ternary_code(t.x, kx), ternary_code(t.y, ky), ternary_code(t.z, kz),
+                         ternary_code(t.w, kw));
+        cnt += nonzero_codes(bytes[r]);
       }
+      store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
       const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
       slot ^= 1;
       if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
-    }
+    });
     const unsigned long long total = block_count(cnt, sm_cnt);
     if (j == 0) {
       const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
@@ -385,6 +408,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
   const int j = threadIdx.x;
   const uint32_t n_items = geo.M * geo.chunks;
   const uint64_t row_words = (geo.d + 15) >> 4;
+  const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
   const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
   const uint32_t t_lo = static_cast<uint32_t>(t), t_hi = static_cast<uint32_t>(t >> 32);
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -395,29 +419,25 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
-    float4 cur[kTileRows], nxt[kTileRows];
-    load_tile(row, static_cast<uint64_t>(k0) * kTile, geo.d, j, cur);
-    for (uint32_t k = k0; k < k1; ++k) {
-      if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, geo.d, j, nxt);
-      const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&tile)[kTileRows], uint32_t k) {
+      uint32_t bytes[kTileRows];
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
-        const float4 v = cur[r];
-        const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
-        const uint4 w = philox4x32_10(make_uint4(static_cast<uint32_t>(i0 >> 2), m, t_lo, t_hi), key0, key1);
+        const float4 v = tile[r];
+        // coordinates 4*blk .. 4*blk+3 share one Philox block
+        const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
+        const uint4 w = philox4x32_10(make_uint4(blk, m, t_lo, t_hi), key0, key1);
         // |v|/s with IEEE division; s = 0 gives NaN and the comparison is false.
         const bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
         const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
         const bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
         const bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
-        cnt += static_cast<uint32_t>(kx) + static_cast<uint32_t>(ky) + static_cast<uint32_t>(kz) +
-               static_cast<uint32_t>(kw);
-        const uint32_t byte = ternary_code(v.x, kx) | (ternary_code(v.y, ky) << 2) |
-                              (ternary_code(v.z, kz) << 4) | (ternary_code(v.w, kw) << 6);
-        store_code_byte(codes8, i0, row_words * 4, byte);
-        cur[r] = nxt[r];
+        bytes[r] = pack4(ternary_code(v.x, kx), ternary_code(v.y, ky), ternary_code(v.z, kz),
+                         ternary_code(v.w, kw));
+        cnt += nonzero_codes(bytes[r]);
       }
-    }
+      store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
+    });
     const unsigned long long total = block_count(cnt, sm_cnt);
     if (j == 0) ws.part_cnt[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
   }
@@ -430,50 +450,80 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
 // Eq. H_t and Eq. QCMD for one coordinate.
 __device__ __forceinline__ void cmd_update(float q, float& x, float& h, const StepScalars& sc) {
   const float hn = fmaf(q, q, h);
-  const float big_h = sc.delta + sqrtf(hn);
-  const float rate = sc.eta / big_h;
+  const float big_h = sc.delta + __fsqrt_rn(hn);
+  const float rate = sc.eta * __frcp_rn(big_h);
   const float u = fmaf(-rate, q, x);
   const float mag = fabsf(u) - sc.lambda * rate;
   x = mag > 0.f ? copysignf(mag, u) : 0.f;
   h = hn;
 }
 
-// Eq. H_t and Eq. QRDA for one coordinate.
+// Eq. H_t and Eq. QRDA for one coordinate.  sc.t holds t, sc.inv_t its reciprocal.
 __device__ __forceinline__ void rda_update(float q, float& x, float& h, float& z, const StepScalars& sc) {
   const float hn = fmaf(q, q, h);
   const float zn = z + q;
-  const float big_h = sc.delta + sqrtf(hn);
-  const float a = fabsf(zn) / sc.t - sc.lambda;
-  const float coef = (sc.t * sc.eta) / big_h;
+  const float big_h = sc.delta + __fsqrt_rn(hn);
+  const float a = fmaf(fabsf(zn), sc.inv_t, -sc.lambda);
+  const float coef = (sc.t * sc.eta) * __frcp_rn(big_h);
   x = a > 0.f ? -copysignf(coef * a, zn) : 0.f;
   h = hn;
   z = zn;
 }
 
-// Adds scale * code for the four codes of one byte (code 1 -> +scale, 2 -> -scale, 0 or 3 -> 0).
-// The sum over workers is kept in fp64: terms of opposite sign cancel, and the update divides
-// by H = delta + sqrt(h), which can be as small as |q| itself, so q must carry no more than
-// its own fp32 rounding error.
-__device__ __forceinline__ void decode_byte(uint32_t byte, double scale, double (&acc)[4]) {
+// The decode keeps, per group of 4 workers, a table of the 256 possible partial sums
+//   lut[G][c0 | c1<<2 | c2<<4 | c3<<6] = sum_k scale[4G+k] * value(c_k)     (value: 1 -> +1, 2 -> -1)
+// in shared memory, in fp64: terms of opposite sign cancel across workers, and the update
+// divides by H = delta + sqrt(h), which can be as small as |q| itself, so q must carry no
+// more than its own fp32 rounding error.
+__device__ __forceinline__ void build_decode_lut(double* lut, const float* __restrict__ scales, uint32_t M) {
+  const uint32_t groups = (M + 3) >> 2;
+  for (uint32_t e = threadIdx.x; e < groups * 256; e += kThreads) {
+    const uint32_t grp = e >> 8, idx = e & 255u;
+    double acc = 0.0;
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const uint32_t c = (byte >> (2 * k)) & 3u;
-    acc[k] += (c == 1u) ? scale : ((c == 2u) ? -scale : 0.0);
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t m = grp * 4 + k;
+      const uint32_t c = (idx >> (2 * k)) & 3u;
+      if (m < M && (c == 1u || c == 2u)) {
+        const double sv = static_cast<double>(scales[m]);
+        acc += (c == 1u) ? sv : -sv;
+      }
+    }
+    lut[e] = acc;
   }
+  __syncthreads();
+}
+
+// In a word whose byte k holds worker k's four 2-bit codes (coordinates 0..3), exchanges the
+// roles of byte and field: afterwards byte c holds the four workers' codes of coordinate c.
+__device__ __forceinline__ uint32_t transpose_2bit_4x4(uint32_t w) {
+  uint32_t t = ((w >> 6) ^ w) & 0x00CC00CCu;
+  w ^= t ^ (t << 6);
+  t = ((w >> 12) ^ w) & 0x0000F0F0u;
+  w ^= t ^ (t << 12);
+  return w;
 }
 
 // Averaged decoded gradient of the four coordinates of group `grp` (Eq. SynQ_t).
 __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes8, uint64_t row_bytes,
-                                               const double* sm_scale, uint32_t M, double inv_m,
+                                               const double* lut, uint32_t M, double inv_m,
                                                uint64_t grp, uint32_t& bad) {
-  double acc[4] = {0.0, 0.0, 0.0, 0.0};
-  for (uint32_t m = 0; m < M; ++m) {
-    const uint32_t byte = __ldg(codes8 + m * row_bytes + grp);
-    bad |= byte & (byte >> 1) & 0x55u;
-    decode_byte(byte, sm_scale[m], acc);
+  double q0 = 0.0, q1 = 0.0, q2 = 0.0, q3 = 0.0;
+  const uint8_t* p = codes8 + grp;
+  for (uint32_t m0 = 0; m0 < M; m0 += 4, lut += 256, p += 4 * row_bytes) {
+    uint32_t w = __ldg(p);
+    if (m0 + 1 < M) w |= static_cast<uint32_t>(__ldg(p + row_bytes)) << 8;
+    if (m0 + 2 < M) w |= static_cast<uint32_t>(__ldg(p + 2 * row_bytes)) << 16;
+    if (m0 + 3 < M) w |= static_cast<uint32_t>(__ldg(p + 3 * row_bytes)) << 24;
+    bad |= w & (w >> 1) & 0x55555555u;
+    w = transpose_2bit_4x4(w);
+    q0 += lut[w & 255u];
+    q1 += lut[(w >> 8) & 255u];
+    q2 += lut[(w >> 16) & 255u];
+    q3 += lut[w >> 24];
   }
-  return make_float4(static_cast<float>(acc[0] * inv_m), static_cast<float>(acc[1] * inv_m),
-                     static_cast<float>(acc[2] * inv_m), static_cast<float>(acc[3] * inv_m));
+  return make_float4(static_cast<float>(q0 * inv_m), static_cast<float>(q1 * inv_m),
+                     static_cast<float>(q2 * inv_m), static_cast<float>(q3 * inv_m));
 }
 
 // ------------------------------------------------------------------ pass C: fused
@@ -482,27 +532,27 @@ __global__ void __launch_bounds__(kThreads)
 decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
                      uint32_t M, double inv_m, float* __restrict__ x, float* __restrict__ h,
                      float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
-  __shared__ double sm_scale[kMaxWorkers];
-  if (threadIdx.x < M) sm_scale[threadIdx.x] = static_cast<double>(scales[threadIdx.x]);
-  __syncthreads();
+  extern __shared__ double sm_lut[];
+  build_decode_lut(sm_lut, scales, M);
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
   const uint64_t groups = (d + 3) >> 2, full = d >> 2;
   const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
   uint32_t bad = 0;
   for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
-    const float4 q = decode_group(codes8, row_bytes, sm_scale, M, inv_m, grp, bad);
     if (grp < full) {
+      // issue the state loads before the decode so that they overlap it
       float4 hv = *reinterpret_cast<const float4*>(h + 4 * grp);
       float4 xv, zv;
+      if (kRule == 0) xv = *reinterpret_cast<const float4*>(x + 4 * grp);
+      else zv = *reinterpret_cast<const float4*>(z + 4 * grp);
+      const float4 q = decode_group(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
       if (kRule == 0) {
-        xv = *reinterpret_cast<const float4*>(x + 4 * grp);
         cmd_update(q.x, xv.x, hv.x, sc);
         cmd_update(q.y, xv.y, hv.y, sc);
         cmd_update(q.z, xv.z, hv.z, sc);
         cmd_update(q.w, xv.w, hv.w, sc);
       } else {
-        zv = *reinterpret_cast<const float4*>(z + 4 * grp);
         rda_update(q.x, xv.x, hv.x, zv.x, sc);
         rda_update(q.y, xv.y, hv.y, zv.y, sc);
         rda_update(q.z, xv.z, hv.z, zv.z, sc);
@@ -512,6 +562,7 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
       *reinterpret_cast<float4*>(h + 4 * grp) = hv;
       *reinterpret_cast<float4*>(x + 4 * grp) = xv;
     } else {  // ragged tail: d % 4 coordinates
+      const float4 q = decode_group(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
       const float qs[4] = {q.x, q.y, q.z, q.w};
       for (uint64_t i = 4 * grp; i < d; ++i) {
         float xi = (kRule == 0) ? x[i] : 0.f, hi = h[i];
@@ -534,16 +585,15 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
 __global__ void __launch_bounds__(kThreads)
 decode_average_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
                       uint32_t M, double inv_m, float* __restrict__ gbar, unsigned int* __restrict__ status) {
-  __shared__ double sm_scale[kMaxWorkers];
-  if (threadIdx.x < M) sm_scale[threadIdx.x] = static_cast<double>(scales[threadIdx.x]);
-  __syncthreads();
+  extern __shared__ double sm_lut[];
+  build_decode_lut(sm_lut, scales, M);
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
   const uint64_t groups = (d + 3) >> 2, full = d >> 2;
   const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
   uint32_t bad = 0;
   for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
-    const float4 q = decode_group(codes8, row_bytes, sm_scale, M, inv_m, grp, bad);
+    const float4 q = decode_group(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
     if (grp < full) {
       *reinterpret_cast<float4*>(gbar + 4 * grp) = q;
     } else {
@@ -605,7 +655,7 @@ void query_launch_shape(LaunchShape* shape) {
   cudaDeviceGetAttribute(&shape->sm_count, cudaDevAttrMultiProcessorCount, dev);
   int a = 0, b = 0;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel, kThreads, 0);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_update_kernel<1>, kThreads, 0);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_update_kernel<1>, kThreads, 2 * 256 * sizeof(double));
   shape->reduce_ctas_per_sm = a > 0 ? a : 1;
   shape->update_ctas_per_sm = b > 0 ? b : 1;
 }
@@ -657,10 +707,11 @@ int launch_decode_update(int rule, const uint32_t* codes, const float* scales, u
                          unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
   const double inv_m = 1.0 / static_cast<double>(M);
   const unsigned grid = update_grid(d, shape);
+  const size_t lut_bytes = static_cast<size_t>((M + 3) / 4) * 256 * sizeof(double);
   if (rule == 0)
-    decode_update_kernel<0><<<grid, kThreads, 0, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
+    decode_update_kernel<0><<<grid, kThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
   else
-    decode_update_kernel<1><<<grid, kThreads, 0, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
+    decode_update_kernel<1><<<grid, kThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
   return 1;
 }
 
@@ -668,8 +719,9 @@ int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d
                           float* gbar, unsigned int* status, const LaunchShape& shape,
                           cudaStream_t stream) {
   const double inv_m = 1.0 / static_cast<double>(M);
-  decode_average_kernel<<<update_grid(d, shape), kThreads, 0, stream>>>(codes, scales, d, M, inv_m, gbar,
-                                                                       status);
+  const size_t lut_bytes = static_cast<size_t>((M + 3) / 4) * 256 * sizeof(double);
+  decode_average_kernel<<<update_grid(d, shape), kThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, gbar,
+                                                                               status);
   return 1;
 }
 
