@@ -155,7 +155,7 @@ __device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64
 }
 
 // ------------------------------------------------------------------ pass A: sum |g|
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
                float* __restrict__ thresholds_out) {
   __shared__ double sm_warp[2][kThreads / 32];
@@ -249,13 +249,29 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
 }
 
 // ------------------------------------------------------------------ pass B helpers
-// One code: 1 for +1, 2 for -1, 0 for 0.
-__device__ __forceinline__ uint32_t ternary_code(float v, bool keep) {
-  return keep ? ((__float_as_uint(v) >> 31) + 1u) : 0u;
+// Code byte of four coordinates, built on the FMA pipe.  pos/neg are 1.0f or 0.0f per
+// coordinate (code 1 = +1, code 2 = -1); the byte value pos0 + 2 neg0 + 4 pos1 + ... + 128 neg3
+// is accumulated on top of 2^23, where an fp32's low mantissa bits are the integer itself.
+struct CodeBits {
+  float pos, neg;
+};
+__device__ __forceinline__ CodeBits split_code(float v, bool keep) {
+  CodeBits c;
+  c.pos = (keep && v > 0.f) ? 1.f : 0.f;
+  c.neg = (keep && v < 0.f) ? 1.f : 0.f;
+  return c;
 }
-
-__device__ __forceinline__ uint32_t pack4(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3) {
-  return c0 + (c1 << 2) + (c2 << 4) + (c3 << 6);
+__device__ __forceinline__ uint32_t pack4(CodeBits c0, CodeBits c1, CodeBits c2, CodeBits c3) {
+  float b = 8388608.f;
+  b = fmaf(c0.pos, 1.f, b);
+  b = fmaf(c0.neg, 2.f, b);
+  b = fmaf(c1.pos, 4.f, b);
+  b = fmaf(c1.neg, 8.f, b);
+  b = fmaf(c2.pos, 16.f, b);
+  b = fmaf(c2.neg, 32.f, b);
+  b = fmaf(c3.pos, 64.f, b);
+  b = fmaf(c3.neg, 128.f, b);
+  return __float_as_uint(b) & 0xffu;
 }
 
 // Number of non-zero 2-bit codes in a byte.
@@ -322,7 +338,7 @@ __device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspac
 }
 
 // ------------------------------------------------------------------ pass B: Q_Delta codes
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
                        uint32_t* __restrict__ codes, float* __restrict__ scales_out,
                        unsigned long long* __restrict__ counts_out) {
@@ -339,32 +355,36 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
-    const float delta = ws.thresholds[m];
+    const float delta = ws.thresholds[m], ndelta = -delta;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    uint32_t cnt = 0;
+    float cntf = 0.f;
     walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t k) {
       double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
       uint32_t bytes[kTileRows];
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
         const float4 t = v[r];
-        const float ax = fabsf(t.x), ay = fabsf(t.y), az = fabsf(t.z), aw = fabsf(t.w);
-        const bool kx = ax > delta, ky = ay > delta, kz = az > delta, kw = aw > delta;
-        if (kx) cx += static_cast<double>(ax);
-        if (ky) cy += static_cast<double>(ay);
-        if (kz) cz += static_cast<double>(az);
-        if (kw) cw += static_cast<double>(aw);
-        bytes[r] = pack4(ternary_code(t.x, kx), ternary_code(t.y, ky), ternary_code(t.z, kz),
-                         ternary_code(t.w, kw));
-        cnt += nonzero_codes(bytes[r]);
+        // strict comparisons; a NaN threshold or value compares false and codes 0
+        const float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
+        const float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
+        const float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
+        const float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+        const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;  // 1.0f where kept
+        // |v| * 1 = |v| and |v| * 0 = +0: the kept magnitudes enter the sum unchanged
+        cx += static_cast<double>(fabsf(t.x) * kx);
+        cy += static_cast<double>(fabsf(t.y) * ky);
+        cz += static_cast<double>(fabsf(t.z) * kz);
+        cw += static_cast<double>(fabsf(t.w) * kw);
+        cntf += (kx + ky) + (kz + kw);  // exact: far below 2^24 per thread and chunk
+        bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
       }
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
       const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
       slot ^= 1;
       if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
     });
-    const unsigned long long total = block_count(cnt, sm_cnt);
+    const unsigned long long total = block_count(static_cast<uint32_t>(cntf), sm_cnt);
     if (j == 0) {
       const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
       ws.part_sum[p] = tile_fold(sm_stack, k1 - k0, geo.log2_group);
@@ -432,8 +452,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
         const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
         const bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
         const bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
-        bytes[r] = pack4(ternary_code(v.x, kx), ternary_code(v.y, ky), ternary_code(v.z, kz),
-                         ternary_code(v.w, kw));
+        bytes[r] = pack4(split_code(v.x, kx), split_code(v.y, ky), split_code(v.z, kz), split_code(v.w, kw));
         cnt += nonzero_codes(bytes[r]);
       }
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
@@ -447,11 +466,25 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
 }
 
 // ------------------------------------------------------------------ pass C helpers
+// Square root and reciprocal from the special-function unit: at most 2 ulp off (relative
+// error below 2.4e-7), two orders of magnitude inside the tolerance on the iterates, for a
+// fraction of the instructions of the correctly rounded forms.  Subnormals are kept.
+__device__ __forceinline__ float sqrt_sfu(float a) {
+  float r;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
+  return r;
+}
+__device__ __forceinline__ float rcp_sfu(float a) {
+  float r;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
+  return r;
+}
+
 // Eq. H_t and Eq. QCMD for one coordinate.
 __device__ __forceinline__ void cmd_update(float q, float& x, float& h, const StepScalars& sc) {
   const float hn = fmaf(q, q, h);
-  const float big_h = sc.delta + __fsqrt_rn(hn);
-  const float rate = sc.eta * __frcp_rn(big_h);
+  const float big_h = sc.delta + sqrt_sfu(hn);
+  const float rate = sc.eta * rcp_sfu(big_h);
   const float u = fmaf(-rate, q, x);
   const float mag = fabsf(u) - sc.lambda * rate;
   x = mag > 0.f ? copysignf(mag, u) : 0.f;
@@ -462,9 +495,9 @@ __device__ __forceinline__ void cmd_update(float q, float& x, float& h, const St
 __device__ __forceinline__ void rda_update(float q, float& x, float& h, float& z, const StepScalars& sc) {
   const float hn = fmaf(q, q, h);
   const float zn = z + q;
-  const float big_h = sc.delta + __fsqrt_rn(hn);
+  const float big_h = sc.delta + sqrt_sfu(hn);
   const float a = fmaf(fabsf(zn), sc.inv_t, -sc.lambda);
-  const float coef = (sc.t * sc.eta) * __frcp_rn(big_h);
+  const float coef = (sc.t * sc.eta) * rcp_sfu(big_h);
   x = a > 0.f ? -copysignf(coef * a, zn) : 0.f;
   h = hn;
   z = zn;
@@ -475,10 +508,14 @@ __device__ __forceinline__ void rda_update(float q, float& x, float& h, float& z
 // in shared memory, in fp64: terms of opposite sign cancel across workers, and the update
 // divides by H = delta + sqrt(h), which can be as small as |q| itself, so q must carry no
 // more than its own fp32 rounding error.
+// kLanes = 1: one copy, [G][256].  kLanes = 32: one copy per lane, [G][256][32], so that the
+// 32 lookups of a warp never meet in a bank (64 KB per group of workers).
+template <int kLanes>
 __device__ __forceinline__ void build_decode_lut(double* lut, const float* __restrict__ scales, uint32_t M) {
   const uint32_t groups = (M + 3) >> 2;
-  for (uint32_t e = threadIdx.x; e < groups * 256; e += kThreads) {
-    const uint32_t grp = e >> 8, idx = e & 255u;
+  for (uint32_t e = threadIdx.x; e < groups * 256 * kLanes; e += blockDim.x) {
+    const uint32_t entry = e / kLanes;
+    const uint32_t grp = entry >> 8, idx = entry & 255u;
     double acc = 0.0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -505,76 +542,118 @@ __device__ __forceinline__ uint32_t transpose_2bit_4x4(uint32_t w) {
 }
 
 // Averaged decoded gradient of the four coordinates of group `grp` (Eq. SynQ_t).
+// kM4 > 0: the number of worker groups ceil(M/4) is a compile-time constant and the loop
+// unrolls; kM4 = 0: any M.
+template <int kM4, int kLanes>
 __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes8, uint64_t row_bytes,
                                                const double* lut, uint32_t M, double inv_m,
                                                uint64_t grp, uint32_t& bad) {
   double q0 = 0.0, q1 = 0.0, q2 = 0.0, q3 = 0.0;
-  const uint8_t* p = codes8 + grp;
-  for (uint32_t m0 = 0; m0 < M; m0 += 4, lut += 256, p += 4 * row_bytes) {
+  const uint32_t m4 = kM4 > 0 ? static_cast<uint32_t>(kM4) : (M + 3) >> 2;
+  if (kLanes > 1) lut += threadIdx.x & 31;
+#pragma unroll
+  for (uint32_t G = 0; G < m4; ++G) {
+    const uint8_t* p = codes8 + grp + static_cast<uint64_t>(4 * G) * row_bytes;
+    const bool whole = (kM4 > 0 && G + 1 < m4);  // only the last group can be short of workers
     uint32_t w = __ldg(p);
-    if (m0 + 1 < M) w |= static_cast<uint32_t>(__ldg(p + row_bytes)) << 8;
-    if (m0 + 2 < M) w |= static_cast<uint32_t>(__ldg(p + 2 * row_bytes)) << 16;
-    if (m0 + 3 < M) w |= static_cast<uint32_t>(__ldg(p + 3 * row_bytes)) << 24;
+    if (whole || 4 * G + 1 < M) w |= static_cast<uint32_t>(__ldg(p + row_bytes)) << 8;
+    if (whole || 4 * G + 2 < M) w |= static_cast<uint32_t>(__ldg(p + 2 * row_bytes)) << 16;
+    if (whole || 4 * G + 3 < M) w |= static_cast<uint32_t>(__ldg(p + 3 * row_bytes)) << 24;
     bad |= w & (w >> 1) & 0x55555555u;
     w = transpose_2bit_4x4(w);
-    q0 += lut[w & 255u];
-    q1 += lut[(w >> 8) & 255u];
-    q2 += lut[(w >> 16) & 255u];
-    q3 += lut[w >> 24];
+    const double* l = lut + static_cast<size_t>(G) * 256 * kLanes;
+    q0 += l[(w & 255u) * kLanes];
+    q1 += l[((w >> 8) & 255u) * kLanes];
+    q2 += l[((w >> 16) & 255u) * kLanes];
+    q3 += l[(w >> 24) * kLanes];
   }
   return make_float4(static_cast<float>(q0 * inv_m), static_cast<float>(q1 * inv_m),
                      static_cast<float>(q2 * inv_m), static_cast<float>(q3 * inv_m));
 }
 
 // ------------------------------------------------------------------ pass C: fused
+// State of one group of four coordinates.
 template <int kRule>
-__global__ void __launch_bounds__(kThreads)
+struct GroupState {
+  float4 h, xz;  // xz: x for QCMD (read and written), z for QRDA
+  __device__ __forceinline__ void load(const float* __restrict__ x, const float* __restrict__ hh,
+                                       const float* __restrict__ z, uint64_t grp) {
+    h = *reinterpret_cast<const float4*>(hh + 4 * grp);
+    xz = *reinterpret_cast<const float4*>((kRule == 0 ? x : z) + 4 * grp);
+  }
+  __device__ __forceinline__ void update_store(float4 q, float* __restrict__ x, float* __restrict__ hh,
+                                               float* __restrict__ z, uint64_t grp, const StepScalars& sc) {
+    if (kRule == 0) {
+      cmd_update(q.x, xz.x, h.x, sc);
+      cmd_update(q.y, xz.y, h.y, sc);
+      cmd_update(q.z, xz.z, h.z, sc);
+      cmd_update(q.w, xz.w, h.w, sc);
+      *reinterpret_cast<float4*>(x + 4 * grp) = xz;
+    } else {
+      float4 xv;
+      rda_update(q.x, xv.x, h.x, xz.x, sc);
+      rda_update(q.y, xv.y, h.y, xz.y, sc);
+      rda_update(q.z, xv.z, h.z, xz.z, sc);
+      rda_update(q.w, xv.w, h.w, xz.w, sc);
+      *reinterpret_cast<float4*>(z + 4 * grp) = xz;
+      *reinterpret_cast<float4*>(x + 4 * grp) = xv;
+    }
+    *reinterpret_cast<float4*>(hh + 4 * grp) = h;
+  }
+};
+
+// kThreadsC threads per CTA; a CTA takes kGroups * kThreadsC consecutive groups per round and a
+// thread owns kGroups of them, kThreadsC apart, with all their loads in flight before it decodes.
+// Up to 12 workers run with per-lane tables (1024 threads, one CTA per SM); more workers share
+// one table per CTA.
+template <int kRule, int kM4, int kLanes, int kThreadsC, int kGroups>
+__global__ void __launch_bounds__(kThreadsC)
 decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
                      uint32_t M, double inv_m, float* __restrict__ x, float* __restrict__ h,
                      float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
   extern __shared__ double sm_lut[];
-  build_decode_lut(sm_lut, scales, M);
+  build_decode_lut<kLanes>(sm_lut, scales, M);
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
   const uint64_t groups = (d + 3) >> 2, full = d >> 2;
-  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * (kGroups * kThreadsC);
   uint32_t bad = 0;
-  for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
-    if (grp < full) {
-      // issue the state loads before the decode so that they overlap it
-      float4 hv = *reinterpret_cast<const float4*>(h + 4 * grp);
-      float4 xv, zv;
-      if (kRule == 0) xv = *reinterpret_cast<const float4*>(x + 4 * grp);
-      else zv = *reinterpret_cast<const float4*>(z + 4 * grp);
-      const float4 q = decode_group(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
-      if (kRule == 0) {
-        cmd_update(q.x, xv.x, hv.x, sc);
-        cmd_update(q.y, xv.y, hv.y, sc);
-        cmd_update(q.z, xv.z, hv.z, sc);
-        cmd_update(q.w, xv.w, hv.w, sc);
-      } else {
-        rda_update(q.x, xv.x, hv.x, zv.x, sc);
-        rda_update(q.y, xv.y, hv.y, zv.y, sc);
-        rda_update(q.z, xv.z, hv.z, zv.z, sc);
-        rda_update(q.w, xv.w, hv.w, zv.w, sc);
-        *reinterpret_cast<float4*>(z + 4 * grp) = zv;
-      }
-      *reinterpret_cast<float4*>(h + 4 * grp) = hv;
-      *reinterpret_cast<float4*>(x + 4 * grp) = xv;
-    } else {  // ragged tail: d % 4 coordinates
-      const float4 q = decode_group(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
-      const float qs[4] = {q.x, q.y, q.z, q.w};
-      for (uint64_t i = 4 * grp; i < d; ++i) {
-        float xi = (kRule == 0) ? x[i] : 0.f, hi = h[i];
-        if (kRule == 0) {
-          cmd_update(qs[i - 4 * grp], xi, hi, sc);
-        } else {
-          float zi = z[i];
-          rda_update(qs[i - 4 * grp], xi, hi, zi, sc);
-          z[i] = zi;
+  for (uint64_t g0 = static_cast<uint64_t>(blockIdx.x) * (kGroups * kThreadsC) + threadIdx.x; g0 < groups;
+       g0 += stride) {
+    if (g0 + (kGroups - 1) * kThreadsC < full) {
+      GroupState<kRule> s[kGroups];
+#pragma unroll
+      for (int i = 0; i < kGroups; ++i) s[i].load(x, h, z, g0 + i * kThreadsC);
+      float4 q[kGroups];
+#pragma unroll
+      for (int i = 0; i < kGroups; ++i)
+        q[i] = decode_group<kM4, kLanes>(codes8, row_bytes, sm_lut, M, inv_m, g0 + i * kThreadsC, bad);
+#pragma unroll
+      for (int i = 0; i < kGroups; ++i) s[i].update_store(q[i], x, h, z, g0 + i * kThreadsC, sc);
+      continue;
+    }
+    for (int i = 0; i < kGroups; ++i) {  // the last round, group by group
+      const uint64_t grp = g0 + static_cast<uint64_t>(i) * kThreadsC;
+      if (grp >= groups) break;
+      const float4 q = decode_group<kM4, kLanes>(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
+      if (grp < full) {
+        GroupState<kRule> s0;
+        s0.load(x, h, z, grp);
+        s0.update_store(q, x, h, z, grp, sc);
+      } else {  // ragged tail: d % 4 coordinates
+        const float qs[4] = {q.x, q.y, q.z, q.w};
+        for (uint64_t c = 4 * grp; c < d; ++c) {
+          float xi = (kRule == 0) ? x[c] : 0.f, hi = h[c];
+          if (kRule == 0) {
+            cmd_update(qs[c - 4 * grp], xi, hi, sc);
+          } else {
+            float zi = z[c];
+            rda_update(qs[c - 4 * grp], xi, hi, zi, sc);
+            z[c] = zi;
+          }
+          x[c] = xi;
+          h[c] = hi;
         }
-        x[i] = xi;
-        h[i] = hi;
       }
     }
   }
@@ -586,14 +665,14 @@ __global__ void __launch_bounds__(kThreads)
 decode_average_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
                       uint32_t M, double inv_m, float* __restrict__ gbar, unsigned int* __restrict__ status) {
   extern __shared__ double sm_lut[];
-  build_decode_lut(sm_lut, scales, M);
+  build_decode_lut<1>(sm_lut, scales, M);
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
   const uint64_t groups = (d + 3) >> 2, full = d >> 2;
   const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
   uint32_t bad = 0;
   for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
-    const float4 q = decode_group(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
+    const float4 q = decode_group<0, 1>(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
     if (grp < full) {
       *reinterpret_cast<float4*>(gbar + 4 * grp) = q;
     } else {
@@ -655,7 +734,7 @@ void query_launch_shape(LaunchShape* shape) {
   cudaDeviceGetAttribute(&shape->sm_count, cudaDevAttrMultiProcessorCount, dev);
   int a = 0, b = 0;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel, kThreads, 0);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_update_kernel<1>, kThreads, 2 * 256 * sizeof(double));
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_average_kernel, kThreads, 2 * 256 * sizeof(double));
   shape->reduce_ctas_per_sm = a > 0 ? a : 1;
   shape->update_ctas_per_sm = b > 0 ? b : 1;
 }
@@ -702,16 +781,57 @@ int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, 
   return 1;
 }
 
+// One instantiation of the fused pass C and its launch shape.
+template <int kRule, int kM4, int kLanes, int kThreadsC, int kGroups>
+static void launch_decode_update_as(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
+                                    float* x, float* h, float* z, const StepScalars& sc,
+                                    unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
+  auto kernel = decode_update_kernel<kRule, kM4, kLanes, kThreadsC, kGroups>;
+  const size_t lut_bytes = static_cast<size_t>((M + 3) / 4) * 256 * kLanes * sizeof(double);
+  static thread_local int ctas_per_sm[64] = {0};  // per device, resolved on first use
+  int dev = 0;
+  cudaGetDevice(&dev);
+  int& resident = ctas_per_sm[dev & 63];
+  if (resident == 0) {
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(lut_bytes));
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kThreadsC, lut_bytes);
+    if (resident < 1) resident = 1;
+  }
+  const uint64_t groups = (d + 3) >> 2;
+  const uint64_t per_cta = static_cast<uint64_t>(kThreadsC) * kGroups;
+  uint64_t grid = (groups + per_cta - 1) / per_cta;
+  const uint64_t max_grid = static_cast<uint64_t>(shape.sm_count) * resident;
+  if (grid > max_grid) grid = max_grid;
+  const double inv_m = 1.0 / static_cast<double>(M);
+  kernel<<<static_cast<unsigned>(grid), kThreadsC, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc,
+                                                                        status);
+}
+
+template <int kRule>
+static void launch_decode_update_rule(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
+                                      float* x, float* h, float* z, const StepScalars& sc,
+                                      unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
+  constexpr int kG = kRule == 0 ? 2 : 1;  // groups per thread with per-lane tables (measured best)
+#define QASG_LANE(m4) \
+  case m4: launch_decode_update_as<kRule, m4, 32, 1024, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+#define QASG_SHARED(m4) \
+  case m4: launch_decode_update_as<kRule, m4, 1, kThreads, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+  switch ((M + 3) / 4) {
+    QASG_LANE(1) QASG_LANE(2) QASG_LANE(3)
+    QASG_SHARED(4) QASG_SHARED(5) QASG_SHARED(6) QASG_SHARED(7) QASG_SHARED(8) QASG_SHARED(9) QASG_SHARED(10)
+    QASG_SHARED(11) QASG_SHARED(12) QASG_SHARED(13) QASG_SHARED(14) QASG_SHARED(15) QASG_SHARED(16)
+  }
+#undef QASG_LANE
+#undef QASG_SHARED
+}
+
 int launch_decode_update(int rule, const uint32_t* codes, const float* scales, uint64_t d,
                          uint32_t M, float* x, float* h, float* z, const StepScalars& sc,
                          unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
-  const double inv_m = 1.0 / static_cast<double>(M);
-  const unsigned grid = update_grid(d, shape);
-  const size_t lut_bytes = static_cast<size_t>((M + 3) / 4) * 256 * sizeof(double);
   if (rule == 0)
-    decode_update_kernel<0><<<grid, kThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
+    launch_decode_update_rule<0>(codes, scales, d, M, x, h, z, sc, status, shape, stream);
   else
-    decode_update_kernel<1><<<grid, kThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc, status);
+    launch_decode_update_rule<1>(codes, scales, d, M, x, h, z, sc, status, shape, stream);
   return 1;
 }
 

@@ -230,6 +230,26 @@ def test_sweep_one_step(ctx, d, M, rule):
     U.assert_zero_pattern(x, ref["x"], ref["a"], LAM)
 
 
+@pytest.mark.parametrize("M", [1, 5, 9, 12, 13, 31, 64])
+@pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
+def test_fused_step_worker_counts(ctx, M, rule):
+    # every dispatch of the decode: per-lane tables (M <= 12), shared tables, short last group
+    d = 70_003
+    g = inputs.optimizer_only_gradients(d, M, t=3, seed=M) * np.float32(0.01)
+    x0, h0, z0 = (v.numpy() for v in inputs.random_state(d, seed=M))
+    g_dev, ld = U.grad_to_dev(g)
+    x, h, z = U.to_dev(x0), U.to_dev(h0), U.to_dev(z0)
+    codes = U.new_codes(M, d)
+    ctx.step(rule, g_dev, d, ld, M, 3, libqasg.make_params(LAM, ETA, DELTA), x, h, z, codes_out=codes)
+    assert ctx.last_async_status() == libqasg.OK
+    ref = O.step(rule, g, x0, h0, z0, 3, LAM, ETA, DELTA)
+    assert np.array_equal(U.codes_np(codes), ref["quant"]["codes"])
+    U.assert_close(x, ref["x"], "x"), U.assert_close(h, ref["h"], "h")
+    if rule == libqasg.RULE_RDA:
+        U.assert_close(z, ref["z"], "z")
+    U.assert_zero_pattern(x, ref["x"], ref["a"], LAM)
+
+
 def test_step_host_matches_step(ctx):
     d, M, t = 50_003, 4, 5
     g = inputs.optimizer_only_gradients(d, M, t, seed=1)
