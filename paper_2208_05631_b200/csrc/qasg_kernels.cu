@@ -71,21 +71,6 @@ __device__ __forceinline__ double warp_pair_tree(double v) {
   return v;
 }
 
-// Pairwise tree over the 1024 column sums of a tile: v is the thread's sum of its 4
-// columns.  The result is valid in thread 0.  `slot` alternates between calls so that
-// one barrier per tile is enough.
-__device__ __forceinline__ double block_pair_tree(double v, double (*sm)[kThreads / 32], int slot) {
-  v = warp_pair_tree(v);
-  if ((threadIdx.x & 31) == 0) sm[slot][threadIdx.x >> 5] = v;
-  __syncthreads();
-  double r = 0.0;
-  if (threadIdx.x == 0) {
-    const double* a = sm[slot];
-    r = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
-  }
-  return r;
-}
-
 // Streaming pairwise summation over the tiles of a chunk (thread 0 only): stack[l] holds
 // the sum of a complete aligned subtree of 2^l tiles.
 __device__ __forceinline__ void tile_push(double* stack, uint32_t k_local, double v) {
@@ -104,6 +89,56 @@ __device__ __forceinline__ double tile_fold(const double* stack, uint32_t n, uin
     if ((n >> lvl) & 1u) carry = stack[lvl] + carry;
   return carry;
 }
+
+// Fixed-order sum over the tiles of one chunk.  Every tile, each thread contributes the sum
+// of its 4 columns; the warp butterfly runs at once, but the eight warp sums of a tile are only
+// parked in shared memory.  Every kBatchTiles tiles (and at the end of the chunk) the CTA meets
+// once: the parked sums are combined tile by tile (pairwise over the 8 warps), then pushed, in
+// tile order, onto the chunk's pairwise stack.  The order of additions is the same as if every
+// tile had been reduced on its own; the warps just do not wait for each other at every tile.
+constexpr int kBatchTiles = 64;
+struct ChunkSumStorage {
+  double warp_sums[kBatchTiles][kThreads / 32];
+  double tile_sums[kBatchTiles];
+  double stack[32];
+};
+
+class ChunkSum {
+ public:
+  __device__ __forceinline__ ChunkSum(ChunkSumStorage* st) : st_(st), pending_(0), pushed_(0) {}
+
+  // Called by all threads, once per tile, in tile order.
+  __device__ __forceinline__ void add_tile(double thread_sum) {
+    const double v = warp_pair_tree(thread_sum);
+    if ((threadIdx.x & 31) == 0) st_->warp_sums[pending_][threadIdx.x >> 5] = v;
+    if (++pending_ == kBatchTiles) flush();
+  }
+
+  // Called by all threads after the chunk's last tile; the chunk sum is valid in thread 0.
+  __device__ __forceinline__ double finish(uint32_t log2_group) {
+    if (pending_) flush();
+    double r = 0.0;
+    if (threadIdx.x == 0) r = tile_fold(st_->stack, pushed_, log2_group);
+    pushed_ = 0;
+    return r;
+  }
+
+ private:
+  __device__ __forceinline__ void flush() {
+    __syncthreads();
+    if (threadIdx.x < pending_) {
+      const double* a = st_->warp_sums[threadIdx.x];
+      st_->tile_sums[threadIdx.x] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (uint32_t i = 0; i < pending_; ++i) tile_push(st_->stack, pushed_ + i, st_->tile_sums[i]);
+    pushed_ += pending_;
+    pending_ = 0;
+  }
+  ChunkSumStorage* st_;
+  uint32_t pending_, pushed_;
+};
 
 // Pairwise tree over a worker's kMaxChunks partial slots (slots >= chunks are +0.0),
 // computed by one warp: 32 adjacent slots per lane, then the lane butterfly.
@@ -158,18 +193,17 @@ __device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64
 __global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
                float* __restrict__ thresholds_out) {
-  __shared__ double sm_warp[2][kThreads / 32];
-  __shared__ double sm_stack[32];
+  __shared__ ChunkSumStorage sm_sum;
   __shared__ bool sm_last;
   const int j = threadIdx.x;
   const uint32_t n_items = geo.M * geo.chunks;
-  int slot = 0;
+  ChunkSum chunk_sum(&sm_sum);
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t k) {
+    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t) {
       double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
 #pragma unroll
       for (int r = 1; r < kTileRows; ++r) {
@@ -178,12 +212,10 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
         cz += static_cast<double>(fabsf(v[r].z));
         cw += static_cast<double>(fabsf(v[r].w));
       }
-      const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
-      slot ^= 1;
-      if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
+      chunk_sum.add_tile((cx + cy) + (cz + cw));
     });
-    if (j == 0)
-      ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = tile_fold(sm_stack, k1 - k0, geo.log2_group);
+    const double total = chunk_sum.finish(geo.log2_group);
+    if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
   }
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   const int warp = j >> 5, lane = j & 31;
@@ -280,18 +312,19 @@ __device__ __forceinline__ uint32_t nonzero_codes(uint32_t byte) {
 }
 
 // Writes the code bytes of the thread's four rows of tile k.  codes8 is the worker's code
-// row; only the last tile can reach past the row's last byte.
+// row; only the last tile can reach past the row's last byte.  The stores are streaming
+// (evict-first): the codes are read back only after the whole gradient has gone by.
 __device__ __forceinline__ void store_code_bytes(uint8_t* __restrict__ codes8, uint32_t k, int j,
                                                  bool full, uint64_t row_bytes,
                                                  const uint32_t (&bytes)[kTileRows]) {
   const uint64_t b0 = static_cast<uint64_t>(k) * (kTile / 4) + j;
   if (full) {
 #pragma unroll
-    for (int r = 0; r < kTileRows; ++r) codes8[b0 + r * (kTileCols / 4)] = static_cast<uint8_t>(bytes[r]);
+    for (int r = 0; r < kTileRows; ++r) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
   } else {
 #pragma unroll
     for (int r = 0; r < kTileRows; ++r)
-      if (b0 + r * (kTileCols / 4) < row_bytes) codes8[b0 + r * (kTileCols / 4)] = static_cast<uint8_t>(bytes[r]);
+      if (b0 + r * (kTileCols / 4) < row_bytes) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
   }
 }
 
@@ -342,15 +375,14 @@ __global__ void __launch_bounds__(kThreads, 4)
 threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
                        uint32_t* __restrict__ codes, float* __restrict__ scales_out,
                        unsigned long long* __restrict__ counts_out) {
-  __shared__ double sm_warp[2][kThreads / 32];
-  __shared__ double sm_stack[32];
+  __shared__ ChunkSumStorage sm_sum;
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
   const uint32_t n_items = geo.M * geo.chunks;
   const uint64_t row_words = (geo.d + 15) >> 4;
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
-  int slot = 0;
+  ChunkSum chunk_sum(&sm_sum);
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
@@ -380,14 +412,13 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
         bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
       }
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
-      const double tile_sum = block_pair_tree((cx + cy) + (cz + cw), sm_warp, slot);
-      slot ^= 1;
-      if (j == 0) tile_push(sm_stack, k - k0, tile_sum);
+      chunk_sum.add_tile((cx + cy) + (cz + cw));
     });
+    const double picked = chunk_sum.finish(geo.log2_group);
     const unsigned long long total = block_count(static_cast<uint32_t>(cntf), sm_cnt);
     if (j == 0) {
       const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
-      ws.part_sum[p] = tile_fold(sm_stack, k1 - k0, geo.log2_group);
+      ws.part_sum[p] = picked;
       ws.part_cnt[p] = total;
     }
   }
