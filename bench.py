@@ -154,6 +154,21 @@ def workload_config(args, note):
             "parallelism": "replicas" if args.gpus > 1 else "single", "note": note}
 
 
+# ------------------------------------------------------------------ multi-rank aggregation
+def max_over_ranks(ms, dist, device):
+    """Slowest rank's time: every rank runs an independent replica, the job is as slow as the slowest."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, d, M, ms_per_step):
+    """Coordinate-workers per second over all replicas: one bench step is 2 fused steps of d*M."""
+    return world * 2.0 * d * M / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------ our arm
 def run_ours(args, rank, world):
     from paper_2208_05631_b200 import libqasg
@@ -204,12 +219,9 @@ def run_ours(args, rank, world):
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     assert ctx.last_async_status() == libqasg.OK
-    if dist is not None:
-        tmax = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
     ms_per_step = elapsed_ms / args.steps
-    value = world * 2.0 * d * M / (ms_per_step * 1e-3)
+    value = whole_job_value(world, d, M, ms_per_step)
 
     # ---------------------------------------------------------------- end to end, host buffers
     e2e = None
@@ -291,15 +303,11 @@ def run_e2e(args, ctx, params, g, x0, h0, z0, dev, dist, world):
         host_step()
     stop.record()
     torch.cuda.synchronize()
-    ms = start.elapsed_time(stop)
-    if dist is not None:
-        tmax = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = max_over_ranks(start.elapsed_time(stop), dist, dev)
     vec = 4 * d
     h2d = 2 * 4 * d * M + (2 * vec) + (2 * vec)      # g twice; QCMD: x, h; QRDA: h, z
     d2h = (2 * vec) + (3 * vec)                      # QCMD: x, h; QRDA: x, h, z
-    return {"value": world * 2.0 * d * M / (ms / steps * 1e-3), "unit": UNIT, "ms_per_step": ms / steps,
+    return {"value": whole_job_value(world, d, M, ms / steps), "unit": UNIT, "ms_per_step": ms / steps,
             "steps": steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
 
