@@ -1,0 +1,148 @@
+"""Timing sweeps of libqasg on one GPU, beyond the single workload bench.py reports.
+
+  python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--max-log2-d 28]
+  python -m paper_2208_05631_b200.sweep logreg [--steps 50]
+
+`step`   - the fused step over d in {2^20 .. 2^28} x M in {2, 4, 8, 16, 32} simulated workers,
+           N(0,1) gradients, both update rules (the paper uses 2-4 workers; this is the scaling
+           of the step in d and in the number of workers).  L2 is flushed before every timed
+           step, so small sizes are not flattered by gradients that stay in the 126 MB L2.
+`logreg` - the two L1-logistic-regression workloads: gradient kernel + fused step per iteration.
+           dense: X 65536 x 4096, 8 workers, minibatch 512; sparse: 10^6 x 2^24 CSR, ~80 non-zeros
+           per row, 16 workers, minibatch 1024.
+
+Prints one JSON line per measured point.  Every number is device time from CUDA events.
+"""
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import inputs, libqasg
+
+LAM, ETA, DELTA, T_STEP = 1e-3, 0.1, 1e-8, 16
+
+
+def _flush_l2(buf):
+    buf.add_(1.0)
+
+
+def _time_calls(fn, reps, flush_buf):
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    for _ in range(reps):
+        if flush_buf is not None:
+            _flush_l2(flush_buf)
+        start.record()
+        fn()
+        stop.record()
+        torch.cuda.synchronize()
+        times.append(start.elapsed_time(stop))
+    return float(np.median(times)), float(min(times))
+
+
+def sweep_step(args):
+    dev = torch.device("cuda", 0)
+    flush = torch.zeros(64 << 20, dtype=torch.float32, device=dev)      # 256 MB > L2
+    quantizer = libqasg.Q_THRESHOLD if args.quantizer == "threshold" else libqasg.Q_TERNARY_STOCH
+    params = libqasg.make_params(LAM, ETA, DELTA, quantizer=quantizer, seed=4)
+    for log2d in range(20, args.max_log2_d + 1, 2):
+        d = 1 << log2d
+        for M in (2, 4, 8, 16, 32):
+            g = inputs.normal_gradients(d, M, seed=4, device=dev)
+            x, h, z = inputs.random_state(d, seed=4, device=dev)
+            ctx = libqasg.Context(d, M, device=0)
+            for rule, name, state_bytes in ((libqasg.RULE_CMD, "qcmd", 16), (libqasg.RULE_RDA, "qrda", 20)):
+                def one():
+                    ctx.step(rule, g, d, d, M, T_STEP, params, x, h, z)
+                for _ in range(3):
+                    one()
+                torch.cuda.synchronize()
+                med, best = _time_calls(one, args.reps, flush)
+                moved = d * (8.0 * M + M / 2.0 + state_bytes)
+                print(json.dumps({"what": "step", "quantizer": args.quantizer, "rule": name, "d": d, "M": M,
+                                  "ms_median": med, "ms_best": best, "coord_workers_per_s": d * M / (med * 1e-3),
+                                  "gbs_moved": moved / 1e9 / (med * 1e-3)}), flush=True)
+            assert ctx.last_async_status() == libqasg.OK
+            ctx.close()
+            del g, x, h, z
+            torch.cuda.empty_cache()
+
+
+def _timed_iterations(ctx, it, warm, steps):
+    for _ in range(warm):
+        it()
+    torch.cuda.synchronize()
+    ctx.profile_begin()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        it()
+    stop.record()
+    torch.cuda.synchronize()
+    kernels = ctx.profile_end()
+    return start.elapsed_time(stop) * 1e3 / steps, {k: v[0] * 1e3 / v[1] for k, v in kernels.items()}
+
+
+def sweep_logreg(args):
+    dev = torch.device("cuda", 0)
+    # dense: "L1-regularised logistic regression, dense synthetic"
+    n, d, M, B = 65536, 4096, 8, 512
+    prob = inputs.logreg_dense_problem(n=n, d=d, M=M, seed=1)
+    X, y = torch.from_numpy(prob["X"]).to(dev), torch.from_numpy(prob["y"]).to(dev)
+    ctx = libqasg.Context(1 << 24, 16, device=0)
+    for rule, name in ((libqasg.RULE_CMD, "qcmd"), (libqasg.RULE_RDA, "qrda")):
+        params = libqasg.make_params(1e-4, ETA, DELTA)
+        x, h, z = (torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(3))
+        g = torch.empty((M, d), dtype=torch.float32, device=dev)
+        t = [0]
+
+        def it():
+            t[0] += 1
+            ctx.logreg_grad_dense(X, y, n, d, M, prob["shard_row0"], None, B, t[0], x, g, d)
+            ctx.step(rule, g, d, d, M, t[0], params, x, h, z)
+        us, kernel_us = _timed_iterations(ctx, it, 5, args.steps)
+        print(json.dumps({"what": "logreg_dense", "rule": name, "n": n, "d": d, "M": M, "B": B,
+                          "us_per_iteration": us, "kernel_us": kernel_us,
+                          "nnz_x": int((x != 0).sum().item())}), flush=True)
+    del X, y
+    # sparse: "sparse-feature logistic regression"
+    n, d, M, B = args.csr_rows, 1 << 24, 16, 1024
+    prob = inputs.logreg_csr_problem(n=n, d=d, M=M, nnz_per_row=80, seed=3)
+    dev_args = [torch.from_numpy(prob[k]).to(dev) for k in ("rowptr", "colidx", "vals", "y")]
+    params = libqasg.make_params(1e-5, ETA, DELTA)
+    x, h, z = (torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(3))
+    g = torch.empty((M, d), dtype=torch.float32, device=dev)
+    t = [0]
+
+    def it_csr():
+        t[0] += 1
+        ctx.logreg_grad_csr(*dev_args, n, d, M, prob["shard_row0"], None, B, t[0], x, g, d)
+        ctx.step(libqasg.RULE_RDA, g, d, d, M, t[0], params, x, h, z)
+    us, kernel_us = _timed_iterations(ctx, it_csr, 3, args.steps)
+    print(json.dumps({"what": "logreg_csr", "rule": "qrda", "n": n, "d": d, "M": M, "B": B,
+                      "nnz": int(prob["rowptr"][-1]), "us_per_iteration": us, "kernel_us": kernel_us,
+                      "nnz_x": int((x != 0).sum().item())}), flush=True)
+    assert ctx.last_async_status() == libqasg.OK
+    ctx.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["step", "logreg"])
+    ap.add_argument("--quantizer", default="threshold", choices=["threshold", "stochastic"])
+    ap.add_argument("--max-log2-d", type=int, default=28)
+    ap.add_argument("--reps", type=int, default=7)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--csr-rows", type=int, default=1_000_000)
+    args = ap.parse_args()
+    assert torch.cuda.is_available(), "needs a CUDA device"
+    if args.what == "step":
+        sweep_step(args)
+    else:
+        sweep_logreg(args)
+
+
+if __name__ == "__main__":
+    main()
