@@ -211,14 +211,37 @@ def wire_bits(d):
 # Server side: decode and average (SynQ_t)
 # ----------------------------------------------------------------------------------
 def decode_average(terns, scales):
-    """SynQ_t = (1/M) sum_m s_m * tern_m, in fp64."""
+    """SynQ_t = (1/M) * sum_m s_m * tern_m, in fp64: the sum over workers in worker order,
+    times the fp64 reciprocal of M (the product form in which the equation is written)."""
     terns = np.asarray(terns)
     scales = np.asarray(scales, dtype=F32)
     m_workers = terns.shape[0]
     acc = np.zeros(terns.shape[1], dtype=F64)
     for m in range(m_workers):
         acc = acc + F64(scales[m]) * terns[m].astype(F64)
-    return acc / F64(m_workers)
+    return acc * (F64(1.0) / F64(m_workers))
+
+
+def requantize(gbar, quantizer, t=1, seed=0, coef=0.75):
+    """Server side of Algorithm 1, "Quantize the aggregated gradient": q_t = Q(SynQ_t).
+
+    The averaged gradient is held in fp32 (it is what would be sent), so gbar (fp64) is rounded
+    to fp32 first and Q is applied to that vector exactly as it is applied to a worker's
+    gradient.  The stochastic quantizer draws from the Philox stream of domain 1, worker 0.
+    Returns dict(tern int8[d], scale fp32, threshold fp32, count int, codes uint32[W], q fp64[d]).
+    """
+    gbar32 = np.asarray(gbar, dtype=F64).astype(F32)
+    d = gbar32.size
+    if quantizer == QUANT_THRESHOLD:
+        tern, scale, threshold, count = threshold_quantize(gbar32, coef)
+    elif quantizer == QUANT_TERNARY_STOCH:
+        _, u = philox_draws(seed, t, 0, np.arange(d, dtype=np.uint64), domain=1)
+        tern, scale = ternary_stochastic_quantize(gbar32, u)
+        threshold, count = F32(0.0), int(np.count_nonzero(tern))
+    else:
+        raise ValueError("quantizer")
+    return dict(tern=tern, scale=F32(scale), threshold=F32(threshold), count=int(count),
+                codes=pack_codes(tern), q=F64(scale) * tern.astype(F64), gbar32=gbar32)
 
 
 # ----------------------------------------------------------------------------------
@@ -306,9 +329,13 @@ def quantize_workers(g, quantizer, t=1, seed=0, coef=0.75):
     return dict(terns=terns, scales=scales, thresholds=thresholds, counts=counts, codes=codes)
 
 
-def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0, coef=0.75):
+def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0, coef=0.75,
+         double_quant=False):
     """One iteration: quantize every worker's gradient, decode and average, update the
     accumulator and apply the rule's closed-form update.  State in, state out (fp64).
+
+    double_quant=True is Algorithm 1 as printed: the average is quantized again on the server
+    (q_t = Q(SynQ_t)) and the workers update from q_t; False is the one-way variant.
 
     quantizer == QUANT_NONE skips quantization: q is the fp64 mean of the rows of g
     (the 32-bit CMD / RDA adagrad baseline).
@@ -322,6 +349,12 @@ def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0
     else:
         quant = quantize_workers(g, quantizer, t=t, seed=seed, coef=coef)
         q = decode_average(quant["terns"], quant["scales"])
+    requant = None
+    if double_quant:
+        if quantizer == QUANT_NONE:
+            raise ValueError("double quantization needs a quantizer")
+        requant = requantize(q, quantizer, t=t, seed=seed, coef=coef)
+        q = requant["q"]
     if rule == RULE_CMD:
         x_new, h_new, a = cmd_step(q, x, h, lam, eta, delta)
         z_new = None if z is None else np.asarray(z, dtype=F64)
@@ -329,4 +362,4 @@ def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0
         x_new, h_new, z_new, a = rda_step(q, h, z, t, lam, eta, delta)
     else:
         raise ValueError("rule")
-    return dict(x=x_new, h=h_new, z=z_new, a=a, q=q, quant=quant)
+    return dict(x=x_new, h=h_new, z=z_new, a=a, q=q, quant=quant, requant=requant)

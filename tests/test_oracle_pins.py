@@ -363,3 +363,68 @@ def test_fused_step_composes_its_parts():
     assert np.mean(out["x"] == 0) > 0.0                      # some exact zeros
     nzmask = out["x"] != 0
     assert (np.sign(out["x"][nzmask]) == -np.sign(out["z"][nzmask])).all()
+
+
+# ------------------------------------------------------------------ double quantization
+def test_threshold_quantizer_is_idempotent():
+    # Q(Q(v)) = Q(v): the entries of Q(v) are 0 or +-s, the threshold 0.75*s*n/d is below s, so
+    # exactly the non-zero entries are kept and their mean magnitude is s again.
+    rng = np.random.default_rng(21)
+    for d in (9, 1000, 50_001):
+        v = rng.standard_normal(d).astype(np.float32) * np.float32(0.3)
+        tern, s, _, n = O.threshold_quantize(v)
+        again = O.requantize(float(s) * tern.astype(np.float64), O.QUANT_THRESHOLD)
+        assert np.array_equal(again["tern"], tern) and again["scale"] == s and again["count"] == n
+        assert np.array_equal(again["q"], float(s) * tern)
+
+
+def test_requantize_is_q_applied_to_the_fp32_average():
+    rng = np.random.default_rng(22)
+    d, M = 3000, 5
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    quant = O.quantize_workers(g, O.QUANT_THRESHOLD)
+    gbar = O.decode_average(quant["terns"], quant["scales"])
+    rq = O.requantize(gbar, O.QUANT_THRESHOLD)
+    gbar32 = gbar.astype(np.float32)
+    # threshold and scale by their definitions (Section 3.5, Section 3.4), from plain fp64 sums
+    delta = 0.75 * np.abs(gbar32.astype(np.float64)).sum() / d
+    assert float(rq["threshold"]) == pytest.approx(delta, rel=1e-6)
+    kept = np.abs(gbar32) > rq["threshold"]
+    assert rq["count"] == int(kept.sum()) and np.array_equal(rq["tern"] != 0, kept)
+    assert np.array_equal(np.sign(rq["tern"]), np.sign(gbar32) * kept)
+    assert float(rq["scale"]) == pytest.approx(np.abs(gbar32.astype(np.float64))[kept].mean(), rel=1e-6)
+    # error identity of the second quantization: ||gbar - q||^2 = ||gbar||^2 - n s^2
+    err = float(((gbar32.astype(np.float64) - rq["q"]) ** 2).sum())
+    assert err == pytest.approx(float((gbar32.astype(np.float64) ** 2).sum()) - rq["count"] * float(rq["scale"]) ** 2, rel=1e-5)
+    assert np.array_equal(O.unpack_codes(rq["codes"], d), rq["tern"])
+
+
+def test_double_quantized_step_uses_q_of_the_average():
+    rng = np.random.default_rng(23)
+    d, M = 800, 4
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    x0, h0, z0 = rng.standard_normal(d) * 0.1, rng.random(d), rng.standard_normal(d) * 0.1
+    one = O.step(O.RULE_RDA, g, x0, h0, z0, 7, 1e-3, 0.1, 1e-8)
+    two = O.step(O.RULE_RDA, g, x0, h0, z0, 7, 1e-3, 0.1, 1e-8, double_quant=True)
+    rq = two["requant"]
+    assert one["requant"] is None and np.array_equal(two["quant"]["codes"], one["quant"]["codes"])
+    assert np.array_equal(rq["gbar32"], one["q"].astype(np.float32))
+    assert set(np.unique(two["q"])) <= {-float(rq["scale"]), 0.0, float(rq["scale"])}
+    assert np.allclose(two["z"], z0 + two["q"], rtol=1e-15) and np.allclose(two["h"], h0 + two["q"] ** 2, rtol=1e-15)
+    # quantizing twice adds error: the paper's remark that one-way quantization is less noisy
+    assert ((two["q"] - one["q"]) ** 2).sum() > 0
+
+
+def test_stochastic_requantize_uses_its_own_stream_and_is_unbiased():
+    gbar = np.array([0.5, -0.25, 0.0, 0.125, -0.5, 0.3], dtype=np.float64)
+    trials = 60_000
+    total = np.zeros(gbar.size)
+    for t in range(1, trials + 1):
+        total += O.requantize(gbar, O.QUANT_TERNARY_STOCH, t=t, seed=5)["q"]
+    p = np.abs(gbar) / 0.5
+    sigma = 0.5 * np.sqrt(p * (1 - p) / trials)
+    assert (np.abs(total / trials - gbar) <= 5 * sigma + 1e-12).all()
+    a = O.requantize(np.linspace(-1, 1, 64), O.QUANT_TERNARY_STOCH, t=3, seed=9)
+    _, u_worker0 = O.philox_draws(9, 3, 0, np.arange(64, dtype=np.uint64), domain=0)
+    tern_w, _ = O.ternary_stochastic_quantize(np.linspace(-1, 1, 64).astype(np.float32), u_worker0)
+    assert not np.array_equal(a["tern"], tern_w)          # domain 1 is a different stream
