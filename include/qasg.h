@@ -139,6 +139,32 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
                       uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h,
                       float* z, uint32_t* codes_out, float* scales_out, void* stream);
 
+/* Server's side of Algorithm 1 with double quantization ("Quantize the aggregated gradient",
+ * Eq. q_t = Q(SynQ_t)): decodes and averages the workers' codes as qasg_decode_average does, rounds
+ * the average to fp32, and applies the same Q to it as to a worker's gradient, without ever
+ * storing the average.
+ *   codes, scales  device, the workers' messages as written by qasg_quantize_pack.
+ *   qcodes         device, uint32 [qasg_code_words(d)]: the codes of q_t, same layout as one worker row.
+ *   qscale         device, fp32 [1]: the scale of q_t.
+ *   qthreshold     device, fp32 [1] or NULL: its threshold (0 for the stochastic quantizer).
+ *   qcount         device, uint64 [1] or NULL: its number of non-zero codes.
+ * The stochastic quantizer draws from the Philox stream with counter word 1 = 1<<16 (a stream of
+ * its own: the workers use 0 .. M-1 there).  The workers then recover q_t with
+ * qasg_decode_average(qcodes, qscale, d, 1, ...) and update with qasg_cmd_step / qasg_rda_step. */
+qasg_status qasg_requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d,
+                            uint32_t M, uint64_t t, const qasg_params* params, uint32_t* qcodes,
+                            float* qscale, float* qthreshold, uint64_t* qcount, void* stream);
+
+/* The whole iteration of Algorithm 1 as printed, with both quantizations: qasg_quantize_pack,
+ * qasg_requantize, then decode of q_t + accumulator + update in one pass.  Arguments as for
+ * qasg_step, plus
+ *   qcodes_out  device uint32 [code_words(d)] or NULL to use the context's scratch.
+ *   qscale_out  device fp32 [1] or NULL. */
+qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
+                             uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h,
+                             float* z, uint32_t* codes_out, float* scales_out, uint32_t* qcodes_out,
+                             float* qscale_out, void* stream);
+
 /* qasg_step for callers whose data lives in host memory.  Copies g (M rows of d floats,
  * row stride ld_g) and the state from the host buffers into the caller's device staging
  * buffers, runs qasg_step there, and copies the new state back, all on `stream`; returns
@@ -227,7 +253,7 @@ uint64_t qasg_launch_count(const qasg_ctx* ctx);
  * adds up, per kernel id (0 <= id < QASG_KERNEL_COUNT, names from qasg_kernel_name), the
  * elapsed milliseconds into ms[id] and the number of launches into launches[id] (both host
  * arrays of QASG_KERNEL_COUNT entries), then stops recording. */
-#define QASG_KERNEL_COUNT 12
+#define QASG_KERNEL_COUNT 16
 qasg_status qasg_profile_begin(qasg_ctx* ctx);
 qasg_status qasg_profile_end(qasg_ctx* ctx, double* ms, uint64_t* launches);
 const char* qasg_kernel_name(int id);

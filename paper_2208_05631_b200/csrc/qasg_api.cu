@@ -14,7 +14,9 @@ struct qasg_ctx {
   uint32_t M_max;
   LaunchShape shape;
   Workspace ws;
+  Workspace wsq;            // server row (the re-quantized average): kRowChunks partial slots, 1 statistic
   uint32_t* code_scratch;   // [M_max][code_words(d_max)] or NULL
+  uint32_t* qcode_scratch;  // [code_words(d_max)] or NULL
   float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
   uint64_t launches;
   bool profiling;
@@ -26,7 +28,8 @@ namespace {
 
 enum KernelId {
   kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
-  kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kKernelIdCount
+  kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kAvgAbsSum, kAvgAbsMax,
+  kAvgThresholdCodes, kAvgStochasticCodes, kKernelIdCount
 };
 static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
 
@@ -113,6 +116,24 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
   }
 }
 
+// Server row on validated arguments: q = Q(average of the decoded workers).
+void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M, uint64_t t,
+                const qasg_params* p, uint32_t* qcodes, float* qscale, float* qthreshold, uint64_t* qcount,
+                cudaStream_t stream) {
+  const Geometry row = make_geometry(d, d, 1, kRowChunks);
+  const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
+  {
+    Launch l(ctx, stochastic ? kAvgAbsMax : kAvgAbsSum, stream);
+    l += launch_avg_stats(stochastic, codes, scales, M, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream);
+  }
+  {
+    Launch l(ctx, stochastic ? kAvgStochasticCodes : kAvgThresholdCodes, stream);
+    l += launch_avg_codes(stochastic, codes, scales, M, row, p->seed, t, ctx->wsq, qcodes, qscale,
+                          reinterpret_cast<unsigned long long*>(qcount), ctx->shape, stream);
+  }
+  if (stochastic && qthreshold) cudaMemsetAsync(qthreshold, 0, sizeof(float), stream);
+}
+
 qasg_status check_gradient(const float* g, uint64_t d, uint64_t ld_g) {
   if (!g) return QASG_ERR_INVALID_ARG;
   if (ld_g < d) return QASG_ERR_INVALID_ARG;
@@ -149,13 +170,25 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ok &= cudaMalloc(&ctx->ws.ticket, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->ws.status, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->logreg_ws, kLogregEntries * 2 * sizeof(float)) == cudaSuccess;
-  if (ok && !(flags & QASG_CREATE_NO_CODE_SCRATCH))
+  ok &= cudaMalloc(&ctx->wsq.part_sum, kRowChunks * sizeof(double)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wsq.part_max, kRowChunks * sizeof(uint32_t)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wsq.part_cnt, kRowChunks * sizeof(unsigned long long)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wsq.thresholds, 64) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wsq.scales, 64) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wsq.counts, 64) == cudaSuccess;
+  ctx->wsq.ticket = ctx->ws.ticket;
+  ctx->wsq.status = ctx->ws.status;
+  if (ok && !(flags & QASG_CREATE_NO_CODE_SCRATCH)) {
     ok &= cudaMalloc(&ctx->code_scratch, static_cast<size_t>(M_max) * qasg_code_words(d_max) * 4) == cudaSuccess;
+    ok &= cudaMalloc(&ctx->qcode_scratch, qasg_code_words(d_max) * 4) == cudaSuccess;
+  }
   if (ok) {
     ok &= cudaMemset(ctx->ws.ticket, 0, 64) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.status, 0, 64) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.thresholds, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.scales, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
+    ok &= cudaMemset(ctx->wsq.thresholds, 0, 64) == cudaSuccess;
+    ok &= cudaMemset(ctx->wsq.scales, 0, 64) == cudaSuccess;
   }
   if (!ok) {
     cudaGetLastError();
@@ -179,6 +212,13 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->ws.status);
   cudaFree(ctx->logreg_ws);
   cudaFree(ctx->code_scratch);
+  cudaFree(ctx->qcode_scratch);
+  cudaFree(ctx->wsq.part_sum);
+  cudaFree(ctx->wsq.part_max);
+  cudaFree(ctx->wsq.part_cnt);
+  cudaFree(ctx->wsq.thresholds);
+  cudaFree(ctx->wsq.scales);
+  cudaFree(ctx->wsq.counts);
   for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   delete ctx;
   return QASG_OK;
@@ -257,6 +297,49 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
   { Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s); l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
                                         ctx->ws.status, ctx->shape, s); }
+  return leave();
+}
+
+qasg_status qasg_requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
+                            uint64_t t, const qasg_params* params, uint32_t* qcodes, float* qscale,
+                            float* qthreshold, uint64_t* qcount, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, false);
+  if (st != QASG_OK) return st;
+  if (!codes || !scales || !qcodes || !qscale || t < 1) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(codes) || !aligned16(qcodes)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  requantize(ctx, codes, scales, d, M, t, params, qcodes, qscale, qthreshold, qcount,
+             static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
+                             uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h, float* z,
+                             uint32_t* codes_out, float* scales_out, uint32_t* qcodes_out, float* qscale_out,
+                             void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
+  if (!x || !h || t < 1 || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(h) || (z && !aligned16(z)) || (codes_out && !aligned16(codes_out)) ||
+      (qcodes_out && !aligned16(qcodes_out)))
+    return QASG_ERR_ALIGNMENT;
+  uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
+  uint32_t* qcodes = qcodes_out ? qcodes_out : ctx->qcode_scratch;
+  if (!codes || !qcodes) return QASG_ERR_WORKSPACE;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
+  requantize(ctx, codes, ctx->ws.scales, d, M, t, params, qcodes, qscale_out, nullptr, nullptr, s);
+  {
+    // the workers decode q_t (one code row, one scale) and update
+    Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s);
+    l += launch_decode_update(rule, qcodes, ctx->wsq.scales, d, 1, x, h, z, scalars(params, t), ctx->ws.status,
+                              ctx->shape, s);
+  }
   return leave();
 }
 
@@ -386,7 +469,8 @@ qasg_status qasg_profile_end(qasg_ctx* ctx, double* ms, uint64_t* launches) {
 const char* qasg_kernel_name(int id) {
   static const char* const names[kKernelIdCount] = {
       "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
-      "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr"};
+      "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr", "avg_abs_sum",
+      "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes"};
   return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
 }
 

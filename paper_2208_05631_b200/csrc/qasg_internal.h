@@ -18,6 +18,8 @@ constexpr int kTile = kTileRows * kTileCols;
 // worker are combined by one warp.
 constexpr int kMaxChunks = 1024;
 constexpr int kMaxWorkers = 64;
+// The server row (the averaged gradient, re-quantized) is one long row: it may use more chunks.
+constexpr int kRowChunks = 8 * kMaxChunks;
 
 enum : unsigned { kFlagNonFinite = 1u, kFlagBadCode = 2u };
 
@@ -31,7 +33,7 @@ struct Geometry {
   uint32_t chunks;  // ceil(tiles / group) <= kMaxChunks
 };
 
-Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M);
+Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks = kMaxChunks);
 
 struct Workspace {
   double* part_sum;              // [M_max][kMaxChunks] chunk partials of a canonical sum
@@ -72,6 +74,15 @@ int launch_decode_update(int rule, const uint32_t* codes, const float* scales, u
 int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                           float* gbar, unsigned int* status, const LaunchShape& shape,
                           cudaStream_t stream);
+// Server row q = Q(average): statistics (threshold or maximum), then codes.  `row` is the geometry of
+// one row of d coordinates with up to kRowChunks chunks; wsq holds kRowChunks partial slots.
+int launch_avg_stats(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
+                     const Geometry& row, float coef, const Workspace& wsq, float* threshold_out,
+                     const LaunchShape& shape, cudaStream_t stream);
+int launch_avg_codes(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
+                     const Geometry& row, uint64_t seed, uint64_t t, const Workspace& wsq, uint32_t* qcodes,
+                     float* scale_out, unsigned long long* count_out, const LaunchShape& shape,
+                     cudaStream_t stream);
 int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h, float* z,
                         const StepScalars& sc, const LaunchShape& shape, cudaStream_t stream);
 

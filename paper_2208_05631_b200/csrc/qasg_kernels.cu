@@ -18,14 +18,14 @@
 namespace qasg {
 
 // ------------------------------------------------------------------ geometry
-Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M) {
+Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks) {
   Geometry geo;
   geo.d = d;
   geo.ld = ld;
   geo.M = M;
   geo.tiles = static_cast<uint32_t>((d + kTile - 1) / kTile);
   uint32_t group = 1, lg = 0;
-  while ((geo.tiles + group - 1) / group > static_cast<uint32_t>(kMaxChunks)) {
+  while ((geo.tiles + group - 1) / group > max_chunks) {
     group <<= 1;
     ++lg;
   }
@@ -758,6 +758,237 @@ dense_update_kernel(const float* __restrict__ q, uint64_t d, float* __restrict__
   }
 }
 
+// ------------------------------------------------------------------ server row: q = Q(average)
+// Double quantization (Algorithm 1, "Quantize the aggregated gradient"): the averaged gradient is
+// quantized again with the same Q.  The average is never stored: these kernels rebuild it from the
+// workers' code bytes, tile by tile, in the same 4 x 1024 tile geometry as a worker's gradient, so
+// its threshold and scale come from the same fixed-order sums.  The row is cut into up to
+// kRowChunks chunks; the last CTA combines their partials with a pairwise tree over 8 blocks of
+// 1024 slots, which is the pairwise tree over all slots.
+
+// The thread's four float4 of tile k of the averaged gradient; coordinates >= d are +0.0.
+__device__ __forceinline__ void decode_tile(const uint8_t* __restrict__ codes8, uint64_t row_bytes,
+                                            const double* lut, uint32_t workers, double inv_m, uint64_t d,
+                                            uint32_t k, int j, float4 (&v)[kTileRows], uint32_t& bad) {
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) {
+    const uint64_t grp = static_cast<uint64_t>(k) * (kTile / 4) + r * (kTileCols / 4) + j;
+    const uint64_t i0 = 4 * grp;
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 < d) {
+      t = decode_group<0, 1>(codes8, row_bytes, lut, workers, inv_m, grp, bad);
+      if (i0 + 1 >= d) t.y = 0.f;
+      if (i0 + 2 >= d) t.z = 0.f;
+      if (i0 + 3 >= d) t.w = 0.f;
+    }
+    v[r] = t;
+  }
+}
+
+// Pairwise tree over up to kRowChunks = 8 * 1024 partial slots; all threads call, result in thread 0.
+__device__ __forceinline__ double block_chunk_tree(const double* part, uint32_t chunks, double* sm8) {
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t base = warp * kMaxChunks;
+  const double v = warp_chunk_tree(part + base, chunks > base ? chunks - base : 0u, lane);
+  __syncthreads();
+  if (lane == 0) sm8[warp] = v;
+  __syncthreads();
+  double r = 0.0;
+  if (threadIdx.x == 0) r = ((sm8[0] + sm8[1]) + (sm8[2] + sm8[3])) + ((sm8[4] + sm8[5]) + (sm8[6] + sm8[7]));
+  return r;
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+avg_abs_sum_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint32_t workers,
+                   double inv_m, Geometry geo, float coef, Workspace ws, float* __restrict__ threshold_out) {
+  extern __shared__ double sm_lut[];
+  __shared__ ChunkSumStorage sm_sum;
+  __shared__ double sm8[kThreads / 32];
+  __shared__ bool sm_last;
+  build_decode_lut<1>(sm_lut, scales, workers);
+  const int j = threadIdx.x;
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  const uint64_t row_bytes = ((geo.d + 15) >> 4) * 4;
+  ChunkSum chunk_sum(&sm_sum);
+  uint32_t bad = 0;
+  for (uint32_t c = blockIdx.x; c < geo.chunks; c += gridDim.x) {
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    for (uint32_t k = k0; k < k1; ++k) {
+      float4 v[kTileRows];
+      decode_tile(codes8, row_bytes, sm_lut, workers, inv_m, geo.d, k, j, v, bad);
+      double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
+#pragma unroll
+      for (int r = 1; r < kTileRows; ++r) {
+        cx += static_cast<double>(fabsf(v[r].x));
+        cy += static_cast<double>(fabsf(v[r].y));
+        cz += static_cast<double>(fabsf(v[r].z));
+        cw += static_cast<double>(fabsf(v[r].w));
+      }
+      chunk_sum.add_tile((cx + cy) + (cz + cw));
+    }
+    const double total = chunk_sum.finish(geo.log2_group);
+    if (j == 0) ws.part_sum[c] = total;
+  }
+  if (bad) atomicOr(ws.status, kFlagBadCode);
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  const double total = block_chunk_tree(ws.part_sum, geo.chunks, sm8);
+  if (j == 0) {
+    const float delta = static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(geo.d));
+    ws.thresholds[0] = delta;
+    if (threshold_out) threshold_out[0] = delta;
+    *ws.ticket = 0u;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+avg_abs_max_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint32_t workers,
+                   double inv_m, Geometry geo, Workspace ws) {
+  extern __shared__ double sm_lut[];
+  __shared__ uint32_t sm_warp[kThreads / 32];
+  __shared__ bool sm_last;
+  build_decode_lut<1>(sm_lut, scales, workers);
+  const int j = threadIdx.x;
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  const uint64_t row_bytes = ((geo.d + 15) >> 4) * 4;
+  uint32_t bad = 0, best = 0u;
+  for (uint32_t c = blockIdx.x; c < geo.chunks; c += gridDim.x) {
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    for (uint32_t k = k0; k < k1; ++k) {
+      float4 v[kTileRows];
+      decode_tile(codes8, row_bytes, sm_lut, workers, inv_m, geo.d, k, j, v, bad);
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) {
+        best = max(best, __float_as_uint(fabsf(v[r].x)));
+        best = max(best, __float_as_uint(fabsf(v[r].y)));
+        best = max(best, __float_as_uint(fabsf(v[r].z)));
+        best = max(best, __float_as_uint(fabsf(v[r].w)));
+      }
+    }
+  }
+  // the maximum is order-free: one partial per CTA
+  best = __reduce_max_sync(0xffffffffu, best);
+  if ((j & 31) == 0) sm_warp[j >> 5] = best;
+  __syncthreads();
+  if (j == 0) {
+    uint32_t bmax = sm_warp[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) bmax = max(bmax, sm_warp[w]);
+    ws.part_max[blockIdx.x] = bmax;
+  }
+  if (bad) atomicOr(ws.status, kFlagBadCode);
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  uint32_t bmax = 0u;
+  for (uint32_t idx = j; idx < gridDim.x; idx += kThreads) bmax = max(bmax, __ldcg(ws.part_max + idx));
+  bmax = __reduce_max_sync(0xffffffffu, bmax);
+  __syncthreads();
+  if ((j & 31) == 0) sm_warp[j >> 5] = bmax;
+  __syncthreads();
+  if (j == 0) {
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) bmax = max(bmax, sm_warp[w]);
+    ws.scales[0] = __uint_as_float(bmax);
+    ws.thresholds[0] = 0.f;
+    *ws.ticket = 0u;
+  }
+}
+
+// kStochastic = false: Q_Delta with ws.thresholds[0]; true: unbiased ternary with ws.scales[0] and the
+// Philox stream of domain 1 (worker field 0).
+template <bool kStochastic>
+__global__ void __launch_bounds__(kThreads, 4)
+avg_codes_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint32_t workers,
+                 double inv_m, Geometry geo, uint64_t seed, uint64_t t, Workspace ws,
+                 uint32_t* __restrict__ qcodes, float* __restrict__ scale_out,
+                 unsigned long long* __restrict__ count_out) {
+  extern __shared__ double sm_lut[];
+  __shared__ ChunkSumStorage sm_sum;
+  __shared__ double sm8[kThreads / 32];
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ bool sm_last;
+  build_decode_lut<1>(sm_lut, scales, workers);
+  const int j = threadIdx.x;
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  uint8_t* qcodes8 = reinterpret_cast<uint8_t*>(qcodes);
+  const uint64_t row_bytes = ((geo.d + 15) >> 4) * 4;
+  const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
+  const float delta = ws.thresholds[0], ndelta = -delta, smax = ws.scales[0];
+  const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
+  const uint32_t t_lo = static_cast<uint32_t>(t), t_hi = static_cast<uint32_t>(t >> 32);
+  ChunkSum chunk_sum(&sm_sum);
+  uint32_t bad = 0;
+  for (uint32_t c = blockIdx.x; c < geo.chunks; c += gridDim.x) {
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    float cntf = 0.f;
+    for (uint32_t k = k0; k < k1; ++k) {
+      float4 v[kTileRows];
+      decode_tile(codes8, row_bytes, sm_lut, workers, inv_m, geo.d, k, j, v, bad);
+      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+      uint32_t bytes[kTileRows];
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) {
+        const float4 q = v[r];
+        float px, nx, py, ny, pz, nz, pw, nw;
+        if (!kStochastic) {
+          px = q.x > delta ? 1.f : 0.f, nx = q.x < ndelta ? 1.f : 0.f;
+          py = q.y > delta ? 1.f : 0.f, ny = q.y < ndelta ? 1.f : 0.f;
+          pz = q.z > delta ? 1.f : 0.f, nz = q.z < ndelta ? 1.f : 0.f;
+          pw = q.w > delta ? 1.f : 0.f, nw = q.w < ndelta ? 1.f : 0.f;
+        } else {
+          const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
+          const uint4 w = philox4x32_10(make_uint4(blk, 1u << 16, t_lo, t_hi), key0, key1);
+          const CodeBits bx = split_code(q.x, philox_uniform(w.x) < __fdiv_rn(fabsf(q.x), smax));
+          const CodeBits by = split_code(q.y, philox_uniform(w.y) < __fdiv_rn(fabsf(q.y), smax));
+          const CodeBits bz = split_code(q.z, philox_uniform(w.z) < __fdiv_rn(fabsf(q.z), smax));
+          const CodeBits bw = split_code(q.w, philox_uniform(w.w) < __fdiv_rn(fabsf(q.w), smax));
+          px = bx.pos, nx = bx.neg, py = by.pos, ny = by.neg, pz = bz.pos, nz = bz.neg, pw = bw.pos, nw = bw.neg;
+        }
+        const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;
+        if (!kStochastic) {
+          cx += static_cast<double>(fabsf(q.x) * kx);
+          cy += static_cast<double>(fabsf(q.y) * ky);
+          cz += static_cast<double>(fabsf(q.z) * kz);
+          cw += static_cast<double>(fabsf(q.w) * kw);
+        }
+        cntf += (kx + ky) + (kz + kw);
+        bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
+      }
+      store_code_bytes(qcodes8, k, j, k < full_tiles, row_bytes, bytes);
+      if (!kStochastic) chunk_sum.add_tile((cx + cy) + (cz + cw));
+    }
+    double picked = 0.0;
+    if (!kStochastic) picked = chunk_sum.finish(geo.log2_group);
+    const unsigned long long total = block_count(static_cast<uint32_t>(cntf), sm_cnt);
+    if (j == 0) {
+      ws.part_sum[c] = picked;
+      ws.part_cnt[c] = total;
+    }
+  }
+  if (bad) atomicOr(ws.status, kFlagBadCode);
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  unsigned long long n = 0;
+  for (uint32_t idx = j; idx < geo.chunks; idx += kThreads) n += __ldcg(ws.part_cnt + idx);
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
+  __shared__ unsigned long long sm_n[kThreads / 32];
+  if ((j & 31) == 0) sm_n[j >> 5] = n;
+  const double picked = kStochastic ? 0.0 : block_chunk_tree(ws.part_sum, geo.chunks, sm8);
+  __syncthreads();
+  if (j == 0) {
+    n = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) n += sm_n[w];
+    const float scale = kStochastic ? smax : (n ? static_cast<float>(picked / static_cast<double>(n)) : 0.f);
+    ws.scales[0] = scale;
+    ws.counts[0] = n;
+    if (scale_out) scale_out[0] = scale;
+    if (count_out) count_out[0] = n;
+    *ws.ticket = 0u;
+  }
+}
+
 // ------------------------------------------------------------------ launchers
 void query_launch_shape(LaunchShape* shape) {
   int dev = 0;
@@ -883,6 +1114,40 @@ int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h
     dense_update_kernel<0><<<grid, kThreads, 0, stream>>>(q, d, x, h, z, sc);
   else
     dense_update_kernel<1><<<grid, kThreads, 0, stream>>>(q, d, x, h, z, sc);
+  return 1;
+}
+
+
+static unsigned row_grid(const Geometry& geo, const LaunchShape& shape) {
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * shape.reduce_ctas_per_sm;
+  return static_cast<unsigned>(geo.chunks < resident ? geo.chunks : resident);
+}
+
+int launch_avg_stats(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
+                     const Geometry& row, float coef, const Workspace& wsq, float* threshold_out,
+                     const LaunchShape& shape, cudaStream_t stream) {
+  const size_t lut_bytes = static_cast<size_t>((workers + 3) / 4) * 256 * sizeof(double);
+  const double inv_m = 1.0 / static_cast<double>(workers);
+  if (stochastic)
+    avg_abs_max_kernel<<<row_grid(row, shape), kThreads, lut_bytes, stream>>>(codes, scales, workers, inv_m, row, wsq);
+  else
+    avg_abs_sum_kernel<<<row_grid(row, shape), kThreads, lut_bytes, stream>>>(codes, scales, workers, inv_m, row,
+                                                                             coef, wsq, threshold_out);
+  return 1;
+}
+
+int launch_avg_codes(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
+                     const Geometry& row, uint64_t seed, uint64_t t, const Workspace& wsq, uint32_t* qcodes,
+                     float* scale_out, unsigned long long* count_out, const LaunchShape& shape,
+                     cudaStream_t stream) {
+  const size_t lut_bytes = static_cast<size_t>((workers + 3) / 4) * 256 * sizeof(double);
+  const double inv_m = 1.0 / static_cast<double>(workers);
+  if (stochastic)
+    avg_codes_kernel<true><<<row_grid(row, shape), kThreads, lut_bytes, stream>>>(
+        codes, scales, workers, inv_m, row, seed, t, wsq, qcodes, scale_out, count_out);
+  else
+    avg_codes_kernel<false><<<row_grid(row, shape), kThreads, lut_bytes, stream>>>(
+        codes, scales, workers, inv_m, row, seed, t, wsq, qcodes, scale_out, count_out);
   return 1;
 }
 

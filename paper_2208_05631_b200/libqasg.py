@@ -25,10 +25,10 @@ EXPORTS = [
     "qasg_create", "qasg_destroy", "qasg_code_words", "qasg_quantize_pack", "qasg_decode_average",
     "qasg_cmd_step", "qasg_rda_step", "qasg_step", "qasg_step_host", "qasg_logreg_grad_dense",
     "qasg_logreg_grad_csr", "qasg_last_async_status", "qasg_launch_count", "qasg_status_string",
-    "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static",
+    "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static", "qasg_requantize", "qasg_step_double",
 ]
 STATIC_MAX_WORKERS = 16
-KERNEL_COUNT = 12
+KERNEL_COUNT = 16
 
 
 class QasgError(RuntimeError):
@@ -70,6 +70,8 @@ def load():
     lib.qasg_cmd_step.argtypes = [vp, vp, vp, vp, u64, u64, pp, vp]
     lib.qasg_rda_step.argtypes = [vp, vp, vp, vp, vp, u64, u64, pp, vp]
     lib.qasg_step.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp]
+    lib.qasg_requantize.argtypes = [vp, vp, vp, u64, u32, u64, pp, vp, vp, vp, vp, vp]
+    lib.qasg_step_double.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.qasg_step_host.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.qasg_logreg_grad_dense.argtypes = [vp, vp, vp, u64, u64, u32, ctypes.POINTER(u64), vp, u32, u64,
                                            vp, vp, u64, vp]
@@ -159,6 +161,18 @@ class Context:
              stream=None):
         _check(load().qasg_step(self._h, rule, _ptr(g), d, ld_g, M, t, ctypes.byref(params), _ptr(x), _ptr(h),
                                 _ptr(z), _ptr(codes_out), _ptr(scales_out), _stream(stream)), "qasg_step")
+
+    def requantize(self, codes, scales, d, M, t, params, qcodes, qscale, qthreshold=None, qcount=None,
+                   stream=None):
+        _check(load().qasg_requantize(self._h, _ptr(codes), _ptr(scales), d, M, t, ctypes.byref(params),
+                                      _ptr(qcodes), _ptr(qscale), _ptr(qthreshold), _ptr(qcount),
+                                      _stream(stream)), "qasg_requantize")
+
+    def step_double(self, rule, g, d, ld_g, M, t, params, x, h, z=None, codes_out=None, scales_out=None,
+                    qcodes_out=None, qscale_out=None, stream=None):
+        _check(load().qasg_step_double(self._h, rule, _ptr(g), d, ld_g, M, t, ctypes.byref(params), _ptr(x),
+                                       _ptr(h), _ptr(z), _ptr(codes_out), _ptr(scales_out), _ptr(qcodes_out),
+                                       _ptr(qscale_out), _stream(stream)), "qasg_step_double")
 
     def step_host(self, rule, g_host, d, ld_g, M, t, params, x_host, h_host, z_host, g_dev, x_dev, h_dev,
                   z_dev, stream=None):
