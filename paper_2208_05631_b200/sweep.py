@@ -1,6 +1,7 @@
 """Timing sweeps of libqasg on one GPU, beyond the single workload bench.py reports.
 
-  python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--max-log2-d 28]
+  python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--double-quant]
+                                               [--min-log2-d 20] [--max-log2-d 28] [--workers 2,4,8,16,32]
   python -m paper_2208_05631_b200.sweep logreg [--steps 50]
 
 `step`   - the fused step over d in {2^20 .. 2^28} x M in {2, 4, 8, 16, 32} simulated workers,
@@ -47,23 +48,34 @@ def sweep_step(args):
     flush = torch.zeros(64 << 20, dtype=torch.float32, device=dev)      # 256 MB > L2
     quantizer = libqasg.Q_THRESHOLD if args.quantizer == "threshold" else libqasg.Q_TERNARY_STOCH
     params = libqasg.make_params(LAM, ETA, DELTA, quantizer=quantizer, seed=4)
-    for log2d in range(20, args.max_log2_d + 1, 2):
+    for log2d in range(args.min_log2_d, args.max_log2_d + 1, 2):
         d = 1 << log2d
-        for M in (2, 4, 8, 16, 32):
+        for M in [int(v) for v in args.workers.split(",")]:
             g = inputs.normal_gradients(d, M, seed=4, device=dev)
             x, h, z = inputs.random_state(d, seed=4, device=dev)
             ctx = libqasg.Context(d, M, device=0)
             for rule, name, state_bytes in ((libqasg.RULE_CMD, "qcmd", 16), (libqasg.RULE_RDA, "qrda", 20)):
                 def one():
-                    ctx.step(rule, g, d, d, M, T_STEP, params, x, h, z)
+                    if args.double_quant:
+                        ctx.step_double(rule, g, d, d, M, T_STEP, params, x, h, z)
+                    else:
+                        ctx.step(rule, g, d, d, M, T_STEP, params, x, h, z)
                 for _ in range(3):
                     one()
                 torch.cuda.synchronize()
                 med, best = _time_calls(one, args.reps, flush)
+                ctx.profile_begin()
+                one()
+                kernel_ms = {k: v[0] / v[1] for k, v in ctx.profile_end().items()}
+                # bytes the method must move: g twice, worker codes written and read once, state once;
+                # double quantization reads the worker codes three times and writes/reads the server's codes
                 moved = d * (8.0 * M + M / 2.0 + state_bytes)
-                print(json.dumps({"what": "step", "quantizer": args.quantizer, "rule": name, "d": d, "M": M,
-                                  "ms_median": med, "ms_best": best, "coord_workers_per_s": d * M / (med * 1e-3),
-                                  "gbs_moved": moved / 1e9 / (med * 1e-3)}), flush=True)
+                if args.double_quant:
+                    moved = d * (8.0 * M + M / 4.0 + 2.0 * M / 4.0 + 2 * 0.25 + state_bytes)
+                print(json.dumps({"what": "step_double" if args.double_quant else "step", "quantizer": args.quantizer,
+                                  "rule": name, "d": d, "M": M, "ms_median": med, "ms_best": best,
+                                  "coord_workers_per_s": d * M / (med * 1e-3),
+                                  "gbs_moved": moved / 1e9 / (med * 1e-3), "kernel_ms": kernel_ms}), flush=True)
             assert ctx.last_async_status() == libqasg.OK
             ctx.close()
             del g, x, h, z
@@ -132,7 +144,10 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("what", choices=["step", "logreg"])
     ap.add_argument("--quantizer", default="threshold", choices=["threshold", "stochastic"])
+    ap.add_argument("--double-quant", action="store_true")
+    ap.add_argument("--min-log2-d", type=int, default=20)
     ap.add_argument("--max-log2-d", type=int, default=28)
+    ap.add_argument("--workers", default="2,4,8,16,32")
     ap.add_argument("--reps", type=int, default=7)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--csr-rows", type=int, default=1_000_000)
