@@ -78,8 +78,9 @@ typedef struct {
 
 /* Creates a context on CUDA device `device` able to serve calls with d <= d_max and
  * M <= M_max.  Allocates the whole workspace here (a few hundred KB of statistics, and,
- * unless QASG_CREATE_NO_CODE_SCRATCH, M_max * qasg_code_words(d_max) * 4 bytes of code
- * scratch); no other call allocates device memory.  On error *out is NULL. */
+ * unless QASG_CREATE_NO_CODE_SCRATCH, (M_max + 1) * qasg_code_words(d_max) * 4 bytes of code
+ * scratch and 4 * d_max bytes for the averaged gradient of the double-quantized step); no
+ * other call allocates device memory.  On error *out is NULL. */
 qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_max,
                         uint32_t flags);
 /* Frees the workspace.  The caller must have synchronized the streams it used. */

@@ -17,6 +17,7 @@ struct qasg_ctx {
   Workspace wsq;            // server row (the re-quantized average): kRowChunks partial slots, 1 statistic
   uint32_t* code_scratch;   // [M_max][code_words(d_max)] or NULL
   uint32_t* qcode_scratch;  // [code_words(d_max)] or NULL
+  float* gbar_scratch;      // [d_max rounded up to 4] or NULL: the averaged gradient of the server row
   float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
   uint64_t launches;
   bool profiling;
@@ -110,26 +111,47 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
     { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream); }
   } else {
     { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream); }
-    { Launch l(ctx, kStochasticCodes, stream); l += launch_stochastic_codes(g, geo, p->seed, t, ctx->ws, codes, scales, counts_out,
+    { Launch l(ctx, kStochasticCodes, stream); l += launch_stochastic_codes(g, geo, p->seed, t, 0u, ctx->ws, codes, scales, counts_out,
                                              ctx->shape, stream); }
     if (thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
   }
 }
 
 // Server row on validated arguments: q = Q(average of the decoded workers).
+// With scratch, the average is written once as an fp32 row (fast per-lane-table decode) and the
+// workers' own two quantization kernels run on that row; without, two kernels rebuild the average
+// from the code bytes and nothing is stored.  Both give the same bits.
 void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M, uint64_t t,
                 const qasg_params* p, uint32_t* qcodes, float* qscale, float* qthreshold, uint64_t* qcount,
                 cudaStream_t stream) {
-  const Geometry row = make_geometry(d, d, 1, kRowChunks);
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
-  {
-    Launch l(ctx, stochastic ? kAvgAbsMax : kAvgAbsSum, stream);
-    l += launch_avg_stats(stochastic, codes, scales, M, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream);
-  }
-  {
-    Launch l(ctx, stochastic ? kAvgStochasticCodes : kAvgThresholdCodes, stream);
-    l += launch_avg_codes(stochastic, codes, scales, M, row, p->seed, t, ctx->wsq, qcodes, qscale,
-                          reinterpret_cast<unsigned long long*>(qcount), ctx->shape, stream);
+  unsigned long long* count_out = reinterpret_cast<unsigned long long*>(qcount);
+  if (ctx->gbar_scratch) {
+    float* gbar = ctx->gbar_scratch;
+    const uint64_t ld = ((d + 3) / 4) * 4;
+    {
+      Launch l(ctx, kDecodeAverage, stream);
+      l += launch_decode_average(codes, scales, d, M, gbar, ctx->ws.status, ctx->shape, stream);
+    }
+    const Geometry row = make_geometry(d, ld, 1);
+    if (!stochastic) {
+      { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(gbar, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream); }
+      { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(gbar, row, ctx->wsq, qcodes, qscale, count_out, ctx->shape, stream); }
+    } else {
+      { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(gbar, row, ctx->wsq, ctx->shape, stream); }
+      { Launch l(ctx, kStochasticCodes, stream); l += launch_stochastic_codes(gbar, row, p->seed, t, 1u << 16, ctx->wsq, qcodes, qscale, count_out, ctx->shape, stream); }
+    }
+  } else {
+    const Geometry row = make_geometry(d, d, 1, kRowChunks);
+    {
+      Launch l(ctx, stochastic ? kAvgAbsMax : kAvgAbsSum, stream);
+      l += launch_avg_stats(stochastic, codes, scales, M, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream);
+    }
+    {
+      Launch l(ctx, stochastic ? kAvgStochasticCodes : kAvgThresholdCodes, stream);
+      l += launch_avg_codes(stochastic, codes, scales, M, row, p->seed, t, ctx->wsq, qcodes, qscale, count_out,
+                            ctx->shape, stream);
+    }
   }
   if (stochastic && qthreshold) cudaMemsetAsync(qthreshold, 0, sizeof(float), stream);
 }
@@ -181,6 +203,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   if (ok && !(flags & QASG_CREATE_NO_CODE_SCRATCH)) {
     ok &= cudaMalloc(&ctx->code_scratch, static_cast<size_t>(M_max) * qasg_code_words(d_max) * 4) == cudaSuccess;
     ok &= cudaMalloc(&ctx->qcode_scratch, qasg_code_words(d_max) * 4) == cudaSuccess;
+    ok &= cudaMalloc(&ctx->gbar_scratch, ((d_max + 3) / 4) * 4 * sizeof(float)) == cudaSuccess;
   }
   if (ok) {
     ok &= cudaMemset(ctx->ws.ticket, 0, 64) == cudaSuccess;
@@ -213,6 +236,7 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->logreg_ws);
   cudaFree(ctx->code_scratch);
   cudaFree(ctx->qcode_scratch);
+  cudaFree(ctx->gbar_scratch);
   cudaFree(ctx->wsq.part_sum);
   cudaFree(ctx->wsq.part_max);
   cudaFree(ctx->wsq.part_cnt);

@@ -64,10 +64,12 @@ int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
                            const LaunchShape& shape, cudaStream_t stream);
+// stream_base is added to the worker index in Philox counter word 1 (0 for workers, 1<<16 for the server row).
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
-                            const Workspace& ws, uint32_t* codes, float* scales_out,
+                            uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
                             cudaStream_t stream);
+// rule 0 = QCMD, 1 = QRDA, 2 = write the averaged gradient to x (h, z unused).
 int launch_decode_update(int rule, const uint32_t* codes, const float* scales, uint64_t d,
                          uint32_t M, float* x, float* h, float* z, const StepScalars& sc,
                          unsigned int* status, const LaunchShape& shape, cudaStream_t stream);

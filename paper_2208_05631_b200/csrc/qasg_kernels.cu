@@ -452,7 +452,7 @@ __device__ __forceinline__ float philox_uniform(uint32_t word) {
 // ------------------------------------------------------------------ pass B': stochastic codes
 __global__ void __launch_bounds__(kThreads)
 stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
-                        Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
+                        uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
                         unsigned long long* __restrict__ counts_out) {
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
@@ -477,7 +477,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
         const float4 v = tile[r];
         // coordinates 4*blk .. 4*blk+3 share one Philox block
         const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
-        const uint4 w = philox4x32_10(make_uint4(blk, m, t_lo, t_hi), key0, key1);
+        const uint4 w = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), key0, key1);
         // |v|/s with IEEE division; s = 0 gives NaN and the comparison is false.
         const bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
         const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
@@ -604,16 +604,22 @@ __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes
 
 // ------------------------------------------------------------------ pass C: fused
 // State of one group of four coordinates.
+// kRule: 0 = QCMD, 1 = QRDA, 2 = no update at all: the averaged gradient is written to x.
 template <int kRule>
 struct GroupState {
   float4 h, xz;  // xz: x for QCMD (read and written), z for QRDA
   __device__ __forceinline__ void load(const float* __restrict__ x, const float* __restrict__ hh,
                                        const float* __restrict__ z, uint64_t grp) {
+    if (kRule == 2) return;
     h = *reinterpret_cast<const float4*>(hh + 4 * grp);
     xz = *reinterpret_cast<const float4*>((kRule == 0 ? x : z) + 4 * grp);
   }
   __device__ __forceinline__ void update_store(float4 q, float* __restrict__ x, float* __restrict__ hh,
                                                float* __restrict__ z, uint64_t grp, const StepScalars& sc) {
+    if (kRule == 2) {
+      *reinterpret_cast<float4*>(x + 4 * grp) = q;
+      return;
+    }
     if (kRule == 0) {
       cmd_update(q.x, xz.x, h.x, sc);
       cmd_update(q.y, xz.y, h.y, sc);
@@ -674,6 +680,10 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
       } else {  // ragged tail: d % 4 coordinates
         const float qs[4] = {q.x, q.y, q.z, q.w};
         for (uint64_t c = 4 * grp; c < d; ++c) {
+          if (kRule == 2) {
+            x[c] = qs[c - 4 * grp];
+            continue;
+          }
           float xi = (kRule == 0) ? x[c] : 0.f, hi = h[c];
           if (kRule == 0) {
             cmd_update(qs[c - 4 * grp], xi, hi, sc);
@@ -691,29 +701,7 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
   if (bad) atomicOr(status, kFlagBadCode);
 }
 
-// ------------------------------------------------------------------ pass C, unfused halves
-__global__ void __launch_bounds__(kThreads)
-decode_average_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
-                      uint32_t M, double inv_m, float* __restrict__ gbar, unsigned int* __restrict__ status) {
-  extern __shared__ double sm_lut[];
-  build_decode_lut<1>(sm_lut, scales, M);
-  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
-  const uint64_t row_bytes = ((d + 15) >> 4) * 4;
-  const uint64_t groups = (d + 3) >> 2, full = d >> 2;
-  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
-  uint32_t bad = 0;
-  for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; grp < groups; grp += stride) {
-    const float4 q = decode_group<0, 1>(codes8, row_bytes, sm_lut, M, inv_m, grp, bad);
-    if (grp < full) {
-      *reinterpret_cast<float4*>(gbar + 4 * grp) = q;
-    } else {
-      const float qs[4] = {q.x, q.y, q.z, q.w};
-      for (uint64_t i = 4 * grp; i < d; ++i) gbar[i] = qs[i - 4 * grp];
-    }
-  }
-  if (bad) atomicOr(status, kFlagBadCode);
-}
-
+// ------------------------------------------------------------------ pass C, update from a dense q
 template <int kRule>
 __global__ void __launch_bounds__(kThreads)
 dense_update_kernel(const float* __restrict__ q, uint64_t d, float* __restrict__ x,
@@ -996,7 +984,7 @@ void query_launch_shape(LaunchShape* shape) {
   cudaDeviceGetAttribute(&shape->sm_count, cudaDevAttrMultiProcessorCount, dev);
   int a = 0, b = 0;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel, kThreads, 0);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_average_kernel, kThreads, 2 * 256 * sizeof(double));
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dense_update_kernel<1>, kThreads, 0);
   shape->reduce_ctas_per_sm = a > 0 ? a : 1;
   shape->update_ctas_per_sm = b > 0 ? b : 1;
 }
@@ -1035,10 +1023,10 @@ int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace&
 }
 
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
-                            const Workspace& ws, uint32_t* codes, float* scales_out,
+                            uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
                             cudaStream_t stream) {
-  stochastic_codes_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, seed, t, ws, codes,
+  stochastic_codes_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, seed, t, stream_base, ws, codes,
                                                                            scales_out, counts_out);
   return 1;
 }
@@ -1073,7 +1061,7 @@ template <int kRule>
 static void launch_decode_update_rule(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                                       float* x, float* h, float* z, const StepScalars& sc,
                                       unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
-  constexpr int kG = kRule == 0 ? 2 : 1;  // groups per thread with per-lane tables (measured best)
+  constexpr int kG = kRule == 1 ? 1 : 2;  // groups per thread with per-lane tables (measured best)
 #define QASG_LANE(m4) \
   case m4: launch_decode_update_as<kRule, m4, 32, 1024, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_SHARED(m4) \
@@ -1092,19 +1080,18 @@ int launch_decode_update(int rule, const uint32_t* codes, const float* scales, u
                          unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
   if (rule == 0)
     launch_decode_update_rule<0>(codes, scales, d, M, x, h, z, sc, status, shape, stream);
-  else
+  else if (rule == 1)
     launch_decode_update_rule<1>(codes, scales, d, M, x, h, z, sc, status, shape, stream);
+  else
+    launch_decode_update_rule<2>(codes, scales, d, M, x, h, z, sc, status, shape, stream);
   return 1;
 }
 
 int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                           float* gbar, unsigned int* status, const LaunchShape& shape,
                           cudaStream_t stream) {
-  const double inv_m = 1.0 / static_cast<double>(M);
-  const size_t lut_bytes = static_cast<size_t>((M + 3) / 4) * 256 * sizeof(double);
-  decode_average_kernel<<<update_grid(d, shape), kThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, gbar,
-                                                                               status);
-  return 1;
+  const StepScalars unused = {0.f, 0.f, 0.f, 0.f, 0.f};
+  return launch_decode_update(2, codes, scales, d, M, gbar, nullptr, nullptr, unused, status, shape, stream);
 }
 
 int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h, float* z,

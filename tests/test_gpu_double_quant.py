@@ -20,6 +20,14 @@ def ctx():
     c.close()
 
 
+@pytest.fixture(scope="module")
+def ctx_no_scratch():
+    # without scratch the server row is rebuilt from the code bytes twice instead of being stored once
+    c = libqasg.Context(6_000_000, 64, device=0, flags=libqasg.CREATE_NO_CODE_SCRATCH)
+    yield c
+    c.close()
+
+
 def _requantize_gpu(ctx, quant, d, M, quantizer, t, seed):
     codes = U.to_dev(quant["codes"].view(np.int32))
     scales = U.to_dev(quant["scales"])
@@ -35,7 +43,9 @@ def _requantize_gpu(ctx, quant, d, M, quantizer, t, seed):
 
 @pytest.mark.parametrize("d,M", [(1, 1), (17, 3), (4097, 8), (70_003, 5), (300_001, 16), (5_000_001, 2)])
 @pytest.mark.parametrize("quantizer", [libqasg.Q_THRESHOLD, libqasg.Q_TERNARY_STOCH])
-def test_requantize_bit_exact(ctx, d, M, quantizer):
+@pytest.mark.parametrize("stored", [True, False])
+def test_requantize_bit_exact(ctx, ctx_no_scratch, d, M, quantizer, stored):
+    ctx = ctx if stored else ctx_no_scratch
     t, seed = 9, 77
     g = inputs.normal_gradients(d, M, seed=d % 1000).numpy() * np.float32(0.05)
     quant = O.quantize_workers(g, quantizer, t=t, seed=seed)
