@@ -21,6 +21,12 @@ import numpy as np
 F32 = np.float32
 F64 = np.float64
 
+QUANT_THRESHOLD = 0
+QUANT_TERNARY_STOCH = 1
+QUANT_NONE = 2
+RULE_CMD = 0
+RULE_RDA = 1
+
 # Geometry of the canonical sum: a tile is TILE_ROWS rows of TILE_COLS consecutive
 # coordinates (row-major), i.e. 4096 consecutive coordinates.
 TILE_ROWS = 4
@@ -222,21 +228,25 @@ def decode_average(terns, scales):
     return acc * (F64(1.0) / F64(m_workers))
 
 
-def requantize(gbar, quantizer, t=1, seed=0, coef=0.75):
+def requantize(gbar, quantizer, t=1, seed=0, coef=0.75, isyn=None):
     """Server side of Algorithm 1, "Quantize the aggregated gradient": q_t = Q(SynQ_t).
 
     The averaged gradient is held in fp32 (it is what would be sent), so gbar (fp64) is rounded
     to fp32 first and Q is applied to that vector exactly as it is applied to a worker's
     gradient.  The stochastic quantizer draws from the Philox stream of domain 1, worker 0.
+    isyn (bool[d]) restricts Q to the coordinates of the synchronous indicator.
     Returns dict(tern int8[d], scale fp32, threshold fp32, count int, codes uint32[W], q fp64[d]).
     """
     gbar32 = np.asarray(gbar, dtype=F64).astype(F32)
     d = gbar32.size
     if quantizer == QUANT_THRESHOLD:
-        tern, scale, threshold, count = threshold_quantize(gbar32, coef)
+        if isyn is None:
+            tern, scale, threshold, count = threshold_quantize(gbar32, coef)
+        else:   # Q(S(SynQ_t, I^Syn)): only the coordinates some worker selected are quantized
+            tern, scale, threshold, count, _ = threshold_quantize_selected(gbar32, isyn, coef)
     elif quantizer == QUANT_TERNARY_STOCH:
         _, u = philox_draws(seed, t, 0, np.arange(d, dtype=np.uint64), domain=1)
-        tern, scale = ternary_stochastic_quantize(gbar32, u)
+        tern, scale = ternary_stochastic_quantize(gbar32, u)     # the average is 0 outside I^Syn
         threshold, count = F32(0.0), int(np.count_nonzero(tern))
     else:
         raise ValueError("quantizer")
@@ -294,13 +304,118 @@ def rda_step(q, h, z, t, lam, eta, delta):
 
 
 # ----------------------------------------------------------------------------------
+# Sparse selection (Section 3.2: indicator I, selection S, "bitwise or" of the indicators)
+# ----------------------------------------------------------------------------------
+def trial_update(rule, g_m, x, h, z, t, lam, eta, delta):
+    """Worker m's local trial iterate x_hat_{t+1}^(m) (Algorithm 1, "Compute the x_hat based on f'_t
+    and H_hat_t"): the rule's closed-form update taken with the worker's own full-precision gradient
+    and H_hat = delta + sqrt(h + g_m^2), h the accumulated squares of the quantized gradients so far.
+    fp64; state is not modified."""
+    if rule == RULE_CMD:
+        return cmd_step(g_m, x, h, lam, eta, delta)[0]
+    return rda_step(g_m, h, z, t, lam, eta, delta)[0]
+
+
+def indicator(rule, g_m, x, h, z, t, lam, eta, delta):
+    """I_d = 1 if x_{t,d} != 0 or x_hat_{t+1,d} != 0 (Eq. of the indicator function), decided in fp32
+    by a fixed sequence of correctly rounded operations, each one its own rounding (no fused
+    multiply-add), so that every implementation takes the same decision:
+
+      QCMD:  x_hat != 0  <=>  |x*H_hat - eta*g| > lambda*eta,   H_hat = delta + sqrt(h + g*g)
+             (the closed form's test |x - eta*g/H_hat| > lambda*eta/H_hat multiplied by H_hat > 0)
+      QRDA:  x_hat != 0  <=>  |z + g| > lambda*t
+
+    Returns a bool vector."""
+    f = F32
+    g_m = np.asarray(g_m, dtype=F32)
+    x = np.asarray(x, dtype=F32)
+    lam, eta, delta = f(lam), f(eta), f(delta)
+    if rule == RULE_CMD:
+        h = np.asarray(h, dtype=F32)
+        big_h = delta + np.sqrt(h + g_m * g_m)
+        lhs = np.abs(x * big_h - eta * g_m)
+        moved = lhs > lam * eta
+    else:
+        z = np.asarray(z, dtype=F32)
+        moved = np.abs(z + g_m) > lam * f(int(t))
+    return (x != 0) | moved
+
+
+def pack_bits(mask):
+    """Bool vector -> uint32 words, bit i&31 of word i>>5, tail bits 0."""
+    mask = np.asarray(mask, dtype=bool).ravel()
+    w = -(-mask.size // 32)
+    buf = np.zeros(w * 32, dtype=np.uint32)
+    buf[: mask.size] = mask
+    return np.bitwise_or.reduce(buf.reshape(w, 32) << np.arange(32, dtype=np.uint32), axis=1).astype(np.uint32)
+
+
+def threshold_quantize_selected(v, selected, coef=0.75):
+    """Q(S(v, I)): Q_Delta applied to the selected components only (k of them): the threshold is
+    coef/k * sum_{I}|v_i|, unselected components are not sent and decode to 0.
+    Returns (tern int8[d], s fp32, Delta fp32, |I_Delta| int, k int)."""
+    v = np.asarray(v, dtype=F32).ravel()
+    selected = np.asarray(selected, dtype=bool).ravel()
+    k = int(np.count_nonzero(selected))
+    absv = np.abs(v)
+    if k == 0:
+        return np.zeros(v.size, dtype=np.int8), F32(0.0), F32(0.0), 0, 0
+    with np.errstate(invalid="ignore", over="ignore"):
+        total = canonical_sum(np.where(selected, absv, F32(0.0)))
+        delta = F32((F64(F32(coef)) * total) / F64(k))
+        pos = selected & (v > delta)
+        neg = selected & (v < -delta)
+    tern = pos.astype(np.int8) - neg.astype(np.int8)
+    kept = pos | neg
+    n = int(np.count_nonzero(kept))
+    if n == 0:
+        return tern, F32(0.0), delta, 0, k
+    picked = canonical_sum(np.where(kept, absv, F32(0.0)))
+    return tern, F32(picked / F64(n)), delta, n, k
+
+
+def ternary_stochastic_quantize_selected(v, u, selected):
+    """The unbiased ternary quantizer on the selected components: s = max_{I}|v|."""
+    v = np.asarray(v, dtype=F32).ravel()
+    selected = np.asarray(selected, dtype=bool).ravel()
+    masked = np.where(selected, v, F32(0.0))
+    return ternary_stochastic_quantize(masked, u)
+
+
+def sparse_wire_bits(d, k):
+    """Bits one worker sends for a sparse model: 32 + d + 2k (Section 3.5, "Encode")."""
+    return 32 + int(d) + 2 * int(k)
+
+
+def select_quantize_workers(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0, coef=0.75):
+    """Workers' side of Algorithm 1 with selection: indicator from the local trial update, then
+    Q(S(g, I)).  Returns the dict of `quantize_workers` plus indicators bool[M,d], ind_words
+    uint32[M, ceil(d/32)], selected int64[M] (k_m), isyn bool[d] (the "bitwise or")."""
+    g = np.asarray(g, dtype=F32)
+    m_workers, d = g.shape
+    out = dict(terns=np.zeros((m_workers, d), np.int8), scales=np.zeros(m_workers, F32),
+               thresholds=np.zeros(m_workers, F32), counts=np.zeros(m_workers, np.int64),
+               selected=np.zeros(m_workers, np.int64), indicators=np.zeros((m_workers, d), bool))
+    for m in range(m_workers):
+        ind = indicator(rule, g[m], x, h, z, t, lam, eta, delta)
+        out["indicators"][m] = ind
+        if quantizer == QUANT_THRESHOLD:
+            tern, s, thr, n, k = threshold_quantize_selected(g[m], ind, coef)
+        else:
+            _, u = philox_draws(seed, t, m, np.arange(d, dtype=np.uint64))
+            tern, s = ternary_stochastic_quantize_selected(g[m], u, ind)
+            thr, n, k = F32(0.0), int(np.count_nonzero(tern)), int(np.count_nonzero(ind))
+        out["terns"][m], out["scales"][m], out["thresholds"][m] = tern, s, thr
+        out["counts"][m], out["selected"][m] = n, k
+    out["codes"] = np.stack([pack_codes(out["terns"][m]) for m in range(m_workers)])
+    out["ind_words"] = np.stack([pack_bits(out["indicators"][m]) for m in range(m_workers)])
+    out["isyn"] = out["indicators"].any(axis=0)
+    return out
+
+
+# ----------------------------------------------------------------------------------
 # The whole step (one-way quantization: local gradients quantized, the average not)
 # ----------------------------------------------------------------------------------
-QUANT_THRESHOLD = 0
-QUANT_TERNARY_STOCH = 1
-QUANT_NONE = 2
-RULE_CMD = 0
-RULE_RDA = 1
 
 
 def quantize_workers(g, quantizer, t=1, seed=0, coef=0.75):
@@ -330,12 +445,14 @@ def quantize_workers(g, quantizer, t=1, seed=0, coef=0.75):
 
 
 def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0, coef=0.75,
-         double_quant=False):
+         double_quant=False, select=False):
     """One iteration: quantize every worker's gradient, decode and average, update the
     accumulator and apply the rule's closed-form update.  State in, state out (fp64).
 
     double_quant=True is Algorithm 1 as printed: the average is quantized again on the server
     (q_t = Q(SynQ_t)) and the workers update from q_t; False is the one-way variant.
+    select=True adds the sparse selection: each worker sends only the coordinates its indicator
+    marks (and, with double_quant, the server quantizes only those of the synchronous indicator).
 
     quantizer == QUANT_NONE skips quantization: q is the fp64 mean of the rows of g
     (the 32-bit CMD / RDA adagrad baseline).
@@ -347,13 +464,16 @@ def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0
         quant = None
         q = g.astype(F64).sum(axis=0) / F64(g.shape[0])
     else:
-        quant = quantize_workers(g, quantizer, t=t, seed=seed, coef=coef)
+        if select:
+            quant = select_quantize_workers(rule, g, x, h, z, t, lam, eta, delta, quantizer, seed=seed, coef=coef)
+        else:
+            quant = quantize_workers(g, quantizer, t=t, seed=seed, coef=coef)
         q = decode_average(quant["terns"], quant["scales"])
     requant = None
     if double_quant:
         if quantizer == QUANT_NONE:
             raise ValueError("double quantization needs a quantizer")
-        requant = requantize(q, quantizer, t=t, seed=seed, coef=coef)
+        requant = requantize(q, quantizer, t=t, seed=seed, coef=coef, isyn=quant["isyn"] if select else None)
         q = requant["q"]
     if rule == RULE_CMD:
         x_new, h_new, a = cmd_step(q, x, h, lam, eta, delta)

@@ -428,3 +428,84 @@ def test_stochastic_requantize_uses_its_own_stream_and_is_unbiased():
     _, u_worker0 = O.philox_draws(9, 3, 0, np.arange(64, dtype=np.uint64), domain=0)
     tern_w, _ = O.ternary_stochastic_quantize(np.linspace(-1, 1, 64).astype(np.float32), u_worker0)
     assert not np.array_equal(a["tern"], tern_w)          # domain 1 is a different stream
+
+
+# ------------------------------------------------------------------ sparse selection
+def _random_sparse_state(rng, d):
+    x = rng.standard_normal(d) * 0.1 * (rng.random(d) < 0.3)          # 70 % exact zeros
+    h = rng.random(d) * (rng.random(d) < 0.8)
+    z = rng.standard_normal(d) * 0.05
+    return x.astype(np.float32), h.astype(np.float32), z.astype(np.float32)
+
+
+def test_indicator_is_the_definition_away_from_the_boundary():
+    # I = [x != 0 or x_hat != 0] with x_hat from the closed forms in fp64; the fp32 decision may
+    # differ only where the compared quantity is within rounding of lambda.
+    rng = np.random.default_rng(31)
+    d, t, lam, eta, delta = 20_000, 7, 1e-2, 0.1, 1e-8
+    x, h, z = _random_sparse_state(rng, d)
+    g = (rng.standard_normal(d) * 0.03).astype(np.float32)
+    for rule in (O.RULE_CMD, O.RULE_RDA):
+        ind = O.indicator(rule, g, x, h, z, t, lam, eta, delta)
+        x_hat = O.trial_update(rule, g, x, h, z, t, lam, eta, delta)
+        want = (x != 0) | (x_hat != 0)
+        if rule == O.RULE_CMD:
+            a = O.cmd_step(g, x, h, lam, eta, delta)[2]
+        else:
+            a = O.rda_step(g, h, z, t, lam, eta, delta)[3]
+        decided = np.abs(a - float(np.float32(lam))) > 1e-6
+        assert np.array_equal(ind[decided], want[decided])
+        assert decided.mean() > 0.999 and 0.2 < ind.mean() < 0.9
+
+
+def test_unselected_coordinates_stay_zero_when_nothing_is_sent_for_them():
+    # If no worker selects coordinate d (x_d = 0 and every trial update leaves it 0) then q_d = 0
+    # and the real update leaves x_d = 0: the selection loses nothing there.
+    rng = np.random.default_rng(32)
+    d, M, t, lam, eta, delta = 5000, 3, 5, 2e-2, 0.1, 1e-8
+    x, h, z = _random_sparse_state(rng, d)
+    z = (z * 0.1).astype(np.float32)
+    g = (rng.standard_normal((M, d)) * 0.02).astype(np.float32)
+    for rule in (O.RULE_CMD, O.RULE_RDA):
+        out = O.step(rule, g, x, h, z, t, lam, eta, delta, select=True)
+        isyn = out["quant"]["isyn"]
+        assert 0 < isyn.sum() < d
+        assert not out["q"][~isyn].any() and not out["x"][~isyn].any()
+        assert np.array_equal(out["h"][~isyn], h[~isyn].astype(np.float64))
+
+
+def test_selected_quantizer_is_q_on_the_selected_subvector():
+    # Q(S(v, I)) equals Q_Delta applied to the compacted vector of the k selected components
+    rng = np.random.default_rng(33)
+    d = 9000
+    v = rng.standard_normal(d).astype(np.float32)
+    sel = rng.random(d) < 0.37
+    tern, s, delta, n, k = O.threshold_quantize_selected(v, sel)
+    sub = v[sel]
+    exact = math.fsum(abs(float(a)) for a in sub)
+    assert k == sub.size and delta == np.float32(0.75 * exact / k)
+    kept = np.abs(sub) > delta
+    assert n == int(kept.sum()) and np.array_equal(tern[sel] != 0, kept) and not tern[~sel].any()
+    assert float(s) == pytest.approx(np.abs(sub.astype(np.float64))[kept].mean(), rel=1e-6)
+    # nothing selected, everything selected
+    assert O.threshold_quantize_selected(v, np.zeros(d, bool))[1:] == (0, 0, 0, 0)
+    full = O.threshold_quantize_selected(v, np.ones(d, bool))
+    ref = O.threshold_quantize(v)
+    assert np.array_equal(full[0], ref[0]) and full[1:4] == ref[1:]
+
+
+def test_indicator_words_or_and_sparse_bit_budget():
+    rng = np.random.default_rng(34)
+    d, M = 1000, 4
+    x, h, z = _random_sparse_state(rng, d)
+    g = (rng.standard_normal((M, d)) * 0.01).astype(np.float32)
+    out = O.select_quantize_workers(O.RULE_CMD, g, x, h, z, 3, 1e-2, 0.1, 1e-8)
+    assert out["ind_words"].shape == (M, 32) and out["ind_words"].dtype == np.uint32
+    for m in range(M):
+        bits = ((out["ind_words"][m][:, None] >> np.arange(32, dtype=np.uint32)) & 1).ravel()[:d].astype(bool)
+        assert np.array_equal(bits, out["indicators"][m]) and out["selected"][m] == bits.sum()
+    assert np.array_equal(O.pack_bits(out["isyn"]), np.bitwise_or.reduce(out["ind_words"], axis=0))
+    assert int(O.pack_bits(np.array([1, 0, 1] + [0] * 30 + [1], bool))[0]) == 5 and O.pack_bits(np.ones(33, bool))[1] == 1
+    k = int(out["selected"][0])
+    assert O.sparse_wire_bits(d, k) == 32 + d + 2 * k
+    assert (O.sparse_wire_bits(d, k) < O.wire_bits(d)) == (k < d / 2)         # cheaper iff k < d/2
