@@ -166,6 +166,42 @@ qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint
                              float* z, uint32_t* codes_out, float* scales_out, uint32_t* qcodes_out,
                              float* qscale_out, void* stream);
 
+/* Workers' side of Algorithm 1 with the sparse selection of Section 3.2: "Compute the indicator
+ * function", "Quantize the selected elements of the gradients" Q(S(g, I)).
+ * Worker m's indicator marks coordinate i when x_i != 0 or when the worker's local trial update,
+ * taken with its own full-precision gradient and H_hat = delta + sqrt(h + g^2), leaves it non-zero.
+ * The test is evaluated in fp32, every operation rounded on its own:
+ *   QCMD: |x*H_hat - eta*g| > lambda*eta        QRDA: |z + g| > lambda*t
+ * Only marked coordinates are quantized: Delta_m = thr_coef/k_m * sum over them of |g| (k_m of
+ * them), the scale is the mean kept magnitude (stochastic quantizer: the maximum over them);
+ * unmarked coordinates code 0.
+ *   x, h, z     device, fp32 [d]: the current state (read only); h used by QCMD, z by QRDA.
+ *   indicators  device, uint32 [M][ceil(d/32)]: bit i&31 of word i>>5 of row m; unused bits 0.
+ *   selected    device, uint64 [M] or NULL: k_m.  A worker's message is then 32 + d + 2*k_m bits
+ *               (Section 3.5 "Encode").
+ *   other arguments as for qasg_quantize_pack. */
+qasg_status qasg_select_quantize_pack(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
+                                      uint64_t ld_g, uint32_t M, uint64_t t, const qasg_params* params,
+                                      const float* x, const float* h, const float* z, uint32_t* codes,
+                                      float* scales, float* thresholds, uint64_t* counts,
+                                      uint32_t* indicators, uint64_t* selected, void* stream);
+
+/* Server's side: "Compute the synchronous indicator", the bitwise OR of the M indicators.
+ *   isyn  device, uint32 [ceil(d/32)].   ksyn  device, uint64 [1]: its number of set bits. */
+qasg_status qasg_indicator_or(qasg_ctx* ctx, const uint32_t* indicators, uint64_t d, uint32_t M,
+                              uint32_t* isyn, uint64_t* ksyn, void* stream);
+
+/* The whole iteration with sparse selection, fused like qasg_step (double_quant = 0) or like
+ * qasg_step_double (double_quant != 0: the server quantizes the average over the coordinates of
+ * the synchronous indicator only, Delta' = thr_coef/k_syn * sum|avg|).
+ *   indicators_out, selected_out, isyn_out, ksyn_out   device, as above, each may be NULL
+ *   (NULL indicators use the context's scratch).  Other arguments as for qasg_step. */
+qasg_status qasg_step_select(qasg_ctx* ctx, qasg_rule rule, int double_quant, const float* g, uint64_t d,
+                             uint64_t ld_g, uint32_t M, uint64_t t, const qasg_params* params, float* x,
+                             float* h, float* z, uint32_t* codes_out, float* scales_out,
+                             uint32_t* indicators_out, uint64_t* selected_out, uint32_t* isyn_out,
+                             uint64_t* ksyn_out, void* stream);
+
 /* qasg_step for callers whose data lives in host memory.  Copies g (M rows of d floats,
  * row stride ld_g) and the state from the host buffers into the caller's device staging
  * buffers, runs qasg_step there, and copies the new state back, all on `stream`; returns
@@ -254,7 +290,7 @@ uint64_t qasg_launch_count(const qasg_ctx* ctx);
  * adds up, per kernel id (0 <= id < QASG_KERNEL_COUNT, names from qasg_kernel_name), the
  * elapsed milliseconds into ms[id] and the number of launches into launches[id] (both host
  * arrays of QASG_KERNEL_COUNT entries), then stops recording. */
-#define QASG_KERNEL_COUNT 16
+#define QASG_KERNEL_COUNT 24
 qasg_status qasg_profile_begin(qasg_ctx* ctx);
 qasg_status qasg_profile_end(qasg_ctx* ctx, double* ms, uint64_t* launches);
 const char* qasg_kernel_name(int id);

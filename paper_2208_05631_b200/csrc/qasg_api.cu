@@ -18,6 +18,8 @@ struct qasg_ctx {
   uint32_t* code_scratch;   // [M_max][code_words(d_max)] or NULL
   uint32_t* qcode_scratch;  // [code_words(d_max)] or NULL
   float* gbar_scratch;      // [d_max rounded up to 4] or NULL: the averaged gradient of the server row
+  uint32_t* ind_scratch;    // [M_max + 1][ceil(d_max/32)] or NULL: workers' indicators, then their OR
+  unsigned long long* ksyn; // [1] number of bits of the synchronous indicator
   float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
   uint64_t launches;
   bool profiling;
@@ -30,7 +32,7 @@ namespace {
 enum KernelId {
   kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
   kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kAvgAbsSum, kAvgAbsMax,
-  kAvgThresholdCodes, kAvgStochasticCodes, kKernelIdCount
+  kAvgThresholdCodes, kAvgStochasticCodes, kSelectStats, kIndicatorOr, kKernelIdCount
 };
 static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
 
@@ -121,9 +123,10 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
 // With scratch, the average is written once as an fp32 row (fast per-lane-table decode) and the
 // workers' own two quantization kernels run on that row; without, two kernels rebuild the average
 // from the code bytes and nothing is stored.  Both give the same bits.
+// denom (device, [1]): number of coordinates of the synchronous indicator when Q runs over those only.
 void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M, uint64_t t,
                 const qasg_params* p, uint32_t* qcodes, float* qscale, float* qthreshold, uint64_t* qcount,
-                cudaStream_t stream) {
+                cudaStream_t stream, const unsigned long long* denom = nullptr) {
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
   unsigned long long* count_out = reinterpret_cast<unsigned long long*>(qcount);
   if (ctx->gbar_scratch) {
@@ -135,7 +138,7 @@ void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint6
     }
     const Geometry row = make_geometry(d, ld, 1);
     if (!stochastic) {
-      { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(gbar, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream); }
+      { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(gbar, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream, denom); }
       { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(gbar, row, ctx->wsq, qcodes, qscale, count_out, ctx->shape, stream); }
     } else {
       { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(gbar, row, ctx->wsq, ctx->shape, stream); }
@@ -145,7 +148,7 @@ void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint6
     const Geometry row = make_geometry(d, d, 1, kRowChunks);
     {
       Launch l(ctx, stochastic ? kAvgAbsMax : kAvgAbsSum, stream);
-      l += launch_avg_stats(stochastic, codes, scales, M, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream);
+      l += launch_avg_stats(stochastic, codes, scales, M, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream, denom);
     }
     {
       Launch l(ctx, stochastic ? kAvgStochasticCodes : kAvgThresholdCodes, stream);
@@ -154,6 +157,35 @@ void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint6
     }
   }
   if (stochastic && qthreshold) cudaMemsetAsync(qthreshold, 0, sizeof(float), stream);
+}
+
+// Workers' side with sparse selection on validated arguments: indicators, then Q(S(g, I)).
+void select_quantize_pack(qasg_ctx* ctx, int rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint64_t t,
+                          const qasg_params* p, const float* x, const float* h, const float* z, uint32_t* codes,
+                          float* scales, float* thresholds, uint64_t* counts, uint32_t* indicators,
+                          uint64_t* selected, cudaStream_t stream) {
+  const Geometry geo = make_geometry(d, ld_g, M);
+  const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
+  SelectScalars sc;
+  sc.lambda_eta = p->lambda * p->eta;
+  sc.eta = p->eta;
+  sc.delta = p->delta;
+  sc.lambda_t = p->lambda * static_cast<float>(t);
+  unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
+  {
+    Launch l(ctx, kSelectStats, stream);
+    l += launch_select_stats(rule, stochastic, g, geo, x, rule == QASG_RULE_CMD ? h : z, sc, p->thr_coef, ctx->ws,
+                             indicators, thresholds, reinterpret_cast<unsigned long long*>(selected), ctx->shape,
+                             stream);
+  }
+  if (!stochastic) {
+    Launch l(ctx, kThresholdCodes, stream);
+    l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream, indicators);
+  } else {
+    Launch l(ctx, kStochasticCodes, stream);
+    l += launch_stochastic_codes(g, geo, p->seed, t, 0u, ctx->ws, codes, scales, counts_out, ctx->shape, stream,
+                                 indicators);
+  }
 }
 
 qasg_status check_gradient(const float* g, uint64_t d, uint64_t ld_g) {
@@ -189,6 +221,8 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ok &= cudaMalloc(&ctx->ws.thresholds, kMaxWorkers * sizeof(float)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->ws.scales, kMaxWorkers * sizeof(float)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->ws.counts, kMaxWorkers * sizeof(unsigned long long)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ws.selected, kMaxWorkers * sizeof(unsigned long long)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->ksyn, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->ws.ticket, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->ws.status, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->logreg_ws, kLogregEntries * 2 * sizeof(float)) == cudaSuccess;
@@ -198,12 +232,14 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ok &= cudaMalloc(&ctx->wsq.thresholds, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.scales, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.counts, 64) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wsq.selected, 64) == cudaSuccess;
   ctx->wsq.ticket = ctx->ws.ticket;
   ctx->wsq.status = ctx->ws.status;
   if (ok && !(flags & QASG_CREATE_NO_CODE_SCRATCH)) {
     ok &= cudaMalloc(&ctx->code_scratch, static_cast<size_t>(M_max) * qasg_code_words(d_max) * 4) == cudaSuccess;
     ok &= cudaMalloc(&ctx->qcode_scratch, qasg_code_words(d_max) * 4) == cudaSuccess;
     ok &= cudaMalloc(&ctx->gbar_scratch, ((d_max + 3) / 4) * 4 * sizeof(float)) == cudaSuccess;
+    ok &= cudaMalloc(&ctx->ind_scratch, static_cast<size_t>(M_max + 1) * ((d_max + 31) / 32) * 4) == cudaSuccess;
   }
   if (ok) {
     ok &= cudaMemset(ctx->ws.ticket, 0, 64) == cudaSuccess;
@@ -237,6 +273,10 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->code_scratch);
   cudaFree(ctx->qcode_scratch);
   cudaFree(ctx->gbar_scratch);
+  cudaFree(ctx->ind_scratch);
+  cudaFree(ctx->ksyn);
+  cudaFree(ctx->ws.selected);
+  cudaFree(ctx->wsq.selected);
   cudaFree(ctx->wsq.part_sum);
   cudaFree(ctx->wsq.part_max);
   cudaFree(ctx->wsq.part_cnt);
@@ -362,6 +402,81 @@ qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint
     // the workers decode q_t (one code row, one scale) and update
     Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s);
     l += launch_decode_update(rule, qcodes, ctx->wsq.scales, d, 1, x, h, z, scalars(params, t), ctx->ws.status,
+                              ctx->shape, s);
+  }
+  return leave();
+}
+
+qasg_status qasg_select_quantize_pack(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
+                                      uint32_t M, uint64_t t, const qasg_params* params, const float* x,
+                                      const float* h, const float* z, uint32_t* codes, float* scales,
+                                      float* thresholds, uint64_t* counts, uint32_t* indicators,
+                                      uint64_t* selected, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
+  if (!x || !codes || !scales || !indicators || t < 1) return QASG_ERR_INVALID_ARG;
+  if ((rule == QASG_RULE_CMD && !h) || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(x) || (h && !aligned16(h)) || (z && !aligned16(z)) || !aligned16(codes) || !aligned16(indicators))
+    return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  select_quantize_pack(ctx, rule, g, d, ld_g, M, t, params, x, h, z, codes, scales, thresholds, counts, indicators,
+                       selected, static_cast<cudaStream_t>(stream));
+  return leave();
+}
+
+qasg_status qasg_indicator_or(qasg_ctx* ctx, const uint32_t* indicators, uint64_t d, uint32_t M, uint32_t* isyn,
+                              uint64_t* ksyn, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st != QASG_OK) return st;
+  if (!indicators || !isyn || !ksyn) return QASG_ERR_INVALID_ARG;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  {
+    Launch l(ctx, kIndicatorOr, static_cast<cudaStream_t>(stream));
+    l += launch_indicator_or(indicators, d, M, isyn, reinterpret_cast<unsigned long long*>(ksyn), ctx->shape,
+                             static_cast<cudaStream_t>(stream));
+  }
+  return leave();
+}
+
+qasg_status qasg_step_select(qasg_ctx* ctx, qasg_rule rule, int double_quant, const float* g, uint64_t d,
+                             uint64_t ld_g, uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h,
+                             float* z, uint32_t* codes_out, float* scales_out, uint32_t* indicators_out,
+                             uint64_t* selected_out, uint32_t* isyn_out, uint64_t* ksyn_out, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
+  if (!x || !h || t < 1 || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(h) || (z && !aligned16(z)) || (codes_out && !aligned16(codes_out)) ||
+      (indicators_out && !aligned16(indicators_out)))
+    return QASG_ERR_ALIGNMENT;
+  uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
+  uint32_t* indicators = indicators_out ? indicators_out : ctx->ind_scratch;
+  uint32_t* isyn = isyn_out;  // else the row after the M_max indicator rows of the scratch
+  if (!isyn && ctx->ind_scratch) isyn = ctx->ind_scratch + static_cast<size_t>(ctx->M_max) * ((ctx->d_max + 31) / 32);
+  const bool need_or = double_quant || isyn_out || ksyn_out;
+  if (!codes || !indicators || (need_or && !isyn) || (double_quant && !ctx->qcode_scratch)) return QASG_ERR_WORKSPACE;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  select_quantize_pack(ctx, rule, g, d, ld_g, M, t, params, x, h, z, codes, scales_out, nullptr, nullptr, indicators,
+                       selected_out, s);
+  unsigned long long* ksyn = ksyn_out ? reinterpret_cast<unsigned long long*>(ksyn_out) : ctx->ksyn;
+  if (need_or) {
+    Launch l(ctx, kIndicatorOr, s);
+    l += launch_indicator_or(indicators, d, M, isyn, ksyn, ctx->shape, s);
+  }
+  if (double_quant) {
+    requantize(ctx, codes, ctx->ws.scales, d, M, t, params, ctx->qcode_scratch, nullptr, nullptr, nullptr, s, ksyn);
+    Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s);
+    l += launch_decode_update(rule, ctx->qcode_scratch, ctx->wsq.scales, d, 1, x, h, z, scalars(params, t),
+                              ctx->ws.status, ctx->shape, s);
+  } else {
+    Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s);
+    l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t), ctx->ws.status,
                               ctx->shape, s);
   }
   return leave();
@@ -494,7 +609,7 @@ const char* qasg_kernel_name(int id) {
   static const char* const names[kKernelIdCount] = {
       "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
       "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr", "avg_abs_sum",
-      "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes"};
+      "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes", "select_stats", "indicator_or"};
   return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
 }
 

@@ -42,6 +42,7 @@ struct Workspace {
   float* thresholds;             // [M_max] Delta_m
   float* scales;                 // [M_max] s_m
   unsigned long long* counts;    // [M_max] non-zero codes
+  unsigned long long* selected;  // [M_max] coordinates the worker's indicator selects (sparse selection)
   unsigned int* ticket;          // grid-completion counter, zero between launches
   unsigned int* status;          // OR of kFlag*
 };
@@ -52,23 +53,37 @@ struct LaunchShape {
   int update_ctas_per_sm;  // same for the coordinate-wise kernels
 };
 
+// Constants of the indicator test, rounded to fp32 on the host: lambda*eta, lambda*t.
+struct SelectScalars {
+  float lambda_eta, eta, delta, lambda_t;
+};
+
 struct StepScalars {
   float lambda, eta, delta, t, inv_t;
 };
 
 // Each launcher enqueues on `stream` and returns the number of kernels it launched.
+// denom (device, [M]) replaces d in Delta = coef * sum / d when the sum runs over selected coordinates.
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
-                   float* thresholds_out, const LaunchShape& shape, cudaStream_t stream);
+                   float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
+                   const unsigned long long* denom = nullptr);
 int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
                    const LaunchShape& shape, cudaStream_t stream);
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
-                           const LaunchShape& shape, cudaStream_t stream);
+                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators = nullptr);
 // stream_base is added to the worker index in Philox counter word 1 (0 for workers, 1<<16 for the server row).
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
                             uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
-                            cudaStream_t stream);
+                            cudaStream_t stream, const uint32_t* indicators = nullptr);
+// Sparse selection: indicators [M][ceil(d/32)] words, bit i&31 of word i>>5.
+int launch_select_stats(int rule, bool stochastic, const float* g, const Geometry& geo, const float* x,
+                        const float* hz, const SelectScalars& sc, float coef, const Workspace& ws,
+                        uint32_t* indicators, float* thresholds_out, unsigned long long* selected_out,
+                        const LaunchShape& shape, cudaStream_t stream);
+int launch_indicator_or(const uint32_t* indicators, uint64_t d, uint32_t M, uint32_t* isyn,
+                        unsigned long long* ksyn, const LaunchShape& shape, cudaStream_t stream);
 // rule 0 = QCMD, 1 = QRDA, 2 = write the averaged gradient to x (h, z unused).
 int launch_decode_update(int rule, const uint32_t* codes, const float* scales, uint64_t d,
                          uint32_t M, float* x, float* h, float* z, const StepScalars& sc,
@@ -80,7 +95,7 @@ int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d
 // one row of d coordinates with up to kRowChunks chunks; wsq holds kRowChunks partial slots.
 int launch_avg_stats(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
                      const Geometry& row, float coef, const Workspace& wsq, float* threshold_out,
-                     const LaunchShape& shape, cudaStream_t stream);
+                     const LaunchShape& shape, cudaStream_t stream, const unsigned long long* denom = nullptr);
 int launch_avg_codes(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
                      const Geometry& row, uint64_t seed, uint64_t t, const Workspace& wsq, uint32_t* qcodes,
                      float* scale_out, unsigned long long* count_out, const LaunchShape& shape,

@@ -192,7 +192,7 @@ __device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64
 // ------------------------------------------------------------------ pass A: sum |g|
 __global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
-               float* __restrict__ thresholds_out) {
+               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom) {
   __shared__ ChunkSumStorage sm_sum;
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -222,7 +222,9 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
     const double total = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
     if (lane == 0) {
-      const float delta = static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(geo.d));
+      // the mean is over all d coordinates, or over the selected ones when a count is given
+      const unsigned long long n = denom ? denom[m] : geo.d;
+      const float delta = n ? static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(n)) : 0.f;
       ws.thresholds[m] = delta;
       if (thresholds_out) thresholds_out[m] = delta;
       if (!isfinite(total)) atomicOr(ws.status, kFlagNonFinite);
@@ -370,11 +372,20 @@ __device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspac
   }
 }
 
+// The four selection bits of coordinates i0..i0+3 of a worker whose indicator row is ind8
+// (bit i&7 of byte i>>3); all ones when no indicator is in use.
+__device__ __forceinline__ uint32_t indicator_nibble(const uint8_t* __restrict__ ind8, uint64_t i0, uint64_t d) {
+  if (i0 >= d) return 0u;
+  return (static_cast<uint32_t>(__ldg(ind8 + (i0 >> 3))) >> (i0 & 4u)) & 15u;
+}
+
 // ------------------------------------------------------------------ pass B: Q_Delta codes
+// kMasked: only coordinates whose indicator bit is set are candidates (sparse selection, Q(S(g, I))).
+template <bool kMasked>
 __global__ void __launch_bounds__(kThreads, 4)
 threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
                        uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                       unsigned long long* __restrict__ counts_out) {
+                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
   __shared__ ChunkSumStorage sm_sum;
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
@@ -388,6 +399,8 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
     const float delta = ws.thresholds[m], ndelta = -delta;
+    const uint8_t* ind8 = kMasked ? reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5))
+                                  : nullptr;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     float cntf = 0.f;
@@ -398,10 +411,16 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
       for (int r = 0; r < kTileRows; ++r) {
         const float4 t = v[r];
         // strict comparisons; a NaN threshold or value compares false and codes 0
-        const float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
-        const float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
-        const float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
-        const float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+        float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
+        float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
+        float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
+        float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+        if (kMasked) {
+          const uint32_t nib = indicator_nibble(ind8, static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j, geo.d);
+          const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
+          const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
+          px *= sx, nx *= sx, py *= sy, ny *= sy, pz *= sz, nz *= sz, pw *= sw, nw *= sw;
+        }
         const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;  // 1.0f where kept
         // |v| * 1 = |v| and |v| * 0 = +0: the kept magnitudes enter the sum unchanged
         cx += static_cast<double>(fabsf(t.x) * kx);
@@ -450,10 +469,11 @@ __device__ __forceinline__ float philox_uniform(uint32_t word) {
 }
 
 // ------------------------------------------------------------------ pass B': stochastic codes
+template <bool kMasked>
 __global__ void __launch_bounds__(kThreads)
 stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
                         uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                        unsigned long long* __restrict__ counts_out) {
+                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -467,6 +487,8 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
     const float scale = ws.scales[m];
+    const uint8_t* ind8 = kMasked ? reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5))
+                                  : nullptr;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
@@ -479,10 +501,14 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
         const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
         const uint4 w = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), key0, key1);
         // |v|/s with IEEE division; s = 0 gives NaN and the comparison is false.
-        const bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
-        const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
-        const bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
-        const bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
+        bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
+        bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
+        bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
+        bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
+        if (kMasked) {
+          const uint32_t nib = indicator_nibble(ind8, static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j, geo.d);
+          kx = kx && (nib & 1u), ky = ky && (nib & 2u), kz = kz && (nib & 4u), kw = kw && (nib & 8u);
+        }
         bytes[r] = pack4(split_code(v.x, kx), split_code(v.y, ky), split_code(v.z, kz), split_code(v.w, kw));
         cnt += nonzero_codes(bytes[r]);
       }
@@ -788,7 +814,8 @@ __device__ __forceinline__ double block_chunk_tree(const double* part, uint32_t 
 
 __global__ void __launch_bounds__(kThreads, 4)
 avg_abs_sum_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint32_t workers,
-                   double inv_m, Geometry geo, float coef, Workspace ws, float* __restrict__ threshold_out) {
+                   double inv_m, Geometry geo, float coef, Workspace ws, float* __restrict__ threshold_out,
+                   const unsigned long long* __restrict__ denom) {
   extern __shared__ double sm_lut[];
   __shared__ ChunkSumStorage sm_sum;
   __shared__ double sm8[kThreads / 32];
@@ -822,7 +849,8 @@ avg_abs_sum_kernel(const uint32_t* __restrict__ codes, const float* __restrict__
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   const double total = block_chunk_tree(ws.part_sum, geo.chunks, sm8);
   if (j == 0) {
-    const float delta = static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(geo.d));
+    const unsigned long long n = denom ? denom[0] : geo.d;
+    const float delta = n ? static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(n)) : 0.f;
     ws.thresholds[0] = delta;
     if (threshold_out) threshold_out[0] = delta;
     *ws.ticket = 0u;
@@ -977,13 +1005,179 @@ avg_codes_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ s
   }
 }
 
+// ------------------------------------------------------------------ sparse selection
+// Indicator of one coordinate of one worker (Section 3.2): x != 0, or the worker's local trial update
+// with its own gradient leaves the coordinate non-zero.  Decided in fp32 by correctly rounded
+// operations taken one by one (no fused multiply-add), so that the bit does not depend on who computes it:
+//   QCMD: |x*H - eta*g| > lambda*eta with H = delta + sqrt(h + g*g)   (hz = h)
+//   QRDA: |z + g| > lambda*t                                          (hz = z)
+template <int kRule>
+__device__ __forceinline__ bool selects(float g, float x, float hz, const SelectScalars& sc) {
+  bool moved;
+  if (kRule == 0) {
+    const float big_h = __fadd_rn(sc.delta, __fsqrt_rn(__fadd_rn(hz, __fmul_rn(g, g))));
+    moved = fabsf(__fsub_rn(__fmul_rn(x, big_h), __fmul_rn(sc.eta, g))) > sc.lambda_eta;
+  } else {
+    moved = fabsf(__fadd_rn(hz, g)) > sc.lambda_t;
+  }
+  return (x != 0.f) || moved;
+}
+
+// A thread's four float4 of tile k of a state vector of exactly d floats (no padding to read into).
+__device__ __forceinline__ void load_state_tile(const float* __restrict__ v, uint64_t d, uint32_t k, int j,
+                                                float4 (&out)[kTileRows]) {
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) {
+    const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 + 4 <= d) {
+      t = load_f4(v + i0);
+    } else if (i0 < d) {
+      t.x = v[i0];
+      if (i0 + 1 < d) t.y = v[i0 + 1];
+      if (i0 + 2 < d) t.z = v[i0 + 2];
+    }
+    out[r] = t;
+  }
+}
+
+// Pass A with selection: writes each worker's indicator bits and reduces, over the selected
+// coordinates only, the sum of |g| (threshold quantizer: Delta_m = coef * sum / k_m) or the maximum
+// (stochastic quantizer), and k_m.  Items run chunk-major so that the M workers of a chunk share
+// the chunk's x and h (or z) in L2.
+template <int kRule, bool kStochastic>
+__global__ void __launch_bounds__(kThreads, 3)
+select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __restrict__ x,
+                    const float* __restrict__ hz, SelectScalars sc, float coef, Workspace ws,
+                    uint32_t* __restrict__ indicators, float* __restrict__ thresholds_out,
+                    unsigned long long* __restrict__ selected_out) {
+  __shared__ ChunkSumStorage sm_sum;
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ bool sm_last;
+  const int j = threadIdx.x;
+  const uint32_t n_items = geo.M * geo.chunks;
+  const uint64_t ind_words = (geo.d + 31) >> 5;
+  ChunkSum chunk_sum(&sm_sum);
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const uint32_t c = item / geo.M, m = item - c * geo.M;
+    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+    uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words);
+    const uint32_t k0 = c * geo.group;
+    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
+    float cntf = 0.f;
+    uint32_t best = 0u;
+    for (uint32_t k = k0; k < k1; ++k) {
+      float4 gv[kTileRows], xv[kTileRows], hv[kTileRows];
+      load_tile(row, static_cast<uint64_t>(k) * kTile, geo.d, j, gv);
+      load_state_tile(x, geo.d, k, j, xv);
+      load_state_tile(hz, geo.d, k, j, hv);
+      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) {
+        const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
+        const bool bx = i0 < geo.d && selects<kRule>(gv[r].x, xv[r].x, hv[r].x, sc);
+        const bool by = i0 + 1 < geo.d && selects<kRule>(gv[r].y, xv[r].y, hv[r].y, sc);
+        const bool bz = i0 + 2 < geo.d && selects<kRule>(gv[r].z, xv[r].z, hv[r].z, sc);
+        const bool bw = i0 + 3 < geo.d && selects<kRule>(gv[r].w, xv[r].w, hv[r].w, sc);
+        const float sx = bx ? 1.f : 0.f, sy = by ? 1.f : 0.f, sz = bz ? 1.f : 0.f, sw = bw ? 1.f : 0.f;
+        if (!kStochastic) {
+          cx += static_cast<double>(fabsf(gv[r].x) * sx);
+          cy += static_cast<double>(fabsf(gv[r].y) * sy);
+          cz += static_cast<double>(fabsf(gv[r].z) * sz);
+          cw += static_cast<double>(fabsf(gv[r].w) * sw);
+        } else {
+          best = max(best, __float_as_uint(fabsf(gv[r].x) * sx));
+          best = max(best, __float_as_uint(fabsf(gv[r].y) * sy));
+          best = max(best, __float_as_uint(fabsf(gv[r].z) * sz));
+          best = max(best, __float_as_uint(fabsf(gv[r].w) * sw));
+        }
+        cntf += (sx + sy) + (sz + sw);
+        // two adjacent threads share an indicator byte; the even one writes it (zeros past d)
+        const uint32_t nib = static_cast<uint32_t>(bx) | (static_cast<uint32_t>(by) << 1) |
+                             (static_cast<uint32_t>(bz) << 2) | (static_cast<uint32_t>(bw) << 3);
+        const uint32_t upper = __shfl_down_sync(0xffffffffu, nib, 1);
+        if ((j & 1) == 0 && (i0 >> 3) < ind_words * 4) ind8[i0 >> 3] = static_cast<uint8_t>(nib | (upper << 4));
+      }
+      if (!kStochastic) chunk_sum.add_tile((cx + cy) + (cz + cw));
+    }
+    double total = 0.0;
+    if (!kStochastic) total = chunk_sum.finish(geo.log2_group);
+    if (kStochastic) {
+      best = __reduce_max_sync(0xffffffffu, best);
+      __syncthreads();
+      if ((j & 31) == 0) sm_cnt[j >> 5] = best;
+      __syncthreads();
+      if (j == 0) {
+        uint32_t bmax = sm_cnt[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) bmax = max(bmax, sm_cnt[w]);
+        ws.part_max[static_cast<uint64_t>(m) * kMaxChunks + c] = bmax;
+      }
+    }
+    const unsigned long long selected = block_count(static_cast<uint32_t>(cntf), sm_cnt);
+    if (j == 0) {
+      const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
+      ws.part_sum[p] = total;
+      ws.part_cnt[p] = selected;
+    }
+  }
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  const int warp = j >> 5, lane = j & 31;
+  for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
+    unsigned long long n = 0;
+    uint32_t bmax = 0u;
+    for (uint32_t idx = lane; idx < geo.chunks; idx += 32) {
+      n += __ldcg(ws.part_cnt + static_cast<uint64_t>(m) * kMaxChunks + idx);
+      if (kStochastic) bmax = max(bmax, __ldcg(ws.part_max + static_cast<uint64_t>(m) * kMaxChunks + idx));
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
+    double total = 0.0;
+    if (!kStochastic) total = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+    if (kStochastic) bmax = __reduce_max_sync(0xffffffffu, bmax);
+    if (lane == 0) {
+      ws.selected[m] = n;
+      if (selected_out) selected_out[m] = n;
+      if (!kStochastic) {
+        const float delta = n ? static_cast<float>((static_cast<double>(coef) * total) / static_cast<double>(n)) : 0.f;
+        ws.thresholds[m] = delta;
+        if (thresholds_out) thresholds_out[m] = delta;
+        if (!isfinite(total)) atomicOr(ws.status, kFlagNonFinite);
+      } else {
+        ws.scales[m] = __uint_as_float(bmax);
+        ws.thresholds[m] = 0.f;
+        if (thresholds_out) thresholds_out[m] = 0.f;
+        if (bmax >= 0x7f800000u) atomicOr(ws.status, kFlagNonFinite);
+      }
+    }
+  }
+  if (j == 0) *ws.ticket = 0u;
+}
+
+// The synchronous indicator: "bitwise or" of the M workers' indicators, and how many bits it has.
+__global__ void __launch_bounds__(kThreads)
+indicator_or_kernel(const uint32_t* __restrict__ indicators, uint64_t words, uint32_t M,
+                    uint32_t* __restrict__ isyn, unsigned long long* __restrict__ ksyn) {
+  unsigned long long bits = 0;
+  for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < words;
+       w += static_cast<uint64_t>(gridDim.x) * kThreads) {
+    uint32_t acc = 0u;
+    for (uint32_t m = 0; m < M; ++m) acc |= __ldg(indicators + m * words + w);
+    isyn[w] = acc;
+    bits += __popc(acc);
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, s);
+  if ((threadIdx.x & 31) == 0 && bits) atomicAdd(ksyn, bits);
+}
+
 // ------------------------------------------------------------------ launchers
 void query_launch_shape(LaunchShape* shape) {
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&shape->sm_count, cudaDevAttrMultiProcessorCount, dev);
   int a = 0, b = 0;
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel, kThreads, 0);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel<false>, kThreads, 0);
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dense_update_kernel<1>, kThreads, 0);
   shape->reduce_ctas_per_sm = a > 0 ? a : 1;
   shape->update_ctas_per_sm = b > 0 ? b : 1;
@@ -1003,8 +1197,9 @@ static unsigned update_grid(uint64_t d, const LaunchShape& shape) {
 }
 
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
-                   float* thresholds_out, const LaunchShape& shape, cudaStream_t stream) {
-  abs_sum_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out);
+                   float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
+                   const unsigned long long* denom) {
+  abs_sum_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom);
   return 1;
 }
 
@@ -1016,18 +1211,52 @@ int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
 
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
-                           const LaunchShape& shape, cudaStream_t stream) {
-  threshold_codes_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                          counts_out);
+                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators) {
+  if (indicators)
+    threshold_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                                  counts_out, indicators);
+  else
+    threshold_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                                   counts_out, nullptr);
   return 1;
 }
 
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
                             uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
-                            cudaStream_t stream) {
-  stochastic_codes_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, seed, t, stream_base, ws, codes,
-                                                                           scales_out, counts_out);
+                            cudaStream_t stream, const uint32_t* indicators) {
+  if (indicators)
+    stochastic_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+        g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, indicators);
+  else
+    stochastic_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+        g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, nullptr);
+  return 1;
+}
+
+int launch_select_stats(int rule, bool stochastic, const float* g, const Geometry& geo, const float* x,
+                        const float* hz, const SelectScalars& sc, float coef, const Workspace& ws,
+                        uint32_t* indicators, float* thresholds_out, unsigned long long* selected_out,
+                        const LaunchShape& shape, cudaStream_t stream) {
+  const unsigned grid = reduce_grid(geo, shape);
+#define QASG_SELECT(R, S) \
+  select_stats_kernel<R, S><<<grid, kThreads, 0, stream>>>(g, geo, x, hz, sc, coef, ws, indicators, thresholds_out, selected_out)
+  if (rule == 0 && !stochastic) QASG_SELECT(0, false);
+  else if (rule == 0) QASG_SELECT(0, true);
+  else if (!stochastic) QASG_SELECT(1, false);
+  else QASG_SELECT(1, true);
+#undef QASG_SELECT
+  return 1;
+}
+
+int launch_indicator_or(const uint32_t* indicators, uint64_t d, uint32_t M, uint32_t* isyn,
+                        unsigned long long* ksyn, const LaunchShape& shape, cudaStream_t stream) {
+  const uint64_t words = (d + 31) >> 5;
+  const uint64_t ctas = (words + kThreads - 1) / kThreads;
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * 8;
+  cudaMemsetAsync(ksyn, 0, sizeof(unsigned long long), stream);
+  indicator_or_kernel<<<static_cast<unsigned>(ctas < resident ? ctas : resident), kThreads, 0, stream>>>(
+      indicators, words, M, isyn, ksyn);
   return 1;
 }
 
@@ -1112,14 +1341,14 @@ static unsigned row_grid(const Geometry& geo, const LaunchShape& shape) {
 
 int launch_avg_stats(bool stochastic, const uint32_t* codes, const float* scales, uint32_t workers,
                      const Geometry& row, float coef, const Workspace& wsq, float* threshold_out,
-                     const LaunchShape& shape, cudaStream_t stream) {
+                     const LaunchShape& shape, cudaStream_t stream, const unsigned long long* denom) {
   const size_t lut_bytes = static_cast<size_t>((workers + 3) / 4) * 256 * sizeof(double);
   const double inv_m = 1.0 / static_cast<double>(workers);
   if (stochastic)
     avg_abs_max_kernel<<<row_grid(row, shape), kThreads, lut_bytes, stream>>>(codes, scales, workers, inv_m, row, wsq);
   else
     avg_abs_sum_kernel<<<row_grid(row, shape), kThreads, lut_bytes, stream>>>(codes, scales, workers, inv_m, row,
-                                                                             coef, wsq, threshold_out);
+                                                                             coef, wsq, threshold_out, denom);
   return 1;
 }
 

@@ -86,6 +86,7 @@ extern "C" qasg_status qasg_quantize_pack_static(int device, const float* g, uin
   ws.part_cnt = reinterpret_cast<unsigned long long*>(s->scratch + kOffPartCnt);
   ws.part_max = reinterpret_cast<uint32_t*>(s->scratch + kOffPartMax);
   ws.counts = reinterpret_cast<unsigned long long*>(s->scratch + kOffCounts);
+  ws.selected = nullptr;  // sparse selection is not offered by this entry point
   ws.thresholds = reinterpret_cast<float*>(s->scratch + kOffThresholds);
   ws.scales = reinterpret_cast<float*>(s->scratch + kOffScales);
   ws.ticket = reinterpret_cast<unsigned int*>(s->scratch + kOffTicket);

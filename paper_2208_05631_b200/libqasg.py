@@ -26,9 +26,10 @@ EXPORTS = [
     "qasg_cmd_step", "qasg_rda_step", "qasg_step", "qasg_step_host", "qasg_logreg_grad_dense",
     "qasg_logreg_grad_csr", "qasg_last_async_status", "qasg_launch_count", "qasg_status_string",
     "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static", "qasg_requantize", "qasg_step_double",
+    "qasg_select_quantize_pack", "qasg_indicator_or", "qasg_step_select",
 ]
 STATIC_MAX_WORKERS = 16
-KERNEL_COUNT = 16
+KERNEL_COUNT = 24
 
 
 class QasgError(RuntimeError):
@@ -72,6 +73,11 @@ def load():
     lib.qasg_step.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp]
     lib.qasg_requantize.argtypes = [vp, vp, vp, u64, u32, u64, pp, vp, vp, vp, vp, vp]
     lib.qasg_step_double.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.qasg_select_quantize_pack.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                              vp, vp]
+    lib.qasg_indicator_or.argtypes = [vp, vp, u64, u32, vp, vp, vp]
+    lib.qasg_step_select.argtypes = [vp, i32, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                     vp]
     lib.qasg_step_host.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.qasg_logreg_grad_dense.argtypes = [vp, vp, vp, u64, u64, u32, ctypes.POINTER(u64), vp, u32, u64,
                                            vp, vp, u64, vp]
@@ -173,6 +179,25 @@ class Context:
         _check(load().qasg_step_double(self._h, rule, _ptr(g), d, ld_g, M, t, ctypes.byref(params), _ptr(x),
                                        _ptr(h), _ptr(z), _ptr(codes_out), _ptr(scales_out), _ptr(qcodes_out),
                                        _ptr(qscale_out), _stream(stream)), "qasg_step_double")
+
+    def select_quantize_pack(self, rule, g, d, ld_g, M, t, params, x, h, z, codes, scales, thresholds=None,
+                             counts=None, indicators=None, selected=None, stream=None):
+        _check(load().qasg_select_quantize_pack(self._h, rule, _ptr(g), d, ld_g, M, t, ctypes.byref(params),
+                                                _ptr(x), _ptr(h), _ptr(z), _ptr(codes), _ptr(scales),
+                                                _ptr(thresholds), _ptr(counts), _ptr(indicators), _ptr(selected),
+                                                _stream(stream)), "qasg_select_quantize_pack")
+
+    def indicator_or(self, indicators, d, M, isyn, ksyn, stream=None):
+        _check(load().qasg_indicator_or(self._h, _ptr(indicators), d, M, _ptr(isyn), _ptr(ksyn), _stream(stream)),
+               "qasg_indicator_or")
+
+    def step_select(self, rule, double_quant, g, d, ld_g, M, t, params, x, h, z=None, codes_out=None,
+                    scales_out=None, indicators_out=None, selected_out=None, isyn_out=None, ksyn_out=None,
+                    stream=None):
+        _check(load().qasg_step_select(self._h, rule, int(bool(double_quant)), _ptr(g), d, ld_g, M, t,
+                                       ctypes.byref(params), _ptr(x), _ptr(h), _ptr(z), _ptr(codes_out),
+                                       _ptr(scales_out), _ptr(indicators_out), _ptr(selected_out), _ptr(isyn_out),
+                                       _ptr(ksyn_out), _stream(stream)), "qasg_step_select")
 
     def step_host(self, rule, g_host, d, ld_g, M, t, params, x_host, h_host, z_host, g_dev, x_dev, h_dev,
                   z_dev, stream=None):
