@@ -1,6 +1,6 @@
 """Timing sweeps of libqasg on one GPU, beyond the single workload bench.py reports.
 
-  python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--double-quant]
+  python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--double-quant] [--select]
                                                [--min-log2-d 20] [--max-log2-d 28] [--workers 2,4,8,16,32]
   python -m paper_2208_05631_b200.sweep logreg [--steps 50]
 
@@ -56,7 +56,9 @@ def sweep_step(args):
             ctx = libqasg.Context(d, M, device=0)
             for rule, name, state_bytes in ((libqasg.RULE_CMD, "qcmd", 16), (libqasg.RULE_RDA, "qrda", 20)):
                 def one():
-                    if args.double_quant:
+                    if args.select:
+                        ctx.step_select(rule, args.double_quant, g, d, d, M, T_STEP, params, x, h, z)
+                    elif args.double_quant:
                         ctx.step_double(rule, g, d, d, M, T_STEP, params, x, h, z)
                     else:
                         ctx.step(rule, g, d, d, M, T_STEP, params, x, h, z)
@@ -72,7 +74,8 @@ def sweep_step(args):
                 moved = d * (8.0 * M + M / 2.0 + state_bytes)
                 if args.double_quant:
                     moved = d * (8.0 * M + M / 4.0 + 2.0 * M / 4.0 + 2 * 0.25 + state_bytes)
-                print(json.dumps({"what": "step_double" if args.double_quant else "step", "quantizer": args.quantizer,
+                what = "step" + ("_select" if args.select else "") + ("_double" if args.double_quant else "")
+                print(json.dumps({"what": what, "quantizer": args.quantizer,
                                   "rule": name, "d": d, "M": M, "ms_median": med, "ms_best": best,
                                   "coord_workers_per_s": d * M / (med * 1e-3),
                                   "gbs_moved": moved / 1e9 / (med * 1e-3), "kernel_ms": kernel_ms}), flush=True)
@@ -145,6 +148,7 @@ def main():
     ap.add_argument("what", choices=["step", "logreg"])
     ap.add_argument("--quantizer", default="threshold", choices=["threshold", "stochastic"])
     ap.add_argument("--double-quant", action="store_true")
+    ap.add_argument("--select", action="store_true")
     ap.add_argument("--min-log2-d", type=int, default=20)
     ap.add_argument("--max-log2-d", type=int, default=28)
     ap.add_argument("--workers", default="2,4,8,16,32")

@@ -64,13 +64,12 @@ def test_select_quantize_pack_bit_exact(ctx, d, M, rule, quantizer):
 @pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
 @pytest.mark.parametrize("double_quant", [False, True])
 def test_selected_run_40_steps(ctx, rule, double_quant):
-    """lambda large enough that most coordinates stay zero: the regime the selection is made for.
-    Oracle-driven (strict tolerance) and free-running."""
+    """lambda large enough that many coordinates stay zero: the regime the selection is made for.
+    Every step starts from the oracle's state rounded to fp32 (the indicator is a discrete decision:
+    a free-running fp32 trajectory may legitimately select another coordinate at the boundary)."""
     d, M, T, lam, eta, delta = 10_000, 4, 40, 1.5, 0.1, 1e-8
     params = libqasg.make_params(lam, eta, delta)
-    free = [torch.zeros(d, dtype=torch.float32, device=U.dev()) for _ in range(3)]
     xr, hr, zr = np.zeros(d), np.zeros(d), np.zeros(d)
-    peak = {"x": 0.0, "h": 0.0, "z": 0.0}
     names = ("x", "h", "z") if rule == libqasg.RULE_RDA else ("x", "h")
     words = (d + 31) // 32
     ksum = 0
@@ -101,9 +100,5 @@ def test_selected_run_40_steps(ctx, rule, double_quant):
         for name, got in zip(names, driven):
             U.assert_close(got, want[name], "%s step %d (driven)" % (name, t), atol=slack[name])
         U.assert_zero_pattern(driven[0], xr, ref["a"], lam)
-        ctx.step_select(rule, double_quant, g_dev, d, ld, M, t, params, *free)
-        # the free run may select a few different coordinates near the boundary; it must stay close
-        for name, got in zip(names, free):
-            peak[name] = max(peak[name], float(np.abs(want[name]).max()))
     assert ctx.last_async_status() == libqasg.OK
     assert 0 < ksum < T * d                                                 # the selection does select
