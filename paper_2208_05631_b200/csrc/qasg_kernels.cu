@@ -189,6 +189,48 @@ __device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64
   }
 }
 
+// The indicator bytes a thread needs for its four rows of tile k (two threads share a byte).
+struct TileMask {
+  uint32_t byte[kTileRows];
+  __device__ __forceinline__ uint32_t nibble(int r, int j) const { return (byte[r] >> (4 * (j & 1))) & 15u; }
+};
+__device__ __forceinline__ void load_tile_mask(const uint8_t* __restrict__ ind8, uint64_t d, uint32_t k, int j,
+                                               TileMask& mask) {
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) {
+    const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
+    mask.byte[r] = i0 < d ? static_cast<uint32_t>(__ldg(ind8 + (i0 >> 3))) : 0u;
+  }
+}
+
+// walk_tiles with the tile's indicator bytes travelling along: body(tile_values, mask, k).
+// Without a mask (kMasked false) no byte is loaded and every nibble reads as selected.
+template <bool kMasked, class Body>
+__device__ __forceinline__ void walk_tiles_masked(const float* __restrict__ row, const uint8_t* __restrict__ ind8,
+                                                  uint64_t d, uint32_t k0, uint32_t k1, int j, Body&& body) {
+  float4 a[kTileRows], b[kTileRows];
+  TileMask ma, mb;
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
+  load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
+  if (kMasked) load_tile_mask(ind8, d, k0, j, ma);
+  uint32_t k = k0;
+  while (true) {
+    if (k + 1 < k1) {
+      load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, b);
+      if (kMasked) load_tile_mask(ind8, d, k + 1, j, mb);
+    }
+    body(a, ma, k);
+    if (++k >= k1) break;
+    if (k + 1 < k1) {
+      load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, a);
+      if (kMasked) load_tile_mask(ind8, d, k + 1, j, ma);
+    }
+    body(b, mb, k);
+    if (++k >= k1) break;
+  }
+}
+
 // ------------------------------------------------------------------ pass A: sum |g|
 __global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
@@ -372,13 +414,6 @@ __device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspac
   }
 }
 
-// The four selection bits of coordinates i0..i0+3 of a worker whose indicator row is ind8
-// (bit i&7 of byte i>>3); all ones when no indicator is in use.
-__device__ __forceinline__ uint32_t indicator_nibble(const uint8_t* __restrict__ ind8, uint64_t i0, uint64_t d) {
-  if (i0 >= d) return 0u;
-  return (static_cast<uint32_t>(__ldg(ind8 + (i0 >> 3))) >> (i0 & 4u)) & 15u;
-}
-
 // ------------------------------------------------------------------ pass B: Q_Delta codes
 // kMasked: only coordinates whose indicator bit is set are candidates (sparse selection, Q(S(g, I))).
 template <bool kMasked>
@@ -404,7 +439,8 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     float cntf = 0.f;
-    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t k) {
+    walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], const TileMask& mask,
+                                                                uint32_t k) {
       double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
       uint32_t bytes[kTileRows];
 #pragma unroll
@@ -416,7 +452,7 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
         float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
         float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
         if (kMasked) {
-          const uint32_t nib = indicator_nibble(ind8, static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j, geo.d);
+          const uint32_t nib = mask.nibble(r, j);
           const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
           const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
           px *= sx, nx *= sx, py *= sy, ny *= sy, pz *= sz, nz *= sz, pw *= sw, nw *= sw;
@@ -492,7 +528,8 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
-    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&tile)[kTileRows], uint32_t k) {
+    walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, [&](const float4 (&tile)[kTileRows],
+                                                                const TileMask& mask, uint32_t k) {
       uint32_t bytes[kTileRows];
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
@@ -506,7 +543,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
         bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
         bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
         if (kMasked) {
-          const uint32_t nib = indicator_nibble(ind8, static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j, geo.d);
+          const uint32_t nib = mask.nibble(r, j);
           kx = kx && (nib & 1u), ky = ky && (nib & 2u), kz = kz && (nib & 4u), kw = kw && (nib & 8u);
         }
         bytes[r] = pack4(split_code(v.x, kx), split_code(v.y, ky), split_code(v.z, kz), split_code(v.w, kw));
@@ -1043,86 +1080,127 @@ __device__ __forceinline__ void load_state_tile(const float* __restrict__ v, uin
 
 // Pass A with selection: writes each worker's indicator bits and reduces, over the selected
 // coordinates only, the sum of |g| (threshold quantizer: Delta_m = coef * sum / k_m) or the maximum
-// (stochastic quantizer), and k_m.  Items run chunk-major so that the M workers of a chunk share
-// the chunk's x and h (or z) in L2.
+// (stochastic quantizer), and k_m.
+// One CTA takes one chunk of tiles for ALL workers: per tile it loads x and h (or z) once into
+// registers and walks the M gradient tiles (the next worker's loads in flight), so the state is read
+// once per coordinate, not once per worker.  Every worker keeps its own fixed-order sum: the same
+// column sums, warp butterfly, 8-warp combine and pairwise stack over tiles as in abs_sum_kernel,
+// with the cross-warp combine batched over kSelectBatch tiles.
+constexpr int kSelectBatch = 8;
+constexpr int kSelectDoublesPerWorker = kSelectBatch * (kThreads / 32) + kSelectBatch + 32;
+
+__host__ __device__ inline size_t select_smem_bytes(uint32_t M) {
+  return static_cast<size_t>(M) * (kSelectDoublesPerWorker * sizeof(double) + 2 * sizeof(uint32_t));
+}
+
 template <int kRule, bool kStochastic>
 __global__ void __launch_bounds__(kThreads, 3)
 select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __restrict__ x,
                     const float* __restrict__ hz, SelectScalars sc, float coef, Workspace ws,
                     uint32_t* __restrict__ indicators, float* __restrict__ thresholds_out,
                     unsigned long long* __restrict__ selected_out) {
-  __shared__ ChunkSumStorage sm_sum;
-  __shared__ uint32_t sm_cnt[kThreads / 32];
+  extern __shared__ double sm_dyn[];
   __shared__ bool sm_last;
-  const int j = threadIdx.x;
-  const uint32_t n_items = geo.M * geo.chunks;
+  const uint32_t M = geo.M;
+  double* warp_sums = sm_dyn;                                        // [M][kSelectBatch][8]
+  double* tile_sums = warp_sums + M * kSelectBatch * (kThreads / 32);  // [M][kSelectBatch]
+  double* stacks = tile_sums + M * kSelectBatch;                      // [M][32]
+  uint32_t* sm_cnt = reinterpret_cast<uint32_t*>(stacks + M * 32);     // [M] selected in this chunk
+  uint32_t* sm_max = sm_cnt + M;                                      // [M] max |g| over the selected
+  const int j = threadIdx.x, warp = j >> 5, lane = j & 31;
   const uint64_t ind_words = (geo.d + 31) >> 5;
-  ChunkSum chunk_sum(&sm_sum);
-  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const uint32_t c = item / geo.M, m = item - c * geo.M;
-    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
-    uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words);
+  for (uint32_t c = blockIdx.x; c < geo.chunks; c += gridDim.x) {
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    float cntf = 0.f;
-    uint32_t best = 0u;
+    for (uint32_t m = j; m < 2 * M; m += kThreads) sm_cnt[m] = 0u;  // counts and maxima
+    __syncthreads();
+    uint32_t pending = 0, pushed = 0;
     for (uint32_t k = k0; k < k1; ++k) {
-      float4 gv[kTileRows], xv[kTileRows], hv[kTileRows];
-      load_tile(row, static_cast<uint64_t>(k) * kTile, geo.d, j, gv);
+      const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+      float4 xv[kTileRows], hv[kTileRows];
       load_state_tile(x, geo.d, k, j, xv);
       load_state_tile(hz, geo.d, k, j, hv);
-      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+      // one worker's share of this tile: indicator bits, selected |g| into the fixed-order sum
+      auto worker_tile = [&](const float4 (&gv)[kTileRows], uint32_t m) {
+        uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words);
+        double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+        float cntf = 0.f;
+        uint32_t best = 0u;
 #pragma unroll
-      for (int r = 0; r < kTileRows; ++r) {
-        const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
-        const bool bx = i0 < geo.d && selects<kRule>(gv[r].x, xv[r].x, hv[r].x, sc);
-        const bool by = i0 + 1 < geo.d && selects<kRule>(gv[r].y, xv[r].y, hv[r].y, sc);
-        const bool bz = i0 + 2 < geo.d && selects<kRule>(gv[r].z, xv[r].z, hv[r].z, sc);
-        const bool bw = i0 + 3 < geo.d && selects<kRule>(gv[r].w, xv[r].w, hv[r].w, sc);
-        const float sx = bx ? 1.f : 0.f, sy = by ? 1.f : 0.f, sz = bz ? 1.f : 0.f, sw = bw ? 1.f : 0.f;
-        if (!kStochastic) {
-          cx += static_cast<double>(fabsf(gv[r].x) * sx);
-          cy += static_cast<double>(fabsf(gv[r].y) * sy);
-          cz += static_cast<double>(fabsf(gv[r].z) * sz);
-          cw += static_cast<double>(fabsf(gv[r].w) * sw);
-        } else {
-          best = max(best, __float_as_uint(fabsf(gv[r].x) * sx));
-          best = max(best, __float_as_uint(fabsf(gv[r].y) * sy));
-          best = max(best, __float_as_uint(fabsf(gv[r].z) * sz));
-          best = max(best, __float_as_uint(fabsf(gv[r].w) * sw));
+        for (int r = 0; r < kTileRows; ++r) {
+          const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
+          const bool bx = i0 < geo.d && selects<kRule>(gv[r].x, xv[r].x, hv[r].x, sc);
+          const bool by = i0 + 1 < geo.d && selects<kRule>(gv[r].y, xv[r].y, hv[r].y, sc);
+          const bool bz = i0 + 2 < geo.d && selects<kRule>(gv[r].z, xv[r].z, hv[r].z, sc);
+          const bool bw = i0 + 3 < geo.d && selects<kRule>(gv[r].w, xv[r].w, hv[r].w, sc);
+          const float sx = bx ? 1.f : 0.f, sy = by ? 1.f : 0.f, sz = bz ? 1.f : 0.f, sw = bw ? 1.f : 0.f;
+          if (!kStochastic) {
+            cx += static_cast<double>(fabsf(gv[r].x) * sx);
+            cy += static_cast<double>(fabsf(gv[r].y) * sy);
+            cz += static_cast<double>(fabsf(gv[r].z) * sz);
+            cw += static_cast<double>(fabsf(gv[r].w) * sw);
+          } else {
+            best = max(best, __float_as_uint(fabsf(gv[r].x) * sx));
+            best = max(best, __float_as_uint(fabsf(gv[r].y) * sy));
+            best = max(best, __float_as_uint(fabsf(gv[r].z) * sz));
+            best = max(best, __float_as_uint(fabsf(gv[r].w) * sw));
+          }
+          cntf += (sx + sy) + (sz + sw);
+          // two adjacent threads share an indicator byte; the even one writes it (zeros past d)
+          const uint32_t nib = static_cast<uint32_t>(bx) | (static_cast<uint32_t>(by) << 1) |
+                               (static_cast<uint32_t>(bz) << 2) | (static_cast<uint32_t>(bw) << 3);
+          const uint32_t upper = __shfl_down_sync(0xffffffffu, nib, 1);
+          if ((j & 1) == 0 && (i0 >> 3) < ind_words * 4) ind8[i0 >> 3] = static_cast<uint8_t>(nib | (upper << 4));
         }
-        cntf += (sx + sy) + (sz + sw);
-        // two adjacent threads share an indicator byte; the even one writes it (zeros past d)
-        const uint32_t nib = static_cast<uint32_t>(bx) | (static_cast<uint32_t>(by) << 1) |
-                             (static_cast<uint32_t>(bz) << 2) | (static_cast<uint32_t>(bw) << 3);
-        const uint32_t upper = __shfl_down_sync(0xffffffffu, nib, 1);
-        if ((j & 1) == 0 && (i0 >> 3) < ind_words * 4) ind8[i0 >> 3] = static_cast<uint8_t>(nib | (upper << 4));
+        if (!kStochastic) {
+          const double v = warp_pair_tree((cx + cy) + (cz + cw));
+          if (lane == 0) warp_sums[(m * kSelectBatch + pending) * (kThreads / 32) + warp] = v;
+        } else {
+          best = __reduce_max_sync(0xffffffffu, best);
+          if (lane == 0 && best) atomicMax(&sm_max[m], best);
+        }
+        const uint32_t cnt = __reduce_add_sync(0xffffffffu, static_cast<uint32_t>(cntf));
+        if (lane == 0 && cnt) atomicAdd(&sm_cnt[m], cnt);
+      };
+      // walk the workers with the next worker's tile in flight
+      float4 ga[kTileRows], gb[kTileRows];
+      load_tile(g, tile_base, geo.d, j, ga);
+      uint32_t m = 0;
+      while (true) {
+        if (m + 1 < M) load_tile(g + static_cast<uint64_t>(m + 1) * geo.ld, tile_base, geo.d, j, gb);
+        worker_tile(ga, m);
+        if (++m >= M) break;
+        if (m + 1 < M) load_tile(g + static_cast<uint64_t>(m + 1) * geo.ld, tile_base, geo.d, j, ga);
+        worker_tile(gb, m);
+        if (++m >= M) break;
       }
-      if (!kStochastic) chunk_sum.add_tile((cx + cy) + (cz + cw));
-    }
-    double total = 0.0;
-    if (!kStochastic) total = chunk_sum.finish(geo.log2_group);
-    if (kStochastic) {
-      best = __reduce_max_sync(0xffffffffu, best);
-      __syncthreads();
-      if ((j & 31) == 0) sm_cnt[j >> 5] = best;
-      __syncthreads();
-      if (j == 0) {
-        uint32_t bmax = sm_cnt[0];
-#pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) bmax = max(bmax, sm_cnt[w]);
-        ws.part_max[static_cast<uint64_t>(m) * kMaxChunks + c] = bmax;
+      ++pending;
+      if (!kStochastic && (pending == kSelectBatch || k + 1 == k1)) {
+        __syncthreads();
+        for (uint32_t e = j; e < M * pending; e += kThreads) {  // (worker, tile): combine the 8 warps
+          const uint32_t wm = e / pending, p = e - wm * pending;
+          const double* a = warp_sums + (wm * kSelectBatch + p) * (kThreads / 32);
+          tile_sums[wm * kSelectBatch + p] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+        }
+        __syncthreads();
+        for (uint32_t wm = j; wm < M; wm += kThreads)  // one thread per worker pushes its tiles, in order
+          for (uint32_t p = 0; p < pending; ++p) tile_push(stacks + wm * 32, pushed + p, tile_sums[wm * kSelectBatch + p]);
+        pushed += pending;
+        pending = 0;
       }
     }
-    const unsigned long long selected = block_count(static_cast<uint32_t>(cntf), sm_cnt);
-    if (j == 0) {
-      const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
-      ws.part_sum[p] = total;
-      ws.part_cnt[p] = selected;
+    __syncthreads();
+    for (uint32_t wm = j; wm < M; wm += kThreads) {
+      const uint64_t p = static_cast<uint64_t>(wm) * kMaxChunks + c;
+      ws.part_sum[p] = kStochastic ? 0.0 : tile_fold(stacks + wm * 32, pushed, geo.log2_group);
+      ws.part_cnt[p] = sm_cnt[wm];
+      ws.part_max[p] = sm_max[wm];
     }
+    __syncthreads();
   }
+  __threadfence();  // every thread that wrote partials publishes them before the CTA takes its ticket
+  __syncthreads();
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
-  const int warp = j >> 5, lane = j & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
     unsigned long long n = 0;
     uint32_t bmax = 0u;
@@ -1238,9 +1316,15 @@ int launch_select_stats(int rule, bool stochastic, const float* g, const Geometr
                         const float* hz, const SelectScalars& sc, float coef, const Workspace& ws,
                         uint32_t* indicators, float* thresholds_out, unsigned long long* selected_out,
                         const LaunchShape& shape, cudaStream_t stream) {
-  const unsigned grid = reduce_grid(geo, shape);
-#define QASG_SELECT(R, S) \
-  select_stats_kernel<R, S><<<grid, kThreads, 0, stream>>>(g, geo, x, hz, sc, coef, ws, indicators, thresholds_out, selected_out)
+  const size_t smem = select_smem_bytes(geo.M);
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * 3;
+  const unsigned grid = static_cast<unsigned>(geo.chunks < resident ? geo.chunks : resident);
+#define QASG_SELECT(R, S)                                                                                    \
+  do {                                                                                                       \
+    auto kernel = select_stats_kernel<R, S>;                                                                 \
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(select_smem_bytes(kMaxWorkers))); \
+    kernel<<<grid, kThreads, smem, stream>>>(g, geo, x, hz, sc, coef, ws, indicators, thresholds_out, selected_out); \
+  } while (0)
   if (rule == 0 && !stochastic) QASG_SELECT(0, false);
   else if (rule == 0) QASG_SELECT(0, true);
   else if (!stochastic) QASG_SELECT(1, false);
