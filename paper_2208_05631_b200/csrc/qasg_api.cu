@@ -92,6 +92,11 @@ qasg_status enter(const qasg_ctx* ctx) {
 
 qasg_status leave() { return cudaGetLastError() == cudaSuccess ? QASG_OK : QASG_ERR_CUDA; }
 
+// About four rounds of resident CTAs: enough items to balance the launch.
+uint32_t target_items(const qasg_ctx* ctx) {
+  return static_cast<uint32_t>(ctx->shape.sm_count * ctx->shape.reduce_ctas_per_sm * 4);
+}
+
 StepScalars scalars(const qasg_params* p, uint64_t t) {
   StepScalars sc;
   sc.lambda = p->lambda;
@@ -106,7 +111,7 @@ StepScalars scalars(const qasg_params* p, uint64_t t) {
 void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint64_t t,
                    const qasg_params* p, uint32_t* codes, float* scales, float* thresholds,
                    uint64_t* counts, cudaStream_t stream) {
-  const Geometry geo = make_geometry(d, ld_g, M);
+  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
   if (p->quantizer == QASG_Q_THRESHOLD) {
     { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream); }
@@ -136,7 +141,7 @@ void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint6
       Launch l(ctx, kDecodeAverage, stream);
       l += launch_decode_average(codes, scales, d, M, gbar, ctx->ws.status, ctx->shape, stream);
     }
-    const Geometry row = make_geometry(d, ld, 1);
+    const Geometry row = make_geometry(d, ld, 1, kMaxChunks, target_items(ctx));
     if (!stochastic) {
       { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(gbar, row, p->thr_coef, ctx->wsq, qthreshold, ctx->shape, stream, denom); }
       { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(gbar, row, ctx->wsq, qcodes, qscale, count_out, ctx->shape, stream); }
@@ -164,7 +169,7 @@ void select_quantize_pack(qasg_ctx* ctx, int rule, const float* g, uint64_t d, u
                           const qasg_params* p, const float* x, const float* h, const float* z, uint32_t* codes,
                           float* scales, float* thresholds, uint64_t* counts, uint32_t* indicators,
                           uint64_t* selected, cudaStream_t stream) {
-  const Geometry geo = make_geometry(d, ld_g, M);
+  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
   SelectScalars sc;
   sc.lambda_eta = p->lambda * p->eta;

@@ -33,7 +33,9 @@ struct Geometry {
   uint32_t chunks;  // ceil(tiles / group) <= kMaxChunks
 };
 
-Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks = kMaxChunks);
+// target_items > 0: prefer longer chunks as long as the launch keeps that many (worker, chunk) items.
+Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks = kMaxChunks,
+                       uint32_t target_items = 0);
 
 struct Workspace {
   double* part_sum;              // [M_max][kMaxChunks] chunk partials of a canonical sum

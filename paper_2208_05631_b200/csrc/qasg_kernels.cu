@@ -18,7 +18,7 @@
 namespace qasg {
 
 // ------------------------------------------------------------------ geometry
-Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks) {
+Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks, uint32_t target_items) {
   Geometry geo;
   geo.d = d;
   geo.ld = ld;
@@ -26,6 +26,13 @@ Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks)
   geo.tiles = static_cast<uint32_t>((d + kTile - 1) / kTile);
   uint32_t group = 1, lg = 0;
   while ((geo.tiles + group - 1) / group > max_chunks) {
+    group <<= 1;
+    ++lg;
+  }
+  // Longer chunks while there are still at least target_items of them in the launch: an item pays a
+  // CTA-wide combine and a partial write, which a single tile does not amortise.  Any aligned
+  // power-of-two grouping is a subtree of the same pairwise tree, so the sums do not change.
+  while (target_items && static_cast<uint64_t>(M) * ((geo.tiles + 2 * group - 1) / (2 * group)) >= target_items) {
     group <<= 1;
     ++lg;
   }
@@ -231,6 +238,71 @@ __device__ __forceinline__ void walk_tiles_masked(const float* __restrict__ row,
   }
 }
 
+// The CTA's whole share of a launch as one stream of tiles: items blockIdx.x, blockIdx.x + gridDim.x, ...
+// (item = worker m, chunk c), each a run of tiles.  The loads of the next tile are issued before the
+// current one is processed, across item boundaries too, so the memory pipeline never drains between
+// items (at small and medium d an item is only a few tiles long).
+//   begin(m, c)            before the first tile of an item
+//   body(values, mask, k)  every tile
+//   end(m, c, n_tiles)     after the last tile of an item (may synchronise the CTA)
+struct ItemPos {
+  uint32_t item, m, c, k0, k1;
+};
+__device__ __forceinline__ ItemPos item_pos(const Geometry& geo, uint32_t item) {
+  ItemPos p;
+  p.item = item;
+  p.m = item / geo.chunks;
+  p.c = item - p.m * geo.chunks;
+  p.k0 = p.c * geo.group;
+  p.k1 = min(p.k0 + geo.group, geo.tiles);
+  return p;
+}
+
+template <bool kMasked, class Begin, class Body, class End>
+__device__ __forceinline__ void stream_items(const float* __restrict__ g, const uint32_t* __restrict__ indicators,
+                                             const Geometry& geo, int j, Begin&& begin, Body&& body, End&& end) {
+  const uint32_t n_items = geo.M * geo.chunks;
+  if (blockIdx.x >= n_items) return;
+  const uint64_t ind_words = (geo.d + 31) >> 5;
+  ItemPos cur = item_pos(geo, blockIdx.x);
+  uint32_t k = cur.k0;
+  float4 a[kTileRows], b[kTileRows];
+  TileMask ma, mb;
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
+  auto load = [&](const ItemPos& p, uint32_t kk, float4 (&v)[kTileRows], TileMask& mk) {
+    load_tile(g + static_cast<uint64_t>(p.m) * geo.ld, static_cast<uint64_t>(kk) * kTile, geo.d, j, v);
+    if (kMasked)
+      load_tile_mask(reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(p.m) * ind_words), geo.d, kk, j, mk);
+  };
+  load(cur, k, a, ma);
+  begin(cur.m, cur.c);
+  auto step = [&](float4 (&cv)[kTileRows], TileMask& cm, float4 (&nv)[kTileRows], TileMask& nm) -> bool {
+    ItemPos nxt = cur;
+    uint32_t nk = k + 1;
+    bool has_next = true;
+    if (nk >= cur.k1) {
+      const uint32_t ni = cur.item + gridDim.x;
+      has_next = ni < n_items;
+      if (has_next) {
+        nxt = item_pos(geo, ni);
+        nk = nxt.k0;
+      }
+    }
+    if (has_next) load(nxt, nk, nv, nm);
+    body(cv, cm, k);
+    if (k + 1 >= cur.k1) {
+      end(cur.m, cur.c, cur.k1 - cur.k0);
+      if (has_next) begin(nxt.m, nxt.c);
+    }
+    cur = nxt;
+    k = nk;
+    return has_next;
+  };
+  while (step(a, ma, b, mb) && step(b, mb, a, ma)) {
+  }
+}
+
 // ------------------------------------------------------------------ pass A: sum |g|
 __global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
@@ -238,27 +310,24 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
   __shared__ ChunkSumStorage sm_sum;
   __shared__ bool sm_last;
   const int j = threadIdx.x;
-  const uint32_t n_items = geo.M * geo.chunks;
   ChunkSum chunk_sum(&sm_sum);
-  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
-    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
-    const uint32_t k0 = c * geo.group;
-    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t) {
-      double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
+  stream_items<false>(
+      g, nullptr, geo, j, [](uint32_t, uint32_t) {},
+      [&](const float4 (&v)[kTileRows], const TileMask&, uint32_t) {
+        double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
 #pragma unroll
-      for (int r = 1; r < kTileRows; ++r) {
-        cx += static_cast<double>(fabsf(v[r].x));
-        cy += static_cast<double>(fabsf(v[r].y));
-        cz += static_cast<double>(fabsf(v[r].z));
-        cw += static_cast<double>(fabsf(v[r].w));
-      }
-      chunk_sum.add_tile((cx + cy) + (cz + cw));
-    });
-    const double total = chunk_sum.finish(geo.log2_group);
-    if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
-  }
+        for (int r = 1; r < kTileRows; ++r) {
+          cx += static_cast<double>(fabsf(v[r].x));
+          cy += static_cast<double>(fabsf(v[r].y));
+          cz += static_cast<double>(fabsf(v[r].z));
+          cw += static_cast<double>(fabsf(v[r].w));
+        }
+        chunk_sum.add_tile((cx + cy) + (cz + cw));
+      },
+      [&](uint32_t m, uint32_t c, uint32_t) {
+        const double total = chunk_sum.finish(geo.log2_group);
+        if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
+      });
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   const int warp = j >> 5, lane = j & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
@@ -425,58 +494,57 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
-  const uint32_t n_items = geo.M * geo.chunks;
   const uint64_t row_words = (geo.d + 15) >> 4;
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
   ChunkSum chunk_sum(&sm_sum);
-  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
-    const float* row = g + static_cast<uint64_t>(m) * geo.ld;
-    uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
-    const float delta = ws.thresholds[m], ndelta = -delta;
-    const uint8_t* ind8 = kMasked ? reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5))
-                                  : nullptr;
-    const uint32_t k0 = c * geo.group;
-    const uint32_t k1 = min(k0 + geo.group, geo.tiles);
-    float cntf = 0.f;
-    walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], const TileMask& mask,
-                                                                uint32_t k) {
-      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
-      uint32_t bytes[kTileRows];
+  uint8_t* codes8 = nullptr;  // per item: the worker's code row, its threshold, the kept count so far
+  float delta = 0.f, ndelta = 0.f, cntf = 0.f;
+  stream_items<kMasked>(
+      g, indicators, geo, j,
+      [&](uint32_t m, uint32_t) {
+        codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
+        delta = ws.thresholds[m];
+        ndelta = -delta;
+        cntf = 0.f;
+      },
+      [&](const float4 (&v)[kTileRows], const TileMask& mask, uint32_t k) {
+        double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+        uint32_t bytes[kTileRows];
 #pragma unroll
-      for (int r = 0; r < kTileRows; ++r) {
-        const float4 t = v[r];
-        // strict comparisons; a NaN threshold or value compares false and codes 0
-        float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
-        float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
-        float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
-        float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
-        if (kMasked) {
-          const uint32_t nib = mask.nibble(r, j);
-          const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
-          const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
-          px *= sx, nx *= sx, py *= sy, ny *= sy, pz *= sz, nz *= sz, pw *= sw, nw *= sw;
+        for (int r = 0; r < kTileRows; ++r) {
+          const float4 t = v[r];
+          // strict comparisons; a NaN threshold or value compares false and codes 0
+          float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
+          float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
+          float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
+          float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+          if (kMasked) {
+            const uint32_t nib = mask.nibble(r, j);
+            const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
+            const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
+            px *= sx, nx *= sx, py *= sy, ny *= sy, pz *= sz, nz *= sz, pw *= sw, nw *= sw;
+          }
+          const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;  // 1.0f where kept
+          // |v| * 1 = |v| and |v| * 0 = +0: the kept magnitudes enter the sum unchanged
+          cx += static_cast<double>(fabsf(t.x) * kx);
+          cy += static_cast<double>(fabsf(t.y) * ky);
+          cz += static_cast<double>(fabsf(t.z) * kz);
+          cw += static_cast<double>(fabsf(t.w) * kw);
+          cntf += (kx + ky) + (kz + kw);  // exact: far below 2^24 per thread and chunk
+          bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
         }
-        const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;  // 1.0f where kept
-        // |v| * 1 = |v| and |v| * 0 = +0: the kept magnitudes enter the sum unchanged
-        cx += static_cast<double>(fabsf(t.x) * kx);
-        cy += static_cast<double>(fabsf(t.y) * ky);
-        cz += static_cast<double>(fabsf(t.z) * kz);
-        cw += static_cast<double>(fabsf(t.w) * kw);
-        cntf += (kx + ky) + (kz + kw);  // exact: far below 2^24 per thread and chunk
-        bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
-      }
-      store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
-      chunk_sum.add_tile((cx + cy) + (cz + cw));
-    });
-    const double picked = chunk_sum.finish(geo.log2_group);
-    const unsigned long long total = block_count(static_cast<uint32_t>(cntf), sm_cnt);
-    if (j == 0) {
-      const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
-      ws.part_sum[p] = picked;
-      ws.part_cnt[p] = total;
-    }
-  }
+        store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
+        chunk_sum.add_tile((cx + cy) + (cz + cw));
+      },
+      [&](uint32_t m, uint32_t c, uint32_t) {
+        const double picked = chunk_sum.finish(geo.log2_group);
+        const unsigned long long total = block_count(static_cast<uint32_t>(cntf), sm_cnt);
+        if (j == 0) {
+          const uint64_t p = static_cast<uint64_t>(m) * kMaxChunks + c;
+          ws.part_sum[p] = picked;
+          ws.part_cnt[p] = total;
+        }
+      });
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   finish_codes<true>(geo, ws, scales_out, counts_out);
   if (j == 0) *ws.ticket = 0u;
