@@ -2,7 +2,7 @@
 
   python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--double-quant] [--select]
                                                [--min-log2-d 20] [--max-log2-d 28] [--workers 2,4,8,16,32]
-  python -m paper_2208_05631_b200.sweep logreg [--steps 50]
+  python -m paper_2208_05631_b200.sweep logreg [--steps 50] [--graph]
 
 `step`   - the fused step over d in {2^20 .. 2^28} x M in {2, 4, 8, 16, 32} simulated workers,
            N(0,1) gradients, both update rules (the paper uses 2-4 workers; this is the scaling
@@ -11,6 +11,10 @@
 `logreg` - the two L1-logistic-regression workloads: gradient kernel + fused step per iteration.
            dense: X 65536 x 4096, 8 workers, minibatch 512; sparse: 10^6 x 2^24 CSR, ~80 non-zeros
            per row, 16 workers, minibatch 1024.
+
+`--graph` captures one iteration (fixed step index) in a CUDA graph and replays it: every call of the
+library only enqueues kernels on the given stream, so a launch-bound loop can be replayed without
+the host in the way.
 
 Prints one JSON line per measured point.  Every number is device time from CUDA events.
 """
@@ -85,6 +89,30 @@ def sweep_step(args):
             torch.cuda.empty_cache()
 
 
+def _timed_graph(it, warm, steps):
+    """Captures one call of `it` in a CUDA graph and times `steps` replays (device time per replay, us)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(warm):
+            it()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        it()
+    for _ in range(warm):
+        graph.replay()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        graph.replay()
+    stop.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(stop) * 1e3 / steps
+
+
 def _timed_iterations(ctx, it, warm, steps):
     for _ in range(warm):
         it()
@@ -118,8 +146,9 @@ def sweep_logreg(args):
             ctx.logreg_grad_dense(X, y, n, d, M, prob["shard_row0"], None, B, t[0], x, g, d)
             ctx.step(rule, g, d, d, M, t[0], params, x, h, z)
         us, kernel_us = _timed_iterations(ctx, it, 5, args.steps)
+        graph_us = _timed_graph(it, 3, args.steps) if args.graph else None
         print(json.dumps({"what": "logreg_dense", "rule": name, "n": n, "d": d, "M": M, "B": B,
-                          "us_per_iteration": us, "kernel_us": kernel_us,
+                          "us_per_iteration": us, "us_per_graph_replay": graph_us, "kernel_us": kernel_us,
                           "nnz_x": int((x != 0).sum().item())}), flush=True)
     del X, y
     # sparse: "sparse-feature logistic regression"
@@ -136,8 +165,10 @@ def sweep_logreg(args):
         ctx.logreg_grad_csr(*dev_args, n, d, M, prob["shard_row0"], None, B, t[0], x, g, d)
         ctx.step(libqasg.RULE_RDA, g, d, d, M, t[0], params, x, h, z)
     us, kernel_us = _timed_iterations(ctx, it_csr, 3, args.steps)
+    graph_us = _timed_graph(it_csr, 3, args.steps) if args.graph else None
     print(json.dumps({"what": "logreg_csr", "rule": "qrda", "n": n, "d": d, "M": M, "B": B,
-                      "nnz": int(prob["rowptr"][-1]), "us_per_iteration": us, "kernel_us": kernel_us,
+                      "nnz": int(prob["rowptr"][-1]), "us_per_iteration": us, "us_per_graph_replay": graph_us,
+                      "kernel_us": kernel_us,
                       "nnz_x": int((x != 0).sum().item())}), flush=True)
     assert ctx.last_async_status() == libqasg.OK
     ctx.close()
@@ -155,6 +186,7 @@ def main():
     ap.add_argument("--reps", type=int, default=7)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--csr-rows", type=int, default=1_000_000)
+    ap.add_argument("--graph", action="store_true")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "needs a CUDA device"
     if args.what == "step":
