@@ -712,7 +712,7 @@ __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes
                                                uint64_t grp, uint32_t& bad) {
   double q0 = 0.0, q1 = 0.0, q2 = 0.0, q3 = 0.0;
   const uint32_t m4 = kM4 > 0 ? static_cast<uint32_t>(kM4) : (M + 3) >> 2;
-  if (kLanes > 1) lut += threadIdx.x & 31;
+  if (kLanes > 1) lut += threadIdx.x & (kLanes - 1);  // kLanes copies: lanes l and l + kLanes share one
 #pragma unroll
   for (uint32_t G = 0; G < m4; ++G) {
     const uint8_t* p = codes8 + grp + static_cast<uint64_t>(4 * G) * row_bytes;
@@ -1445,14 +1445,20 @@ static void launch_decode_update_rule(const uint32_t* codes, const float* scales
   constexpr int kG = kRule == 1 ? 1 : 2;  // groups per thread with per-lane tables (measured best)
 #define QASG_LANE(m4) \
   case m4: launch_decode_update_as<kRule, m4, 32, 1024, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+#define QASG_LANES(m4, lanes) \
+  case m4: launch_decode_update_as<kRule, m4, lanes, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_SHARED(m4) \
   case m4: launch_decode_update_as<kRule, m4, 1, kThreads, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
   switch ((M + 3) / 4) {
     QASG_LANE(1) QASG_LANE(2) QASG_LANE(3)
-    QASG_SHARED(4) QASG_SHARED(5) QASG_SHARED(6) QASG_SHARED(7) QASG_SHARED(8) QASG_SHARED(9) QASG_SHARED(10)
-    QASG_SHARED(11) QASG_SHARED(12) QASG_SHARED(13) QASG_SHARED(14) QASG_SHARED(15) QASG_SHARED(16)
+    // 16 copies (32 KB per worker group) keep the two half-warps of a 64-bit lookup apart; 8 copies
+    // leave two lanes per copy
+    QASG_LANES(4, 16) QASG_LANES(5, 16) QASG_LANES(6, 16) QASG_LANES(7, 16)
+    QASG_LANES(8, 8) QASG_LANES(9, 8) QASG_LANES(10, 8) QASG_LANES(11, 8) QASG_LANES(12, 8) QASG_LANES(13, 8)
+    QASG_SHARED(14) QASG_SHARED(15) QASG_SHARED(16)
   }
 #undef QASG_LANE
+#undef QASG_LANES
 #undef QASG_SHARED
 }
 

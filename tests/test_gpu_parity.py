@@ -230,7 +230,7 @@ def test_sweep_one_step(ctx, d, M, rule):
     U.assert_zero_pattern(x, ref["x"], ref["a"], LAM)
 
 
-@pytest.mark.parametrize("M", [1, 5, 9, 12, 13, 31, 64])
+@pytest.mark.parametrize("M", [1, 5, 9, 12, 13, 16, 28, 31, 52, 53, 64])
 @pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
 def test_fused_step_worker_counts(ctx, M, rule):
     # every dispatch of the decode: per-lane tables (M <= 12), shared tables, short last group
