@@ -76,3 +76,39 @@ def test_full_size_step_against_the_oracle():
     U.assert_zero_pattern(xr[idx_t], x_ref, a, LAM)
     assert (x_ref == 0).any() and (x_ref != 0).any()
     ctx.close()
+
+
+def test_more_than_2_to_31_coordinates():
+    """One worker with d = 2^31 + 4099 coordinates: coordinate, byte and word indices pass 2^31 and the
+    row is longer than 2^33 bytes.  Threshold, scale, count and the complete code row are compared."""
+    try:
+        import psutil
+        if psutil.virtual_memory().available < 80 * 2 ** 30:
+            pytest.skip("needs 80 GB of host memory for the oracle")
+    except ImportError:
+        pass
+    if not torch.cuda.is_available() or torch.cuda.get_device_properties(0).total_memory < 40 * 2 ** 30:
+        pytest.skip("needs 40 GB of device memory")
+    d = (1 << 31) + 4099
+    ld = (d + 3) // 4 * 4
+    dev = U.dev()
+    g = inputs.normal_gradients(d, 1, seed=6, device=dev, ld=ld)
+    ctx = libqasg.Context(d, 1, device=0, flags=libqasg.CREATE_NO_CODE_SCRATCH)
+    codes = torch.zeros((1, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+    scales = torch.zeros(1, dtype=torch.float32, device=dev)
+    thr = torch.zeros(1, dtype=torch.float32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+    ctx.quantize_pack(g, d, ld, 1, 1, libqasg.make_params(), codes, scales, thr, cnt)
+    assert ctx.last_async_status() == libqasg.OK
+    row = g[0, :d].cpu().numpy()
+    del g
+    tern, s, delta, n = O.threshold_quantize(row)
+    del row
+    assert thr.cpu().numpy()[0].view(np.uint32) == np.float32(delta).view(np.uint32)
+    assert scales.cpu().numpy()[0].view(np.uint32) == np.float32(s).view(np.uint32)
+    assert int(cnt.cpu().numpy()[0]) == n
+    got = U.codes_np(codes[0])
+    half = (tern.size // 32) * 16          # pack in two pieces to bound the oracle's temporaries
+    assert np.array_equal(got[: half // 16], O.pack_codes(tern[:half]))
+    assert np.array_equal(got[half // 16:], O.pack_codes(tern[half:]))
+    ctx.close()
