@@ -169,7 +169,8 @@ void select_quantize_pack(qasg_ctx* ctx, int rule, const float* g, uint64_t d, u
                           const qasg_params* p, const float* x, const float* h, const float* z, uint32_t* codes,
                           float* scales, float* thresholds, uint64_t* counts, uint32_t* indicators,
                           uint64_t* selected, cudaStream_t stream) {
-  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
+  // the selection kernel's items are chunks (each for all M workers), not (worker, chunk) pairs
+  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx) * M);
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
   SelectScalars sc;
   sc.lambda_eta = p->lambda * p->eta;
