@@ -3,8 +3,10 @@
 //   pass A  abs_sum_kernel / abs_max_kernel     per-worker sum|g| -> Delta_m, or max|g| -> s_m
 //   pass B  threshold_codes_kernel              ternary codes, packed; s_m = mean of kept |g|
 //           stochastic_codes_kernel             unbiased ternary codes from Philox draws
-//   pass C  decode_update_kernel                decode + average + accumulator + QCMD/QRDA
-//           decode_average_kernel, dense_update_kernel   the same in two unfused halves
+//   pass C  decode_update_kernel                decode + average + accumulator + QCMD/QRDA (or the
+//                                               average alone), dense_update_kernel: update from a dense q
+//   server  avg_abs_sum/avg_abs_max/avg_codes   double quantization: Q applied to the average
+//   select  select_stats, indicator_or          sparse selection: indicators, statistics over the selected
 //
 // All three passes are HBM streams.  Passes A and B walk each worker's gradient in
 // 4096-coordinate tiles with 128-bit loads (thread j owns columns 4j..4j+3 of each of
