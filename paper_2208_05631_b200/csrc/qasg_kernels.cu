@@ -774,8 +774,8 @@ struct GroupState {
 
 // kThreadsC threads per CTA; a CTA takes kGroups * kThreadsC consecutive groups per round and a
 // thread owns kGroups of them, kThreadsC apart, with all their loads in flight before it decodes.
-// Up to 12 workers run with per-lane tables (1024 threads, one CTA per SM); more workers share
-// one table per CTA.
+// Up to 12 workers run with 16 copies of the tables (512 threads, two CTAs per SM); up to 52 with 16 or 8
+// copies and one CTA of 1024 threads per SM; more workers share one table per CTA.
 template <int kRule, int kM4, int kLanes, int kThreadsC, int kGroups>
 __global__ void __launch_bounds__(kThreadsC)
 decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
@@ -1445,8 +1445,9 @@ static void launch_decode_update_rule(const uint32_t* codes, const float* scales
                                       float* x, float* h, float* z, const StepScalars& sc,
                                       unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
   constexpr int kG = kRule == 1 ? 1 : 2;  // groups per thread with per-lane tables (measured best)
+  // up to 12 workers: 16 copies of the tables (conflict-free for 64-bit lookups), two CTAs of 512 threads per SM
 #define QASG_LANE(m4) \
-  case m4: launch_decode_update_as<kRule, m4, 32, 1024, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+  case m4: launch_decode_update_as<kRule, m4, 16, 512, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_LANES(m4, lanes) \
   case m4: launch_decode_update_as<kRule, m4, lanes, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_SHARED(m4) \
