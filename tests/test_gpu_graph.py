@@ -1,0 +1,48 @@
+"""qasg_step only enqueues kernels on the caller's stream (no allocation, no synchronisation), so a
+launch-bound loop can be captured once in a CUDA graph and replayed.  The replayed steps must give
+exactly the bits of eagerly launched ones."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2208_05631_b200 import inputs, libqasg
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
+def test_fused_step_replayed_from_a_cuda_graph(rule):
+    dev = torch.device("cuda:0")
+    d, M, t = 40_003, 8, 5
+    ld = (d + 3) // 4 * 4
+    g = torch.zeros((M, ld), dtype=torch.float32, device=dev)
+    g[:, :d] = torch.from_numpy(inputs.optimizer_only_gradients(d, M, t, seed=2) * np.float32(0.01)).to(dev)
+    x0, h0, z0 = inputs.random_state(d, seed=2, device=dev)
+    ctx = libqasg.Context(d, M, device=0)
+    params = libqasg.make_params(1e-3, 0.1, 1e-8)
+
+    eager = [v.clone() for v in (x0, h0, z0)]
+    for _ in range(3):
+        ctx.step(rule, g, d, ld, M, t, params, *eager)
+    torch.cuda.synchronize()
+
+    state = [v.clone() for v in (x0, h0, z0)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                      # warm-up outside the capture
+        warm = [v.clone() for v in (x0, h0, z0)]
+        ctx.step(rule, g, d, ld, M, t, params, *warm)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.step(rule, g, d, ld, M, t, params, *state)
+    for v, v0 in zip(state, (x0, h0, z0)):
+        v.copy_(v0)                                    # the capture itself ran nothing
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    for got, want in zip(state, eager):
+        assert torch.equal(got, want)
+    assert ctx.last_async_status() == libqasg.OK
+    ctx.close()
