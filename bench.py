@@ -50,9 +50,9 @@ def bytes_per_coord(M):
 # capture summarised in profiles/step_kernels_d2p24_M8_ncu_full.md (d = 2^24; passes A and B stream,
 # so their traffic grows in proportion to d).  Valid only for the kernel source it was taken from.
 NCU_TRAFFIC = {
-    "kernels_sha256": "69508b8e3c9a9d31d249b0c7c6369ee9718df3bbeadf7e7daa3b31d9dd44f82a",
+    "kernels_sha256": "83a54c4d6d39a070c9be4e79f2d1b36116cc1dd572ba02ae001d482fc53ae1d1",
     "M": 8,
-    "bytes_per_coord": {"abs_sum": 540701696 / 2 ** 24, "threshold_codes": 568721664 / 2 ** 24},
+    "bytes_per_coord": {"abs_sum": 540939776 / 2 ** 24, "threshold_codes": 568223232 / 2 ** 24},
 }
 
 
