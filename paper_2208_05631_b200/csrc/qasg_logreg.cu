@@ -59,19 +59,24 @@ logreg_dense_coef_kernel(const float* __restrict__ X, const float* __restrict__ 
   }
 }
 
-// grid (d/128, M); thread (cq = tid & 31 -> 4 columns, rl = tid >> 5 -> rows rl, rl+8, ...).
-__global__ void __launch_bounds__(kThreads)
+// grid (d/128, M), 1024 threads: thread (cq = tid & 31 -> 4 columns, rl = tid >> 5 -> rows rl, rl+32, ...).
+// The 32 row lanes are combined in lane order, so the result does not depend on timing.
+constexpr int kColsumThreads = 1024;
+__global__ void __launch_bounds__(kColsumThreads)
 logreg_dense_colsum_kernel(const float* __restrict__ X, uint64_t d, uint32_t B, const float* __restrict__ coef,
                            const uint32_t* __restrict__ rows, float* __restrict__ g, uint64_t ld_g) {
-  __shared__ float4 sm[kThreads / 32][32];
+  constexpr int kRowLanes = kColsumThreads / 32;
+  __shared__ float4 sm[kRowLanes][32];
   const uint32_t m = blockIdx.y, cq = threadIdx.x & 31, rl = threadIdx.x >> 5;
   const uint64_t col = (static_cast<uint64_t>(blockIdx.x) * 32 + cq) * 4;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   if (col < d) {
-    for (uint32_t b = rl; b < B; b += kThreads / 32) {
-      const float c = coef[static_cast<uint64_t>(m) * B + b];
-      const uint64_t r = rows[static_cast<uint64_t>(m) * B + b];
-      const float4 a = __ldg(reinterpret_cast<const float4*>(X + r * d + col));
+    const float* cm = coef + static_cast<uint64_t>(m) * B;
+    const uint32_t* rm = rows + static_cast<uint64_t>(m) * B;
+#pragma unroll 4
+    for (uint32_t b = rl; b < B; b += kRowLanes) {
+      const float c = cm[b];
+      const float4 a = __ldg(reinterpret_cast<const float4*>(X + static_cast<uint64_t>(rm[b]) * d + col));
       acc.x = fmaf(c, a.x, acc.x);
       acc.y = fmaf(c, a.y, acc.y);
       acc.z = fmaf(c, a.z, acc.z);
@@ -82,7 +87,7 @@ logreg_dense_colsum_kernel(const float* __restrict__ X, uint64_t d, uint32_t B, 
   __syncthreads();
   if (rl == 0 && col < d) {
 #pragma unroll
-    for (int k = 1; k < kThreads / 32; ++k) {
+    for (int k = 1; k < kRowLanes; ++k) {
       const float4 o = sm[k][cq];
       acc.x += o.x;
       acc.y += o.y;
@@ -128,7 +133,7 @@ int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
   const unsigned grid1 = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
   logreg_dense_coef_kernel<<<grid1, kThreads, 0, stream>>>(X, y, d, M, sh, batch_rows, B, t, x, coef_ws, rows_ws);
   const dim3 grid2(static_cast<unsigned>((d + 127) / 128), M);
-  logreg_dense_colsum_kernel<<<grid2, kThreads, 0, stream>>>(X, d, B, coef_ws, rows_ws, g, ld_g);
+  logreg_dense_colsum_kernel<<<grid2, kColsumThreads, 0, stream>>>(X, d, B, coef_ws, rows_ws, g, ld_g);
   return 2;
 }
 
