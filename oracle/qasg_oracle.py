@@ -317,24 +317,22 @@ def trial_update(rule, g_m, x, h, z, t, lam, eta, delta):
 
 
 def indicator(rule, g_m, x, h, z, t, lam, eta, delta):
-    """I_d = 1 if x_{t,d} != 0 or x_hat_{t+1,d} != 0 (Eq. of the indicator function), decided in fp32
-    by a fixed sequence of correctly rounded operations, each one its own rounding (no fused
-    multiply-add), so that every implementation takes the same decision:
+    """I_d = 1 if x_{t,d} != 0 or x_hat_{t+1,d} != 0 (Eq. of the indicator function), decided in fp32,
+    the precision of the data.  Where x_d != 0 the bit is set whatever the trial update gives, so
+    the trial update matters only where x_d = 0, and there its closed form reduces to:
 
-      QCMD:  x_hat != 0  <=>  |x*H_hat - eta*g| > lambda*eta,   H_hat = delta + sqrt(h + g*g)
-             (the closed form's test |x - eta*g/H_hat| > lambda*eta/H_hat multiplied by H_hat > 0)
-      QRDA:  x_hat != 0  <=>  |z + g| > lambda*t
+      QCMD:  x_hat = sign(-g) * (eta/H_hat) * [|g| - lambda]_+ , non-zero  <=>  |g| > lambda
+             (H_hat = delta + sqrt(h + g^2) > 0 scales both sides of the test and drops out)
+      QRDA:  x_hat != 0  <=>  |z + g| / t > lambda  <=>  |z + g| > lambda * t
+             (one fp32 addition and one fp32 product, each rounded once)
 
     Returns a bool vector."""
     f = F32
     g_m = np.asarray(g_m, dtype=F32)
     x = np.asarray(x, dtype=F32)
-    lam, eta, delta = f(lam), f(eta), f(delta)
+    lam = f(lam)
     if rule == RULE_CMD:
-        h = np.asarray(h, dtype=F32)
-        big_h = delta + np.sqrt(h + g_m * g_m)
-        lhs = np.abs(x * big_h - eta * g_m)
-        moved = lhs > lam * eta
+        moved = np.abs(g_m) > lam
     else:
         z = np.asarray(z, dtype=F32)
         moved = np.abs(z + g_m) > lam * f(int(t))
