@@ -170,12 +170,14 @@ qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint
  * function", "Quantize the selected elements of the gradients" Q(S(g, I)).
  * Worker m's indicator marks coordinate i when x_i != 0 or when the worker's local trial update,
  * taken with its own full-precision gradient and H_hat = delta + sqrt(h + g^2), leaves it non-zero.
- * The test is evaluated in fp32, every operation rounded on its own:
- *   QCMD: |x*H_hat - eta*g| > lambda*eta        QRDA: |z + g| > lambda*t
+ * Where x_i != 0 the bit is set whatever the trial gives; where x_i = 0 the closed form of the
+ * trial update is non-zero iff (fp32, every operation rounded on its own)
+ *   QCMD: |g| > lambda   (H_hat > 0 scales both sides and drops out)      QRDA: |z + g| > lambda*t
  * Only marked coordinates are quantized: Delta_m = thr_coef/k_m * sum over them of |g| (k_m of
  * them), the scale is the mean kept magnitude (stochastic quantizer: the maximum over them);
  * unmarked coordinates code 0.
- *   x, h, z     device, fp32 [d]: the current state (read only); h used by QCMD, z by QRDA.
+ *   x, h, z     device, fp32 [d]: the current state (read only).  z is read by QRDA only and may
+ *               be NULL for QCMD; h is read by neither test and may be NULL.
  *   indicators  device, uint32 [M][ceil(d/32)]: bit i&31 of word i>>5 of row m; unused bits 0.
  *   selected    device, uint64 [M] or NULL: k_m.  A worker's message is then 32 + d + 2*k_m bits
  *               (Section 3.5 "Encode").

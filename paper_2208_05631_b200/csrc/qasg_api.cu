@@ -173,9 +173,7 @@ void select_quantize_pack(qasg_ctx* ctx, int rule, const float* g, uint64_t d, u
   const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx) * M);
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
   SelectScalars sc;
-  sc.lambda_eta = p->lambda * p->eta;
-  sc.eta = p->eta;
-  sc.delta = p->delta;
+  sc.lambda = p->lambda;
   sc.lambda_t = p->lambda * static_cast<float>(t);
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
   {
@@ -424,7 +422,7 @@ qasg_status qasg_select_quantize_pack(qasg_ctx* ctx, qasg_rule rule, const float
   if (st != QASG_OK) return st;
   if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
   if (!x || !codes || !scales || !indicators || t < 1) return QASG_ERR_INVALID_ARG;
-  if ((rule == QASG_RULE_CMD && !h) || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (rule == QASG_RULE_RDA && !z) return QASG_ERR_INVALID_ARG;  // neither test reads h
   if (!aligned16(x) || (h && !aligned16(h)) || (z && !aligned16(z)) || !aligned16(codes) || !aligned16(indicators))
     return QASG_ERR_ALIGNMENT;
   if ((st = enter(ctx)) != QASG_OK) return st;

@@ -57,7 +57,7 @@ struct LaunchShape {
 
 // Constants of the indicator test, rounded to fp32 on the host: lambda*eta, lambda*t.
 struct SelectScalars {
-  float lambda_eta, eta, delta, lambda_t;
+  float lambda, lambda_t;  // QCMD compares |g| with lambda, QRDA |z + g| with lambda*t
 };
 
 struct StepScalars {

@@ -1114,25 +1114,26 @@ avg_codes_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ s
 
 // ------------------------------------------------------------------ sparse selection
 // Indicator of one coordinate of one worker (Section 3.2): x != 0, or the worker's local trial update
-// with its own gradient leaves the coordinate non-zero.  Decided in fp32 by correctly rounded
-// operations taken one by one (no fused multiply-add), so that the bit does not depend on who computes it:
-//   QCMD: |x*H - eta*g| > lambda*eta with H = delta + sqrt(h + g*g)   (hz = h)
-//   QRDA: |z + g| > lambda*t                                          (hz = z)
+// with its own gradient leaves the coordinate non-zero.  Where x != 0 the bit is set whatever the trial
+// gives; where x == 0 the closed form of the trial update is non-zero iff
+//   QCMD: |g| > lambda          (H_hat = delta + sqrt(h + g*g) > 0 scales both sides and drops out)
+//   QRDA: |z + g| > lambda*t    (hz = z; one correctly rounded addition, no fused multiply-add)
+// so one fp32 comparison decides the bit and it does not depend on who computes it.
 template <int kRule>
 __device__ __forceinline__ bool selects(float g, float x, float hz, const SelectScalars& sc) {
-  bool moved;
-  if (kRule == 0) {
-    const float big_h = __fadd_rn(sc.delta, __fsqrt_rn(__fadd_rn(hz, __fmul_rn(g, g))));
-    moved = fabsf(__fsub_rn(__fmul_rn(x, big_h), __fmul_rn(sc.eta, g))) > sc.lambda_eta;
-  } else {
-    moved = fabsf(__fadd_rn(hz, g)) > sc.lambda_t;
-  }
+  const bool moved = kRule == 0 ? fabsf(g) > sc.lambda : fabsf(__fadd_rn(hz, g)) > sc.lambda_t;
   return (x != 0.f) || moved;
 }
 
 // A thread's four float4 of tile k of a state vector of exactly d floats (no padding to read into).
 __device__ __forceinline__ void load_state_tile(const float* __restrict__ v, uint64_t d, uint32_t k, int j,
-                                                float4 (&out)[kTileRows]) {
+                                                bool whole, float4 (&out)[kTileRows]) {
+  if (whole) {  // the tile lies inside [0, d): no bounds tests
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r)
+      out[r] = load_f4(v + static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j);
+    return;
+  }
 #pragma unroll
   for (int r = 0; r < kTileRows; ++r) {
     const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
@@ -1187,9 +1188,15 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
     uint32_t pending = 0, pushed = 0;
     for (uint32_t k = k0; k < k1; ++k) {
       const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+      const bool whole = tile_base + kTile <= geo.d;
       float4 xv[kTileRows], hv[kTileRows];
-      load_state_tile(x, geo.d, k, j, xv);
-      load_state_tile(hz, geo.d, k, j, hv);
+      load_state_tile(x, geo.d, k, j, whole, xv);
+      if (kRule == 1) {
+        load_state_tile(hz, geo.d, k, j, whole, hv);
+      } else {  // the QCMD test reads no accumulator
+#pragma unroll
+        for (int r = 0; r < kTileRows; ++r) hv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
       // one worker's share of this tile: indicator bits, selected |g| into the fixed-order sum
       auto worker_tile = [&](const float4 (&gv)[kTileRows], uint32_t m) {
         uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words);
@@ -1199,10 +1206,10 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
 #pragma unroll
         for (int r = 0; r < kTileRows; ++r) {
           const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
-          const bool bx = i0 < geo.d && selects<kRule>(gv[r].x, xv[r].x, hv[r].x, sc);
-          const bool by = i0 + 1 < geo.d && selects<kRule>(gv[r].y, xv[r].y, hv[r].y, sc);
-          const bool bz = i0 + 2 < geo.d && selects<kRule>(gv[r].z, xv[r].z, hv[r].z, sc);
-          const bool bw = i0 + 3 < geo.d && selects<kRule>(gv[r].w, xv[r].w, hv[r].w, sc);
+          const bool bx = (whole || i0 < geo.d) && selects<kRule>(gv[r].x, xv[r].x, hv[r].x, sc);
+          const bool by = (whole || i0 + 1 < geo.d) && selects<kRule>(gv[r].y, xv[r].y, hv[r].y, sc);
+          const bool bz = (whole || i0 + 2 < geo.d) && selects<kRule>(gv[r].z, xv[r].z, hv[r].z, sc);
+          const bool bw = (whole || i0 + 3 < geo.d) && selects<kRule>(gv[r].w, xv[r].w, hv[r].w, sc);
           const float sx = bx ? 1.f : 0.f, sy = by ? 1.f : 0.f, sz = bz ? 1.f : 0.f, sw = bw ? 1.f : 0.f;
           if (!kStochastic) {
             cx += static_cast<double>(fabsf(gv[r].x) * sx);
