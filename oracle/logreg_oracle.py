@@ -83,6 +83,20 @@ def grad_workers_csr(rowptr, colidx, vals, y, shard_row0, batch, t, x, d, batch_
     return out
 
 
+def touched_columns(rowptr, colidx, shard_row0, batch, t, d, batch_ids=None):
+    """Which coordinates each worker's minibatch can make non-zero: column i is touched by
+    worker m when some row of its minibatch stores an entry in column i (Section 5.1: the
+    text data sets are sparse, so a minibatch gradient has few non-zero coordinates).  A
+    coordinate that is not touched has gradient exactly +0.0.  Returns bool [M, d]."""
+    m_workers = len(shard_row0) - 1
+    out = np.zeros((m_workers, int(d)), dtype=bool)
+    for m in range(m_workers):
+        rows = batch_rows(shard_row0, m, batch, t) if batch_ids is None else np.asarray(batch_ids[m])
+        for r in rows:
+            out[m, np.asarray(colidx[int(rowptr[r]):int(rowptr[r + 1])], dtype=np.int64)] = True
+    return out
+
+
 def objective(X, y, x, lam):
     """Full objective f(x) + lambda*||x||_1 over all rows (dense X), fp64."""
     s = np.asarray(X, dtype=F64) @ np.asarray(x, dtype=F64)

@@ -442,8 +442,21 @@ def quantize_workers(g, quantizer, t=1, seed=0, coef=0.75):
     return dict(terns=terns, scales=scales, thresholds=thresholds, counts=counts, codes=codes)
 
 
+def densify_touched(g, touched):
+    """A gradient held in sparse form: worker m stores only the entries its minibatch touched
+    (touched[m, i] True); every other entry IS +0.0, whatever the array g holds there.  The
+    quantizer and the update are those of the dense vector this returns (M x d, fp32): a zero
+    entry is inside [-Delta, Delta] and codes 0 (Section 3.4), adds nothing to sum|g| nor to
+    max|g|, and is kept with probability 0 by the stochastic quantizer."""
+    g = np.asarray(g, dtype=F32)
+    touched = np.asarray(touched, dtype=bool)
+    if touched.shape != g.shape:
+        raise ValueError("touched must have the shape of g")
+    return np.where(touched, g, F32(0.0)).astype(F32)
+
+
 def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0, coef=0.75,
-         double_quant=False, select=False):
+         double_quant=False, select=False, touched=None):
     """One iteration: quantize every worker's gradient, decode and average, update the
     accumulator and apply the rule's closed-form update.  State in, state out (fp64).
 
@@ -452,12 +465,17 @@ def step(rule, g, x, h, z, t, lam, eta, delta, quantizer=QUANT_THRESHOLD, seed=0
     select=True adds the sparse selection: each worker sends only the coordinates its indicator
     marks (and, with double_quant, the server quantizes only those of the synchronous indicator).
 
+    touched (bool M x d) marks the stored entries of sparse gradients: the step is that of
+    `densify_touched(g, touched)`.
+
     quantizer == QUANT_NONE skips quantization: q is the fp64 mean of the rows of g
     (the 32-bit CMD / RDA adagrad baseline).
     Returns dict(x, h, z, a, q, quant) where `a` is the quantity compared with lambda
     and `quant` the output of `quantize_workers` (None without quantization).
     """
     g = np.asarray(g, dtype=F32)
+    if touched is not None:
+        g = densify_touched(g, touched)
     if quantizer == QUANT_NONE:
         quant = None
         q = g.astype(F64).sum(axis=0) / F64(g.shape[0])

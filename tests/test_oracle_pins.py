@@ -509,3 +509,33 @@ def test_indicator_words_or_and_sparse_bit_budget():
     k = int(out["selected"][0])
     assert O.sparse_wire_bits(d, k) == 32 + d + 2 * k
     assert (O.sparse_wire_bits(d, k) < O.wire_bits(d)) == (k < d / 2)         # cheaper iff k < d/2
+
+
+# ------------------------------------------------------------------ sparse (touched) gradients
+def test_touched_step_is_the_dense_step_of_the_stored_entries():
+    """Entries a worker does not store are +0.0 by definition: whatever the array holds there is
+    ignored, they code 0 under both quantizers, and the threshold is 0.75/d times the sum over the
+    stored entries alone (checked against an exactly rounded sum), d still the full dimension."""
+    rng = np.random.default_rng(41)
+    M, d = 3, 9000
+    touched = rng.random((M, d)) < 0.02
+    touched[0, :40] = True
+    vals = rng.standard_normal((M, d)).astype(np.float32)
+    clean = np.where(touched, vals, np.float32(0.0)).astype(np.float32)
+    dirty = np.where(touched, vals, np.float32(np.nan)).astype(np.float32)
+    assert np.array_equal(O.densify_touched(dirty, touched), clean)
+    assert not np.signbit(O.densify_touched(-np.abs(dirty), touched)[~touched]).any()
+    x, h, z = rng.standard_normal(d) * 0.1, rng.random(d), rng.standard_normal(d) * 0.1
+    for quantizer in (O.QUANT_THRESHOLD, O.QUANT_TERNARY_STOCH):
+        for rule in (O.RULE_CMD, O.RULE_RDA):
+            a = O.step(rule, dirty, x, h, z, 3, 1e-3, 0.1, 1e-8, quantizer=quantizer, seed=5, touched=touched)
+            b = O.step(rule, clean, x, h, z, 3, 1e-3, 0.1, 1e-8, quantizer=quantizer, seed=5)
+            assert np.array_equal(a["x"], b["x"]) and np.array_equal(a["h"], b["h"])
+            assert np.array_equal(a["quant"]["codes"], b["quant"]["codes"])
+            assert (a["quant"]["terns"][~touched] == 0).all()
+        if quantizer == O.QUANT_THRESHOLD:
+            for m in range(M):
+                exact = math.fsum(abs(float(v)) for v in vals[m][touched[m]])
+                assert a["quant"]["thresholds"][m] == np.float32(0.75 * exact / d)
+    with pytest.raises(ValueError):
+        O.densify_touched(vals, touched[:, :-1])
