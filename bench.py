@@ -59,10 +59,12 @@ NCU_TRAFFIC = {
 def ncu_traffic(kernel, d, M):
     """Bytes per launch from the stored ncu counters, or None once the kernels have changed."""
     import hashlib
-    src = os.path.join(ROOT, "paper_2208_05631_b200", "csrc", "qasg_kernels.cu")
+    digest = hashlib.sha256()
     try:
-        with open(src, "rb") as f:
-            same = hashlib.sha256(f.read()).hexdigest() == NCU_TRAFFIC["kernels_sha256"]
+        for name in ("qasg_device.cuh", "qasg_kernels.cu"):   # the step kernels and what they inline
+            with open(os.path.join(ROOT, "paper_2208_05631_b200", "csrc", name), "rb") as f:
+                digest.update(f.read())
+        same = digest.hexdigest() == NCU_TRAFFIC["kernels_sha256"]
     except OSError:
         same = False
     if not same or M != NCU_TRAFFIC["M"] or kernel not in NCU_TRAFFIC["bytes_per_coord"]:

@@ -244,6 +244,40 @@ qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int
                                  const uint32_t* batch_rows, uint32_t B, uint64_t t,
                                  const float* x, float* g, uint64_t ld_g, void* stream);
 
+/* Gradients held in sparse form (the text data sets of Section 5.1, Table 1, have a few dozen
+ * non-zeros per row, so a minibatch gradient touches a small part of the d coordinates, and "a zero
+ * entry lies inside [-Delta, Delta] and codes 0", Section 3.4).  The rows of g keep their dense
+ * layout [M][ld_g], but only the entries marked in
+ *   touched   device, uint32 [M][ceil(d/32)], 16-byte aligned: bit i&31 of word i>>5 of row m; bits at
+ *             or past d are ignored
+ * are stored: every other entry IS +0.0, its memory is never read and may hold anything.  Results are
+ * bit for bit those of the dense entry points on the row with +0.0 in the unmarked places (Delta_m
+ * still divides by the full d); the memory traffic shrinks to the touched sectors plus d/8 bytes of
+ * bits per worker.
+ *
+ * qasg_logreg_grad_csr_touched: the CSR gradient in this form.  g and touched carry state from call
+ * to call: on entry the bits must mark every entry of g[.., 0..d) that is not +0.0 (before the first
+ * call: g and touched all zero, once).  The call zeroes the marked entries and the bits, then
+ * accumulates the minibatch with atomic adds and sets the bit of every entry it adds to (a touched
+ * entry may still sum to 0).  Nothing else of g is written or read. */
+qasg_status qasg_logreg_grad_csr_touched(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
+                                         const float* vals, const float* y, uint64_t n_rows,
+                                         uint64_t d, uint32_t M, const uint64_t* shard_row0,
+                                         const uint32_t* batch_rows, uint32_t B, uint64_t t,
+                                         const float* x, float* g, uint64_t ld_g, uint32_t* touched,
+                                         void* stream);
+
+/* qasg_quantize_pack and qasg_step on gradients held in sparse form (see above).  Arguments as
+ * for the dense entry points, plus touched (read only). */
+qasg_status qasg_quantize_pack_touched(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g,
+                                       uint32_t M, uint64_t t, const qasg_params* params,
+                                       const uint32_t* touched, uint32_t* codes, float* scales,
+                                       float* thresholds, uint64_t* counts, void* stream);
+qasg_status qasg_step_touched(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
+                              uint32_t M, uint64_t t, const qasg_params* params, const uint32_t* touched,
+                              float* x, float* h, float* z, uint32_t* codes_out, float* scales_out,
+                              void* stream);
+
 /* The threshold quantizer of qasg_quantize_pack for callers that cannot allocate device
  * memory.  (The paper has no counterpart: this entry point exists for the sake of its
  * callers, not of the method.)

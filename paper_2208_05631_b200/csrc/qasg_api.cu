@@ -32,7 +32,8 @@ namespace {
 enum KernelId {
   kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
   kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kAvgAbsSum, kAvgAbsMax,
-  kAvgThresholdCodes, kAvgStochasticCodes, kSelectStats, kIndicatorOr, kKernelIdCount
+  kAvgThresholdCodes, kAvgStochasticCodes, kSelectStats, kIndicatorOr, kTouchedClear, kLogregCsrTouched,
+  kKernelIdCount
 };
 static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
 
@@ -110,16 +111,16 @@ StepScalars scalars(const qasg_params* p, uint64_t t) {
 // Passes A and B on validated arguments.
 void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint64_t t,
                    const qasg_params* p, uint32_t* codes, float* scales, float* thresholds,
-                   uint64_t* counts, cudaStream_t stream) {
+                   uint64_t* counts, cudaStream_t stream, const uint32_t* touched = nullptr) {
   const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
   if (p->quantizer == QASG_Q_THRESHOLD) {
-    { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream); }
-    { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream); }
+    { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream, nullptr, touched); }
+    { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream, nullptr, touched); }
   } else {
-    { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream); }
+    { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream, touched); }
     { Launch l(ctx, kStochasticCodes, stream); l += launch_stochastic_codes(g, geo, p->seed, t, 0u, ctx->ws, codes, scales, counts_out,
-                                             ctx->shape, stream); }
+                                             ctx->shape, stream, nullptr, touched); }
     if (thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
   }
 }
@@ -368,6 +369,47 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
   return leave();
 }
 
+qasg_status qasg_quantize_pack_touched(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                                       uint64_t t, const qasg_params* params, const uint32_t* touched,
+                                       uint32_t* codes, float* scales, float* thresholds, uint64_t* counts,
+                                       void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, false);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (!touched || !codes || !scales || t < 1) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(codes) || !aligned16(touched)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales, thresholds, counts, static_cast<cudaStream_t>(stream),
+                touched);
+  return leave();
+}
+
+qasg_status qasg_step_touched(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                              uint64_t t, const qasg_params* params, const uint32_t* touched, float* x, float* h,
+                              float* z, uint32_t* codes_out, float* scales_out, void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, true);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
+  if (!touched || !x || !h || t < 1 || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(h) || (z && !aligned16(z)) || (codes_out && !aligned16(codes_out)) ||
+      !aligned16(touched))
+    return QASG_ERR_ALIGNMENT;
+  uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
+  if (!codes) return QASG_ERR_WORKSPACE;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s, touched);
+  {
+    Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s);
+    l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t), ctx->ws.status,
+                              ctx->shape, s);
+  }
+  return leave();
+}
+
 qasg_status qasg_requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                             uint64_t t, const qasg_params* params, uint32_t* qcodes, float* qscale,
                             float* qthreshold, uint64_t* qcount, void* stream) {
@@ -562,6 +604,26 @@ qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int
   return leave();
 }
 
+qasg_status qasg_logreg_grad_csr_touched(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
+                                         const float* vals, const float* y, uint64_t n_rows, uint64_t d,
+                                         uint32_t M, const uint64_t* shard_row0, const uint32_t* batch_rows,
+                                         uint32_t B, uint64_t t, const float* x, float* g, uint64_t ld_g,
+                                         uint32_t* touched, void* stream) {
+  qasg_status st = check_logreg(ctx, y, n_rows, d, M, shard_row0, B, t, x, g, ld_g);
+  if (st != QASG_OK) return st;
+  if (!rowptr || !colidx || !vals || !touched) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(touched)) return QASG_ERR_ALIGNMENT;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  { Launch l(ctx, kTouchedClear, s); l += launch_touched_clear(g, d, ld_g, M, touched, ctx->shape, s); }
+  {
+    Launch l(ctx, kLogregCsrTouched, s);
+    l += launch_logreg_csr(rowptr, colidx, vals, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->shape, s,
+                           touched);
+  }
+  return leave();
+}
+
 qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream) {
   if (!ctx) return QASG_ERR_INVALID_ARG;
   if (enter(ctx) != QASG_OK) return QASG_ERR_CUDA;
@@ -613,7 +675,8 @@ const char* qasg_kernel_name(int id) {
   static const char* const names[kKernelIdCount] = {
       "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
       "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr", "avg_abs_sum",
-      "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes", "select_stats", "indicator_or"};
+      "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes", "select_stats", "indicator_or",
+      "touched_clear", "logreg_csr_touched"};
   return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
 }
 

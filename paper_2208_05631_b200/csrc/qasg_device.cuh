@@ -1,0 +1,460 @@
+// Device-side building blocks shared by the kernel files: tile loads, the fixed-order sums,
+// the grid-completion ticket, the stream of tiles of a CTA, code-byte packing, Philox4x32-10.
+#pragma once
+#include "qasg_internal.h"
+
+namespace qasg {
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ float4 load_f4(const float* p) {
+  return __ldg(reinterpret_cast<const float4*>(p));
+}
+
+// The four float4 a thread owns in the tile starting at coordinate tile_base.
+// Coordinates >= d read as +0.0 (they neither count nor code).
+__device__ __forceinline__ void load_tile(const float* __restrict__ row, uint64_t tile_base,
+                                          uint64_t d, int j, float4 (&v)[kTileRows]) {
+  if (tile_base + kTile <= d) {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) v[r] = load_f4(row + tile_base + r * kTileCols + 4 * j);
+  } else {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) {
+      const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
+      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i0 < d) {
+        t = load_f4(row + i0);  // stays inside the row: ld is a multiple of 4 and >= d
+        if (i0 + 1 >= d) t.y = 0.f;
+        if (i0 + 2 >= d) t.z = 0.f;
+        if (i0 + 3 >= d) t.w = 0.f;
+      }
+      v[r] = t;
+    }
+  }
+}
+
+// Pairwise tree over the 32 lanes (adjacent pairs first).  Addition commutes bit for bit,
+// so both partners of every exchange hold the same value.
+__device__ __forceinline__ double warp_pair_tree(double v) {
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+  return v;
+}
+
+// Streaming pairwise summation over the tiles of a chunk (thread 0 only): stack[l] holds
+// the sum of a complete aligned subtree of 2^l tiles.
+__device__ __forceinline__ void tile_push(double* stack, uint32_t k_local, double v) {
+  int lvl = 0;
+  while (k_local & 1u) {
+    v = stack[lvl] + v;
+    k_local >>= 1;
+    ++lvl;
+  }
+  stack[lvl] = v;
+}
+// Completes the chunk's tree after n <= 2^log2_group tiles (missing tiles are +0.0).
+__device__ __forceinline__ double tile_fold(const double* stack, uint32_t n, uint32_t log2_group) {
+  double carry = 0.0;
+  for (uint32_t lvl = 0; lvl <= log2_group; ++lvl)
+    if ((n >> lvl) & 1u) carry = stack[lvl] + carry;
+  return carry;
+}
+
+// Fixed-order sum over the tiles of one chunk.  Every tile, each thread contributes the sum
+// of its 4 columns; the warp butterfly runs at once, but the eight warp sums of a tile are only
+// parked in shared memory.  Every kBatchTiles tiles (and at the end of the chunk) the CTA meets
+// once: the parked sums are combined tile by tile (pairwise over the 8 warps), then pushed, in
+// tile order, onto the chunk's pairwise stack.  The order of additions is the same as if every
+// tile had been reduced on its own; the warps just do not wait for each other at every tile.
+constexpr int kBatchTiles = 64;
+struct ChunkSumStorage {
+  double warp_sums[kBatchTiles][kThreads / 32];
+  double tile_sums[kBatchTiles];
+  double stack[32];
+};
+
+class ChunkSum {
+ public:
+  __device__ __forceinline__ ChunkSum(ChunkSumStorage* st) : st_(st), pending_(0), pushed_(0) {}
+
+  // Called by all threads, once per tile, in tile order.
+  __device__ __forceinline__ void add_tile(double thread_sum) {
+    const double v = warp_pair_tree(thread_sum);
+    if ((threadIdx.x & 31) == 0) st_->warp_sums[pending_][threadIdx.x >> 5] = v;
+    if (++pending_ == kBatchTiles) flush();
+  }
+
+  // Called by all threads after the chunk's last tile; the chunk sum is valid in thread 0.
+  __device__ __forceinline__ double finish(uint32_t log2_group) {
+    if (pending_) flush();
+    double r = 0.0;
+    if (threadIdx.x == 0) r = tile_fold(st_->stack, pushed_, log2_group);
+    pushed_ = 0;
+    return r;
+  }
+
+ private:
+  __device__ __forceinline__ void flush() {
+    __syncthreads();
+    if (threadIdx.x < pending_) {
+      const double* a = st_->warp_sums[threadIdx.x];
+      st_->tile_sums[threadIdx.x] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (uint32_t i = 0; i < pending_; ++i) tile_push(st_->stack, pushed_ + i, st_->tile_sums[i]);
+    pushed_ += pending_;
+    pending_ = 0;
+  }
+  ChunkSumStorage* st_;
+  uint32_t pending_, pushed_;
+};
+
+// Pairwise tree over a worker's kMaxChunks partial slots (slots >= chunks are +0.0),
+// computed by one warp: 32 adjacent slots per lane, then the lane butterfly.
+__device__ __forceinline__ double warp_chunk_tree(const double* part, uint32_t chunks, int lane) {
+  double top[4];
+#pragma unroll 1
+  for (int q = 0; q < 4; ++q) {  // 8 adjacent slots at a time keeps the register count low
+    double v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const uint32_t idx = lane * 32 + q * 8 + k;
+      v[k] = idx < chunks ? __ldcg(part + idx) : 0.0;
+    }
+    top[q] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+  }
+  return warp_pair_tree((top[0] + top[1]) + (top[2] + top[3]));
+}
+
+// True in every thread of the CTA that finishes last.  All global writes this CTA made
+// before the call (by thread 0) are visible to that CTA.
+__device__ __forceinline__ bool grid_last_cta(unsigned int* ticket, bool* sm_flag) {
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int prev = atomicAdd(ticket, 1u);
+    *sm_flag = (prev == gridDim.x - 1);
+  }
+  __syncthreads();
+  const bool last = *sm_flag;
+  if (last) __threadfence();
+  return last;
+}
+
+// Calls body(tile_values, k) for the tiles k0 <= k < k1 of one worker row, keeping the loads
+// of tile k+1 in flight while tile k is processed (two register buffers, no copies).
+template <class Body>
+__device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64_t d, uint32_t k0,
+                                           uint32_t k1, int j, Body&& body) {
+  float4 a[kTileRows], b[kTileRows];
+  load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
+  uint32_t k = k0;
+  while (true) {
+    if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, b);
+    body(a, k);
+    if (++k >= k1) break;
+    if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, a);
+    body(b, k);
+    if (++k >= k1) break;
+  }
+}
+
+// The indicator bytes a thread needs for its four rows of tile k (two threads share a byte).
+struct TileMask {
+  uint32_t byte[kTileRows];
+  __device__ __forceinline__ uint32_t nibble(int r, int j) const { return (byte[r] >> (4 * (j & 1))) & 15u; }
+};
+__device__ __forceinline__ void load_tile_mask(const uint8_t* __restrict__ ind8, uint64_t d, uint32_t k, int j,
+                                               TileMask& mask) {
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) {
+    const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
+    mask.byte[r] = i0 < d ? static_cast<uint32_t>(__ldg(ind8 + (i0 >> 3))) : 0u;
+  }
+}
+
+// walk_tiles with the tile's indicator bytes travelling along: body(tile_values, mask, k).
+// Without a mask (kMasked false) no byte is loaded and every nibble reads as selected.
+template <bool kMasked, class Body>
+__device__ __forceinline__ void walk_tiles_masked(const float* __restrict__ row, const uint8_t* __restrict__ ind8,
+                                                  uint64_t d, uint32_t k0, uint32_t k1, int j, Body&& body) {
+  float4 a[kTileRows], b[kTileRows];
+  TileMask ma, mb;
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
+  load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
+  if (kMasked) load_tile_mask(ind8, d, k0, j, ma);
+  uint32_t k = k0;
+  while (true) {
+    if (k + 1 < k1) {
+      load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, b);
+      if (kMasked) load_tile_mask(ind8, d, k + 1, j, mb);
+    }
+    body(a, ma, k);
+    if (++k >= k1) break;
+    if (k + 1 < k1) {
+      load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, a);
+      if (kMasked) load_tile_mask(ind8, d, k + 1, j, ma);
+    }
+    body(b, mb, k);
+    if (++k >= k1) break;
+  }
+}
+
+// The CTA's whole share of a launch as one stream of tiles: items blockIdx.x, blockIdx.x + gridDim.x, ...
+// (item = worker m, chunk c), each a run of tiles.  The loads of the next tile are issued before the
+// current one is processed, across item boundaries too, so the memory pipeline never drains between
+// items (at small and medium d an item is only a few tiles long).
+//   begin(m, c)            before the first tile of an item
+//   body(values, mask, k)  every tile
+//   end(m, c, n_tiles)     after the last tile of an item (may synchronise the CTA)
+struct ItemPos {
+  uint32_t item, m, c, k0, k1;
+};
+__device__ __forceinline__ ItemPos item_pos(const Geometry& geo, uint32_t item) {
+  ItemPos p;
+  p.item = item;
+  p.m = item / geo.chunks;
+  p.c = item - p.m * geo.chunks;
+  p.k0 = p.c * geo.group;
+  p.k1 = min(p.k0 + geo.group, geo.tiles);
+  return p;
+}
+
+template <bool kMasked, class Begin, class Body, class End>
+__device__ __forceinline__ void stream_items(const float* __restrict__ g, const uint32_t* __restrict__ indicators,
+                                             const Geometry& geo, int j, Begin&& begin, Body&& body, End&& end) {
+  const uint32_t n_items = geo.M * geo.chunks;
+  if (blockIdx.x >= n_items) return;
+  const uint64_t ind_words = (geo.d + 31) >> 5;
+  ItemPos cur = item_pos(geo, blockIdx.x);
+  uint32_t k = cur.k0;
+  float4 a[kTileRows], b[kTileRows];
+  TileMask ma, mb;
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
+  auto load = [&](const ItemPos& p, uint32_t kk, float4 (&v)[kTileRows], TileMask& mk) {
+    load_tile(g + static_cast<uint64_t>(p.m) * geo.ld, static_cast<uint64_t>(kk) * kTile, geo.d, j, v);
+    if (kMasked)
+      load_tile_mask(reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(p.m) * ind_words), geo.d, kk, j, mk);
+  };
+  load(cur, k, a, ma);
+  begin(cur.m, cur.c);
+  auto step = [&](float4 (&cv)[kTileRows], TileMask& cm, float4 (&nv)[kTileRows], TileMask& nm) -> bool {
+    ItemPos nxt = cur;
+    uint32_t nk = k + 1;
+    bool has_next = true;
+    if (nk >= cur.k1) {
+      const uint32_t ni = cur.item + gridDim.x;
+      has_next = ni < n_items;
+      if (has_next) {
+        nxt = item_pos(geo, ni);
+        nk = nxt.k0;
+      }
+    }
+    if (has_next) load(nxt, nk, nv, nm);
+    body(cv, cm, k);
+    if (k + 1 >= cur.k1) {
+      end(cur.m, cur.c, cur.k1 - cur.k0);
+      if (has_next) begin(nxt.m, nxt.c);
+    }
+    cur = nxt;
+    k = nk;
+    return has_next;
+  };
+  while (step(a, ma, b, mb) && step(b, mb, a, ma)) {
+  }
+}
+
+// ------------------------------------------------------------------ gradients held in sparse form
+// A worker's row stores only the entries its `touched` bits mark (bit i&31 of word i>>5); every other
+// entry is +0.0 by definition and its memory is never read.  The tile geometry and every sum stay those
+// of the dense row (adding +0.0 changes no bit of an fp64 sum of non-negative terms), so the results
+// are those of the dense kernels on the densified row, while the loads shrink to the touched sectors.
+
+// The thread's four float4 of tile k: loaded only where the nibble of touched bits is non-zero,
+// untouched lanes forced to +0.0.  `ragged` is true for a last tile that reaches past d.
+__device__ __forceinline__ void load_touched_tile(const float* __restrict__ row, uint64_t d, uint32_t k, int j,
+                                                  const TileMask& mask, bool ragged, float4 (&v)[kTileRows]) {
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) {
+    const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
+    uint32_t nib = mask.nibble(r, j);
+    if (ragged) {  // bits at or past d do not count, whatever the caller left there
+      if (i0 >= d) nib = 0u;
+      else if (i0 + 4 > d) nib &= (1u << (d - i0)) - 1u;
+    }
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (nib) {
+      t = load_f4(row + i0);  // stays inside the row: ld is a multiple of 4 and >= d
+      if (!(nib & 1u)) t.x = 0.f;
+      if (!(nib & 2u)) t.y = 0.f;
+      if (!(nib & 4u)) t.z = 0.f;
+      if (!(nib & 8u)) t.w = 0.f;
+    }
+    v[r] = t;
+  }
+}
+
+// body(values, k) for the tiles k0 <= k < k1 of one row.  The touched bytes run two tiles ahead of the
+// arithmetic and the values they admit one tile ahead, so neither load is waited for in steady state.
+template <class Body>
+__device__ __forceinline__ void walk_touched_tiles(const float* __restrict__ row, const uint8_t* __restrict__ touched8,
+                                                   uint64_t d, uint32_t tiles, uint32_t k0, uint32_t k1, int j,
+                                                   Body&& body) {
+  float4 a[kTileRows], b[kTileRows];
+  TileMask m_next, m_after;
+  const uint32_t ragged_tile = (d % kTile) ? tiles - 1 : 0xffffffffu;
+  load_tile_mask(touched8, d, k0, j, m_next);
+  if (k0 + 1 < k1) load_tile_mask(touched8, d, k0 + 1, j, m_after);
+  load_touched_tile(row, d, k0, j, m_next, k0 == ragged_tile, a);
+  m_next = m_after;
+  uint32_t k = k0;
+  while (true) {
+    if (k + 2 < k1) load_tile_mask(touched8, d, k + 2, j, m_after);
+    if (k + 1 < k1) load_touched_tile(row, d, k + 1, j, m_next, k + 1 == ragged_tile, b);
+    body(a, k);
+    m_next = m_after;  // after the arithmetic: by now the bytes have arrived
+    if (++k >= k1) break;
+    if (k + 2 < k1) load_tile_mask(touched8, d, k + 2, j, m_after);
+    if (k + 1 < k1) load_touched_tile(row, d, k + 1, j, m_next, k + 1 == ragged_tile, a);
+    body(b, k);
+    m_next = m_after;
+    if (++k >= k1) break;
+  }
+}
+
+// stream_items for touched rows: the same items and callbacks (the mask handed to body is all ones:
+// the values already are +0.0 wherever nothing is stored).
+template <class Begin, class Body, class End>
+__device__ __forceinline__ void stream_touched_items(const float* __restrict__ g, const uint32_t* __restrict__ touched,
+                                                     const Geometry& geo, int j, Begin&& begin, Body&& body,
+                                                     End&& end) {
+  const uint32_t n_items = geo.M * geo.chunks;
+  const uint64_t words = (geo.d + 31) >> 5;
+  TileMask all;
+#pragma unroll
+  for (int r = 0; r < kTileRows; ++r) all.byte[r] = 0xffu;
+  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const ItemPos p = item_pos(geo, item);
+    begin(p.m, p.c);
+    walk_touched_tiles(g + static_cast<uint64_t>(p.m) * geo.ld,
+                       reinterpret_cast<const uint8_t*>(touched + static_cast<uint64_t>(p.m) * words), geo.d,
+                       geo.tiles, p.k0, p.k1, j, [&](const float4 (&v)[kTileRows], uint32_t k) { body(v, all, k); });
+    end(p.m, p.c, p.k1 - p.k0);
+  }
+}
+
+// ------------------------------------------------------------------ pass B helpers
+// Code byte of four coordinates, built on the FMA pipe.  pos/neg are 1.0f or 0.0f per
+// coordinate (code 1 = +1, code 2 = -1); the byte value pos0 + 2 neg0 + 4 pos1 + ... + 128 neg3
+// is accumulated on top of 2^23, where an fp32's low mantissa bits are the integer itself.
+struct CodeBits {
+  float pos, neg;
+};
+__device__ __forceinline__ CodeBits split_code(float v, bool keep) {
+  CodeBits c;
+  c.pos = (keep && v > 0.f) ? 1.f : 0.f;
+  c.neg = (keep && v < 0.f) ? 1.f : 0.f;
+  return c;
+}
+__device__ __forceinline__ uint32_t pack4(CodeBits c0, CodeBits c1, CodeBits c2, CodeBits c3) {
+  float b = 8388608.f;
+  b = fmaf(c0.pos, 1.f, b);
+  b = fmaf(c0.neg, 2.f, b);
+  b = fmaf(c1.pos, 4.f, b);
+  b = fmaf(c1.neg, 8.f, b);
+  b = fmaf(c2.pos, 16.f, b);
+  b = fmaf(c2.neg, 32.f, b);
+  b = fmaf(c3.pos, 64.f, b);
+  b = fmaf(c3.neg, 128.f, b);
+  return __float_as_uint(b) & 0xffu;
+}
+
+// Number of non-zero 2-bit codes in a byte.
+__device__ __forceinline__ uint32_t nonzero_codes(uint32_t byte) {
+  return __popc((byte | (byte >> 1)) & 0x55u);
+}
+
+// Writes the code bytes of the thread's four rows of tile k.  codes8 is the worker's code
+// row; only the last tile can reach past the row's last byte.  The stores are streaming
+// (evict-first): the codes are read back only after the whole gradient has gone by.
+__device__ __forceinline__ void store_code_bytes(uint8_t* __restrict__ codes8, uint32_t k, int j,
+                                                 bool full, uint64_t row_bytes,
+                                                 const uint32_t (&bytes)[kTileRows]) {
+  const uint64_t b0 = static_cast<uint64_t>(k) * (kTile / 4) + j;
+  if (full) {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
+  } else {
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r)
+      if (b0 + r * (kTileCols / 4) < row_bytes) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
+  }
+}
+
+// Sums per-thread counts over the CTA; the result is valid in thread 0.
+__device__ __forceinline__ unsigned long long block_count(uint32_t cnt, uint32_t* sm_cnt) {
+  cnt = __reduce_add_sync(0xffffffffu, cnt);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sm_cnt[threadIdx.x >> 5] = cnt;
+  __syncthreads();
+  unsigned long long total = 0;
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) total += sm_cnt[w];
+  }
+  return total;
+}
+
+// Last-CTA epilogue shared by both code kernels: per-worker totals of the counts, and for
+// the threshold quantizer the scale s_m = P_m / n_m.
+template <bool kThreshold>
+__device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspace& ws,
+                                             float* scales_out, unsigned long long* counts_out) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
+    unsigned long long n = 0;
+    for (uint32_t idx = lane; idx < geo.chunks; idx += 32)
+      n += __ldcg(ws.part_cnt + static_cast<uint64_t>(m) * kMaxChunks + idx);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
+    float scale;
+    if (kThreshold) {
+      const double picked = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+      scale = n ? static_cast<float>(picked / static_cast<double>(n)) : 0.f;
+    } else {
+      scale = ws.scales[m];
+    }
+    if (lane == 0) {
+      ws.counts[m] = n;
+      if (kThreshold) ws.scales[m] = scale;
+      if (scales_out) scales_out[m] = scale;
+      if (counts_out) counts_out[m] = n;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ Philox4x32-10
+// Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3" (SC'11):
+// ten rounds of  (c0,c1,c2,c3) <- (hi(M1*c2)^c1^k0, lo(M1*c2), hi(M0*c0)^c3^k1, lo(M0*c0)),
+// the key advancing by the Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+  constexpr uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u;
+  constexpr uint32_t kW0 = 0x9E3779B9u, kW1 = 0xBB67AE85u;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(kM0, c.x), lo0 = kM0 * c.x;
+    const uint32_t hi1 = __umulhi(kM1, c.z), lo1 = kM1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += kW0;
+    k1 += kW1;
+  }
+  return c;
+}
+
+__device__ __forceinline__ float philox_uniform(uint32_t word) {
+  return static_cast<float>(word >> 8) * 5.9604644775390625e-08f;  // 2^-24, exact
+}
+
+}  // namespace qasg

@@ -66,19 +66,23 @@ struct StepScalars {
 
 // Each launcher enqueues on `stream` and returns the number of kernels it launched.
 // denom (device, [M]) replaces d in Delta = coef * sum / d when the sum runs over selected coordinates.
+// touched ([M][ceil(d/32)] words, bit i&31 of word i>>5): the rows of g are held in sparse form, only the
+// marked entries are stored (and read), every other entry is +0.0.
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
                    float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
-                   const unsigned long long* denom = nullptr);
+                   const unsigned long long* denom = nullptr, const uint32_t* touched = nullptr);
 int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
-                   const LaunchShape& shape, cudaStream_t stream);
+                   const LaunchShape& shape, cudaStream_t stream, const uint32_t* touched = nullptr);
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
-                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators = nullptr);
+                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators = nullptr,
+                           const uint32_t* touched = nullptr);
 // stream_base is added to the worker index in Philox counter word 1 (0 for workers, 1<<16 for the server row).
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
                             uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
-                            cudaStream_t stream, const uint32_t* indicators = nullptr);
+                            cudaStream_t stream, const uint32_t* indicators = nullptr,
+                            const uint32_t* touched = nullptr);
 // Sparse selection: indicators [M][ceil(d/32)] words, bit i&31 of word i>>5.
 int launch_select_stats(int rule, bool stochastic, const float* g, const Geometry& geo, const float* x,
                         const float* hz, const SelectScalars& sc, float coef, const Workspace& ws,
@@ -113,7 +117,12 @@ int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
 int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float* vals,
                       const float* y, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
                       const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
-                      uint64_t ld_g, const LaunchShape& shape, cudaStream_t stream);
+                      uint64_t ld_g, const LaunchShape& shape, cudaStream_t stream, uint32_t* touched = nullptr);
+// With `touched` the launcher does not clear g: it adds into rows that are zero wherever the bits are zero
+// and sets the bit of every entry it adds to.  launch_touched_clear re-establishes that state from the
+// bits a previous gradient left: zeroes the marked entries of g, then the bits.
+int launch_touched_clear(float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint32_t* touched,
+                         const LaunchShape& shape, cudaStream_t stream);
 
 void query_launch_shape(LaunchShape* shape);
 

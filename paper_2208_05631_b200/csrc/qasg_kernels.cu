@@ -15,7 +15,7 @@
 // the grid: column sums down the rows, a pairwise tree over the 1024 columns (in-thread,
 // warp butterfly, across warps), a pairwise tree over tiles.  The CTA that finishes last
 // combines the per-chunk partials, so no extra launch or host round trip is needed.
-#include "qasg_internal.h"
+#include "qasg_device.cuh"
 
 namespace qasg {
 
@@ -44,278 +44,19 @@ Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks,
   return geo;
 }
 
-// ------------------------------------------------------------------ device helpers
-__device__ __forceinline__ float4 load_f4(const float* p) {
-  return __ldg(reinterpret_cast<const float4*>(p));
-}
-
-// The four float4 a thread owns in the tile starting at coordinate tile_base.
-// Coordinates >= d read as +0.0 (they neither count nor code).
-__device__ __forceinline__ void load_tile(const float* __restrict__ row, uint64_t tile_base,
-                                          uint64_t d, int j, float4 (&v)[kTileRows]) {
-  if (tile_base + kTile <= d) {
-#pragma unroll
-    for (int r = 0; r < kTileRows; ++r) v[r] = load_f4(row + tile_base + r * kTileCols + 4 * j);
-  } else {
-#pragma unroll
-    for (int r = 0; r < kTileRows; ++r) {
-      const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
-      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (i0 < d) {
-        t = load_f4(row + i0);  // stays inside the row: ld is a multiple of 4 and >= d
-        if (i0 + 1 >= d) t.y = 0.f;
-        if (i0 + 2 >= d) t.z = 0.f;
-        if (i0 + 3 >= d) t.w = 0.f;
-      }
-      v[r] = t;
-    }
-  }
-}
-
-// Pairwise tree over the 32 lanes (adjacent pairs first).  Addition commutes bit for bit,
-// so both partners of every exchange hold the same value.
-__device__ __forceinline__ double warp_pair_tree(double v) {
-#pragma unroll
-  for (int s = 1; s < 32; s <<= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-  return v;
-}
-
-// Streaming pairwise summation over the tiles of a chunk (thread 0 only): stack[l] holds
-// the sum of a complete aligned subtree of 2^l tiles.
-__device__ __forceinline__ void tile_push(double* stack, uint32_t k_local, double v) {
-  int lvl = 0;
-  while (k_local & 1u) {
-    v = stack[lvl] + v;
-    k_local >>= 1;
-    ++lvl;
-  }
-  stack[lvl] = v;
-}
-// Completes the chunk's tree after n <= 2^log2_group tiles (missing tiles are +0.0).
-__device__ __forceinline__ double tile_fold(const double* stack, uint32_t n, uint32_t log2_group) {
-  double carry = 0.0;
-  for (uint32_t lvl = 0; lvl <= log2_group; ++lvl)
-    if ((n >> lvl) & 1u) carry = stack[lvl] + carry;
-  return carry;
-}
-
-// Fixed-order sum over the tiles of one chunk.  Every tile, each thread contributes the sum
-// of its 4 columns; the warp butterfly runs at once, but the eight warp sums of a tile are only
-// parked in shared memory.  Every kBatchTiles tiles (and at the end of the chunk) the CTA meets
-// once: the parked sums are combined tile by tile (pairwise over the 8 warps), then pushed, in
-// tile order, onto the chunk's pairwise stack.  The order of additions is the same as if every
-// tile had been reduced on its own; the warps just do not wait for each other at every tile.
-constexpr int kBatchTiles = 64;
-struct ChunkSumStorage {
-  double warp_sums[kBatchTiles][kThreads / 32];
-  double tile_sums[kBatchTiles];
-  double stack[32];
-};
-
-class ChunkSum {
- public:
-  __device__ __forceinline__ ChunkSum(ChunkSumStorage* st) : st_(st), pending_(0), pushed_(0) {}
-
-  // Called by all threads, once per tile, in tile order.
-  __device__ __forceinline__ void add_tile(double thread_sum) {
-    const double v = warp_pair_tree(thread_sum);
-    if ((threadIdx.x & 31) == 0) st_->warp_sums[pending_][threadIdx.x >> 5] = v;
-    if (++pending_ == kBatchTiles) flush();
-  }
-
-  // Called by all threads after the chunk's last tile; the chunk sum is valid in thread 0.
-  __device__ __forceinline__ double finish(uint32_t log2_group) {
-    if (pending_) flush();
-    double r = 0.0;
-    if (threadIdx.x == 0) r = tile_fold(st_->stack, pushed_, log2_group);
-    pushed_ = 0;
-    return r;
-  }
-
- private:
-  __device__ __forceinline__ void flush() {
-    __syncthreads();
-    if (threadIdx.x < pending_) {
-      const double* a = st_->warp_sums[threadIdx.x];
-      st_->tile_sums[threadIdx.x] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
-    }
-    __syncthreads();
-    if (threadIdx.x == 0)
-      for (uint32_t i = 0; i < pending_; ++i) tile_push(st_->stack, pushed_ + i, st_->tile_sums[i]);
-    pushed_ += pending_;
-    pending_ = 0;
-  }
-  ChunkSumStorage* st_;
-  uint32_t pending_, pushed_;
-};
-
-// Pairwise tree over a worker's kMaxChunks partial slots (slots >= chunks are +0.0),
-// computed by one warp: 32 adjacent slots per lane, then the lane butterfly.
-__device__ __forceinline__ double warp_chunk_tree(const double* part, uint32_t chunks, int lane) {
-  double top[4];
-#pragma unroll 1
-  for (int q = 0; q < 4; ++q) {  // 8 adjacent slots at a time keeps the register count low
-    double v[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const uint32_t idx = lane * 32 + q * 8 + k;
-      v[k] = idx < chunks ? __ldcg(part + idx) : 0.0;
-    }
-    top[q] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
-  }
-  return warp_pair_tree((top[0] + top[1]) + (top[2] + top[3]));
-}
-
-// True in every thread of the CTA that finishes last.  All global writes this CTA made
-// before the call (by thread 0) are visible to that CTA.
-__device__ __forceinline__ bool grid_last_cta(unsigned int* ticket, bool* sm_flag) {
-  if (threadIdx.x == 0) {
-    __threadfence();
-    const unsigned int prev = atomicAdd(ticket, 1u);
-    *sm_flag = (prev == gridDim.x - 1);
-  }
-  __syncthreads();
-  const bool last = *sm_flag;
-  if (last) __threadfence();
-  return last;
-}
-
-// Calls body(tile_values, k) for the tiles k0 <= k < k1 of one worker row, keeping the loads
-// of tile k+1 in flight while tile k is processed (two register buffers, no copies).
-template <class Body>
-__device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64_t d, uint32_t k0,
-                                           uint32_t k1, int j, Body&& body) {
-  float4 a[kTileRows], b[kTileRows];
-  load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
-  uint32_t k = k0;
-  while (true) {
-    if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, b);
-    body(a, k);
-    if (++k >= k1) break;
-    if (k + 1 < k1) load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, a);
-    body(b, k);
-    if (++k >= k1) break;
-  }
-}
-
-// The indicator bytes a thread needs for its four rows of tile k (two threads share a byte).
-struct TileMask {
-  uint32_t byte[kTileRows];
-  __device__ __forceinline__ uint32_t nibble(int r, int j) const { return (byte[r] >> (4 * (j & 1))) & 15u; }
-};
-__device__ __forceinline__ void load_tile_mask(const uint8_t* __restrict__ ind8, uint64_t d, uint32_t k, int j,
-                                               TileMask& mask) {
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) {
-    const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
-    mask.byte[r] = i0 < d ? static_cast<uint32_t>(__ldg(ind8 + (i0 >> 3))) : 0u;
-  }
-}
-
-// walk_tiles with the tile's indicator bytes travelling along: body(tile_values, mask, k).
-// Without a mask (kMasked false) no byte is loaded and every nibble reads as selected.
-template <bool kMasked, class Body>
-__device__ __forceinline__ void walk_tiles_masked(const float* __restrict__ row, const uint8_t* __restrict__ ind8,
-                                                  uint64_t d, uint32_t k0, uint32_t k1, int j, Body&& body) {
-  float4 a[kTileRows], b[kTileRows];
-  TileMask ma, mb;
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
-  load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
-  if (kMasked) load_tile_mask(ind8, d, k0, j, ma);
-  uint32_t k = k0;
-  while (true) {
-    if (k + 1 < k1) {
-      load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, b);
-      if (kMasked) load_tile_mask(ind8, d, k + 1, j, mb);
-    }
-    body(a, ma, k);
-    if (++k >= k1) break;
-    if (k + 1 < k1) {
-      load_tile(row, static_cast<uint64_t>(k + 1) * kTile, d, j, a);
-      if (kMasked) load_tile_mask(ind8, d, k + 1, j, ma);
-    }
-    body(b, mb, k);
-    if (++k >= k1) break;
-  }
-}
-
-// The CTA's whole share of a launch as one stream of tiles: items blockIdx.x, blockIdx.x + gridDim.x, ...
-// (item = worker m, chunk c), each a run of tiles.  The loads of the next tile are issued before the
-// current one is processed, across item boundaries too, so the memory pipeline never drains between
-// items (at small and medium d an item is only a few tiles long).
-//   begin(m, c)            before the first tile of an item
-//   body(values, mask, k)  every tile
-//   end(m, c, n_tiles)     after the last tile of an item (may synchronise the CTA)
-struct ItemPos {
-  uint32_t item, m, c, k0, k1;
-};
-__device__ __forceinline__ ItemPos item_pos(const Geometry& geo, uint32_t item) {
-  ItemPos p;
-  p.item = item;
-  p.m = item / geo.chunks;
-  p.c = item - p.m * geo.chunks;
-  p.k0 = p.c * geo.group;
-  p.k1 = min(p.k0 + geo.group, geo.tiles);
-  return p;
-}
-
-template <bool kMasked, class Begin, class Body, class End>
-__device__ __forceinline__ void stream_items(const float* __restrict__ g, const uint32_t* __restrict__ indicators,
-                                             const Geometry& geo, int j, Begin&& begin, Body&& body, End&& end) {
-  const uint32_t n_items = geo.M * geo.chunks;
-  if (blockIdx.x >= n_items) return;
-  const uint64_t ind_words = (geo.d + 31) >> 5;
-  ItemPos cur = item_pos(geo, blockIdx.x);
-  uint32_t k = cur.k0;
-  float4 a[kTileRows], b[kTileRows];
-  TileMask ma, mb;
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
-  auto load = [&](const ItemPos& p, uint32_t kk, float4 (&v)[kTileRows], TileMask& mk) {
-    load_tile(g + static_cast<uint64_t>(p.m) * geo.ld, static_cast<uint64_t>(kk) * kTile, geo.d, j, v);
-    if (kMasked)
-      load_tile_mask(reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(p.m) * ind_words), geo.d, kk, j, mk);
-  };
-  load(cur, k, a, ma);
-  begin(cur.m, cur.c);
-  auto step = [&](float4 (&cv)[kTileRows], TileMask& cm, float4 (&nv)[kTileRows], TileMask& nm) -> bool {
-    ItemPos nxt = cur;
-    uint32_t nk = k + 1;
-    bool has_next = true;
-    if (nk >= cur.k1) {
-      const uint32_t ni = cur.item + gridDim.x;
-      has_next = ni < n_items;
-      if (has_next) {
-        nxt = item_pos(geo, ni);
-        nk = nxt.k0;
-      }
-    }
-    if (has_next) load(nxt, nk, nv, nm);
-    body(cv, cm, k);
-    if (k + 1 >= cur.k1) {
-      end(cur.m, cur.c, cur.k1 - cur.k0);
-      if (has_next) begin(nxt.m, nxt.c);
-    }
-    cur = nxt;
-    k = nk;
-    return has_next;
-  };
-  while (step(a, ma, b, mb) && step(b, mb, a, ma)) {
-  }
-}
-
 // ------------------------------------------------------------------ pass A: sum |g|
+// kTouched: the rows are held in sparse form, `touched` marks their stored entries.
+template <bool kTouched>
 __global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
-               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom) {
+               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom,
+               const uint32_t* __restrict__ touched) {
   __shared__ ChunkSumStorage sm_sum;
   __shared__ bool sm_last;
   const int j = threadIdx.x;
   ChunkSum chunk_sum(&sm_sum);
-  stream_items<false>(
-      g, nullptr, geo, j, [](uint32_t, uint32_t) {},
-      [&](const float4 (&v)[kTileRows], const TileMask&, uint32_t) {
+  auto begin = [](uint32_t, uint32_t) {};
+  auto body = [&](const float4 (&v)[kTileRows], const TileMask&, uint32_t) {
         double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
 #pragma unroll
         for (int r = 1; r < kTileRows; ++r) {
@@ -325,11 +66,15 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
           cw += static_cast<double>(fabsf(v[r].w));
         }
         chunk_sum.add_tile((cx + cy) + (cz + cw));
-      },
-      [&](uint32_t m, uint32_t c, uint32_t) {
+      };
+  auto end = [&](uint32_t m, uint32_t c, uint32_t) {
         const double total = chunk_sum.finish(geo.log2_group);
         if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
-      });
+      };
+  if (kTouched)
+    stream_touched_items(g, touched, geo, j, begin, body, end);
+  else
+    stream_items<false>(g, nullptr, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   const int warp = j >> 5, lane = j & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
@@ -347,8 +92,9 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
 }
 
 // ------------------------------------------------------------------ pass A': max |g|
+template <bool kTouched>
 __global__ void __launch_bounds__(kThreads)
-abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
+abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws, const uint32_t* __restrict__ touched) {
   __shared__ uint32_t sm_warp[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -359,7 +105,7 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t best = 0u;  // bit patterns of non-negative floats order like their values
-    walk_tiles(row, geo.d, k0, k1, j, [&](const float4 (&v)[kTileRows], uint32_t) {
+    auto body = [&](const float4 (&v)[kTileRows], uint32_t) {
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
         best = max(best, __float_as_uint(fabsf(v[r].x)));
@@ -367,7 +113,12 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
         best = max(best, __float_as_uint(fabsf(v[r].z)));
         best = max(best, __float_as_uint(fabsf(v[r].w)));
       }
-    });
+    };
+    if (kTouched)
+      walk_touched_tiles(row, reinterpret_cast<const uint8_t*>(touched + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5)),
+                         geo.d, geo.tiles, k0, k1, j, body);
+    else
+      walk_tiles(row, geo.d, k0, k1, j, body);
     best = __reduce_max_sync(0xffffffffu, best);
     __syncthreads();  // the previous item's readers are done with sm_warp
     if ((j & 31) == 0) sm_warp[j >> 5] = best;
@@ -395,103 +146,15 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
   if (j == 0) *ws.ticket = 0u;
 }
 
-// ------------------------------------------------------------------ pass B helpers
-// Code byte of four coordinates, built on the FMA pipe.  pos/neg are 1.0f or 0.0f per
-// coordinate (code 1 = +1, code 2 = -1); the byte value pos0 + 2 neg0 + 4 pos1 + ... + 128 neg3
-// is accumulated on top of 2^23, where an fp32's low mantissa bits are the integer itself.
-struct CodeBits {
-  float pos, neg;
-};
-__device__ __forceinline__ CodeBits split_code(float v, bool keep) {
-  CodeBits c;
-  c.pos = (keep && v > 0.f) ? 1.f : 0.f;
-  c.neg = (keep && v < 0.f) ? 1.f : 0.f;
-  return c;
-}
-__device__ __forceinline__ uint32_t pack4(CodeBits c0, CodeBits c1, CodeBits c2, CodeBits c3) {
-  float b = 8388608.f;
-  b = fmaf(c0.pos, 1.f, b);
-  b = fmaf(c0.neg, 2.f, b);
-  b = fmaf(c1.pos, 4.f, b);
-  b = fmaf(c1.neg, 8.f, b);
-  b = fmaf(c2.pos, 16.f, b);
-  b = fmaf(c2.neg, 32.f, b);
-  b = fmaf(c3.pos, 64.f, b);
-  b = fmaf(c3.neg, 128.f, b);
-  return __float_as_uint(b) & 0xffu;
-}
-
-// Number of non-zero 2-bit codes in a byte.
-__device__ __forceinline__ uint32_t nonzero_codes(uint32_t byte) {
-  return __popc((byte | (byte >> 1)) & 0x55u);
-}
-
-// Writes the code bytes of the thread's four rows of tile k.  codes8 is the worker's code
-// row; only the last tile can reach past the row's last byte.  The stores are streaming
-// (evict-first): the codes are read back only after the whole gradient has gone by.
-__device__ __forceinline__ void store_code_bytes(uint8_t* __restrict__ codes8, uint32_t k, int j,
-                                                 bool full, uint64_t row_bytes,
-                                                 const uint32_t (&bytes)[kTileRows]) {
-  const uint64_t b0 = static_cast<uint64_t>(k) * (kTile / 4) + j;
-  if (full) {
-#pragma unroll
-    for (int r = 0; r < kTileRows; ++r) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
-  } else {
-#pragma unroll
-    for (int r = 0; r < kTileRows; ++r)
-      if (b0 + r * (kTileCols / 4) < row_bytes) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
-  }
-}
-
-// Sums per-thread counts over the CTA; the result is valid in thread 0.
-__device__ __forceinline__ unsigned long long block_count(uint32_t cnt, uint32_t* sm_cnt) {
-  cnt = __reduce_add_sync(0xffffffffu, cnt);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) sm_cnt[threadIdx.x >> 5] = cnt;
-  __syncthreads();
-  unsigned long long total = 0;
-  if (threadIdx.x == 0) {
-#pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) total += sm_cnt[w];
-  }
-  return total;
-}
-
-// Last-CTA epilogue shared by both code kernels: per-worker totals of the counts, and for
-// the threshold quantizer the scale s_m = P_m / n_m.
-template <bool kThreshold>
-__device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspace& ws,
-                                             float* scales_out, unsigned long long* counts_out) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
-    unsigned long long n = 0;
-    for (uint32_t idx = lane; idx < geo.chunks; idx += 32)
-      n += __ldcg(ws.part_cnt + static_cast<uint64_t>(m) * kMaxChunks + idx);
-#pragma unroll
-    for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
-    float scale;
-    if (kThreshold) {
-      const double picked = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
-      scale = n ? static_cast<float>(picked / static_cast<double>(n)) : 0.f;
-    } else {
-      scale = ws.scales[m];
-    }
-    if (lane == 0) {
-      ws.counts[m] = n;
-      if (kThreshold) ws.scales[m] = scale;
-      if (scales_out) scales_out[m] = scale;
-      if (counts_out) counts_out[m] = n;
-    }
-  }
-}
-
 // ------------------------------------------------------------------ pass B: Q_Delta codes
-// kMasked: only coordinates whose indicator bit is set are candidates (sparse selection, Q(S(g, I))).
-template <bool kMasked>
+// kMode 0: dense rows.  1: only coordinates whose indicator bit is set are candidates (sparse selection,
+// Q(S(g, I))); `bits` are the indicators.  2: rows held in sparse form; `bits` mark the stored entries.
+template <int kMode>
 __global__ void __launch_bounds__(kThreads, 4)
 threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
                        uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
+                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ bits) {
+  constexpr bool kMasked = kMode == 1;
   __shared__ ChunkSumStorage sm_sum;
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
@@ -501,15 +164,13 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
   ChunkSum chunk_sum(&sm_sum);
   uint8_t* codes8 = nullptr;  // per item: the worker's code row, its threshold, the kept count so far
   float delta = 0.f, ndelta = 0.f, cntf = 0.f;
-  stream_items<kMasked>(
-      g, indicators, geo, j,
-      [&](uint32_t m, uint32_t) {
+  auto begin = [&](uint32_t m, uint32_t) {
         codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
         delta = ws.thresholds[m];
         ndelta = -delta;
         cntf = 0.f;
-      },
-      [&](const float4 (&v)[kTileRows], const TileMask& mask, uint32_t k) {
+      };
+  auto body = [&](const float4 (&v)[kTileRows], const TileMask& mask, uint32_t k) {
         double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
         uint32_t bytes[kTileRows];
 #pragma unroll
@@ -537,8 +198,8 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
         }
         store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
         chunk_sum.add_tile((cx + cy) + (cz + cw));
-      },
-      [&](uint32_t m, uint32_t c, uint32_t) {
+      };
+  auto end = [&](uint32_t m, uint32_t c, uint32_t) {
         const double picked = chunk_sum.finish(geo.log2_group);
         const unsigned long long total = block_count(static_cast<uint32_t>(cntf), sm_cnt);
         if (j == 0) {
@@ -546,40 +207,23 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
           ws.part_sum[p] = picked;
           ws.part_cnt[p] = total;
         }
-      });
+      };
+  if (kMode == 2)
+    stream_touched_items(g, bits, geo, j, begin, body, end);
+  else
+    stream_items<kMasked>(g, bits, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   finish_codes<true>(geo, ws, scales_out, counts_out);
   if (j == 0) *ws.ticket = 0u;
 }
 
-// ------------------------------------------------------------------ Philox4x32-10
-// Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3" (SC'11):
-// ten rounds of  (c0,c1,c2,c3) <- (hi(M1*c2)^c1^k0, lo(M1*c2), hi(M0*c0)^c3^k1, lo(M0*c0)),
-// the key advancing by the Weyl constants between rounds.
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
-  constexpr uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u;
-  constexpr uint32_t kW0 = 0x9E3779B9u, kW1 = 0xBB67AE85u;
-#pragma unroll
-  for (int round = 0; round < 10; ++round) {
-    const uint32_t hi0 = __umulhi(kM0, c.x), lo0 = kM0 * c.x;
-    const uint32_t hi1 = __umulhi(kM1, c.z), lo1 = kM1 * c.z;
-    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
-    k0 += kW0;
-    k1 += kW1;
-  }
-  return c;
-}
-
-__device__ __forceinline__ float philox_uniform(uint32_t word) {
-  return static_cast<float>(word >> 8) * 5.9604644775390625e-08f;  // 2^-24, exact
-}
-
 // ------------------------------------------------------------------ pass B': stochastic codes
-template <bool kMasked>
+template <int kMode>  // as for threshold_codes_kernel
 __global__ void __launch_bounds__(kThreads)
 stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
                         uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
+                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ bits) {
+  constexpr bool kMasked = kMode == 1;
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -593,13 +237,12 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
     const float scale = ws.scales[m];
-    const uint8_t* ind8 = kMasked ? reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5))
-                                  : nullptr;
+    const uint8_t* ind8 = kMode ? reinterpret_cast<const uint8_t*>(bits + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5))
+                                : nullptr;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
-    walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, [&](const float4 (&tile)[kTileRows],
-                                                                const TileMask& mask, uint32_t k) {
+    auto body = [&](const float4 (&tile)[kTileRows], const TileMask& mask, uint32_t k) {
       uint32_t bytes[kTileRows];
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
@@ -620,7 +263,16 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
         cnt += nonzero_codes(bytes[r]);
       }
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
-    });
+    };
+    if (kMode == 2) {
+      TileMask all;
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r) all.byte[r] = 0xffu;
+      walk_touched_tiles(row, ind8, geo.d, geo.tiles, k0, k1, j,
+                         [&](const float4 (&tile)[kTileRows], uint32_t k) { body(tile, all, k); });
+    } else {
+      walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, body);
+    }
     const unsigned long long total = block_count(cnt, sm_cnt);
     if (j == 0) ws.part_cnt[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
   }
@@ -1353,38 +1005,53 @@ static unsigned update_grid(uint64_t d, const LaunchShape& shape) {
 
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
                    float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
-                   const unsigned long long* denom) {
-  abs_sum_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom);
+                   const unsigned long long* denom, const uint32_t* touched) {
+  if (touched)
+    abs_sum_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom,
+                                                                          touched);
+  else
+    abs_sum_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom,
+                                                                           nullptr);
   return 1;
 }
 
 int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
-                   const LaunchShape& shape, cudaStream_t stream) {
-  abs_max_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws);
+                   const LaunchShape& shape, cudaStream_t stream, const uint32_t* touched) {
+  if (touched)
+    abs_max_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, touched);
+  else
+    abs_max_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, nullptr);
   return 1;
 }
 
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
-                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators) {
-  if (indicators)
-    threshold_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                                  counts_out, indicators);
+                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators,
+                           const uint32_t* touched) {
+  if (touched)
+    threshold_codes_kernel<2><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                               counts_out, touched);
+  else if (indicators)
+    threshold_codes_kernel<1><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                               counts_out, indicators);
   else
-    threshold_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                                   counts_out, nullptr);
+    threshold_codes_kernel<0><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                               counts_out, nullptr);
   return 1;
 }
 
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
                             uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
-                            cudaStream_t stream, const uint32_t* indicators) {
-  if (indicators)
-    stochastic_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+                            cudaStream_t stream, const uint32_t* indicators, const uint32_t* touched) {
+  if (touched)
+    stochastic_codes_kernel<2><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+        g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, touched);
+  else if (indicators)
+    stochastic_codes_kernel<1><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
         g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, indicators);
   else
-    stochastic_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+    stochastic_codes_kernel<0><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
         g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, nullptr);
   return 1;
 }

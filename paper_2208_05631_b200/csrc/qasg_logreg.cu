@@ -3,7 +3,9 @@
 // Dense: GEMV-shaped and memory-bound.  Kernel 1 computes one coefficient per minibatch
 // row (a warp per row, 128-bit loads); kernel 2 forms the coefficient-weighted column sums
 // with a fixed summation order, reading the rows a second time out of L2.
-// CSR: one warp per minibatch row computes the margin and scatters with atomic adds.
+// CSR: one warp per minibatch row computes the margin and scatters with atomic adds.  The sparse form
+// keeps the dense rows of g zero between calls and a bit per entry that a minibatch touched, so a call
+// moves the touched sectors only (no clearing or re-reading of M*d floats).
 #include "qasg_internal.h"
 
 namespace qasg {
@@ -98,11 +100,12 @@ logreg_dense_colsum_kernel(const float* __restrict__ X, uint64_t d, uint32_t B, 
   }
 }
 
+template <bool kTouched>
 __global__ void __launch_bounds__(kThreads)
 logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ colidx,
                   const float* __restrict__ vals, const float* __restrict__ y, uint32_t M, Shards sh,
                   const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t, const float* __restrict__ x,
-                  float* __restrict__ g, uint64_t ld_g) {
+                  float* __restrict__ g, uint64_t ld_g, uint32_t* __restrict__ touched, uint64_t touched_words) {
   const uint32_t warp = (blockIdx.x * kThreads + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= M * B) return;
   const uint32_t m = warp / B, b = warp - m * B;
@@ -114,7 +117,32 @@ logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict_
   for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
   const float c = logistic_coef(y[r], acc, 1.f / static_cast<float>(B));
   float* row = g + static_cast<uint64_t>(m) * ld_g;
-  for (int64_t k = lo + lane; k < hi; k += 32) atomicAdd(row + __ldg(colidx + k), c * __ldg(vals + k));
+  uint32_t* bits = kTouched ? touched + static_cast<uint64_t>(m) * touched_words : nullptr;
+  for (int64_t k = lo + lane; k < hi; k += 32) {
+    const uint32_t col = static_cast<uint32_t>(__ldg(colidx + k));
+    atomicAdd(row + col, c * __ldg(vals + k));
+    if (kTouched) atomicOr(bits + (col >> 5), 1u << (col & 31u));
+  }
+}
+
+// One thread per word of touched bits: zeroes the entries of g the word marks, then the word.
+__global__ void __launch_bounds__(kThreads)
+touched_clear_kernel(float* __restrict__ g, uint64_t ld_g, uint32_t M, uint32_t* __restrict__ touched,
+                     uint64_t touched_words, uint64_t d) {
+  const uint64_t total = static_cast<uint64_t>(M) * touched_words;
+  for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < total;
+       w += static_cast<uint64_t>(gridDim.x) * kThreads) {
+    uint32_t bits = touched[w];
+    if (!bits) continue;
+    const uint64_t m = w / touched_words, word = w - m * touched_words;
+    float* base = g + m * ld_g + word * 32;
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      if (word * 32 + b < d) base[b] = 0.f;  // a stray bit past d marks nothing
+      bits &= bits - 1;
+    }
+    touched[w] = 0u;
+  }
 }
 
 static Shards make_shards(const uint64_t* shard_row0_host, uint32_t M) {
@@ -140,12 +168,28 @@ int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
 int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float* vals,
                       const float* y, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
                       const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
-                      uint64_t ld_g, const LaunchShape&, cudaStream_t stream) {
+                      uint64_t ld_g, const LaunchShape&, cudaStream_t stream, uint32_t* touched) {
   const Shards sh = make_shards(shard_row0_host, M);
-  cudaMemset2DAsync(g, ld_g * sizeof(float), 0, d * sizeof(float), M, stream);
   const uint64_t warps = static_cast<uint64_t>(M) * B;
   const unsigned grid = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
-  logreg_csr_kernel<<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, M, sh, batch_rows, B, t, x, g, ld_g);
+  if (touched) {
+    logreg_csr_kernel<true><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, M, sh, batch_rows, B, t, x, g,
+                                                          ld_g, touched, (d + 31) >> 5);
+  } else {
+    cudaMemset2DAsync(g, ld_g * sizeof(float), 0, d * sizeof(float), M, stream);
+    logreg_csr_kernel<false><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, M, sh, batch_rows, B, t, x, g,
+                                                           ld_g, nullptr, 0);
+  }
+  return 1;
+}
+
+int launch_touched_clear(float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint32_t* touched,
+                         const LaunchShape& shape, cudaStream_t stream) {
+  const uint64_t words = (d + 31) >> 5;
+  const uint64_t ctas = (static_cast<uint64_t>(M) * words + kThreads - 1) / kThreads;
+  const uint64_t cap = static_cast<uint64_t>(shape.sm_count) * 32;
+  touched_clear_kernel<<<static_cast<unsigned>(ctas < cap ? ctas : cap), kThreads, 0, stream>>>(g, ld_g, M, touched,
+                                                                                              words, d);
   return 1;
 }
 

@@ -27,6 +27,7 @@ EXPORTS = [
     "qasg_logreg_grad_csr", "qasg_last_async_status", "qasg_launch_count", "qasg_status_string",
     "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static", "qasg_requantize", "qasg_step_double",
     "qasg_select_quantize_pack", "qasg_indicator_or", "qasg_step_select",
+    "qasg_logreg_grad_csr_touched", "qasg_quantize_pack_touched", "qasg_step_touched",
 ]
 STATIC_MAX_WORKERS = 16
 KERNEL_COUNT = 24
@@ -83,6 +84,10 @@ def load():
                                            vp, vp, u64, vp]
     lib.qasg_logreg_grad_csr.argtypes = [vp, vp, vp, vp, vp, u64, u64, u32, ctypes.POINTER(u64), vp, u32,
                                          u64, vp, vp, u64, vp]
+    lib.qasg_logreg_grad_csr_touched.argtypes = [vp, vp, vp, vp, vp, u64, u64, u32, ctypes.POINTER(u64), vp, u32,
+                                                 u64, vp, vp, u64, vp, vp]
+    lib.qasg_quantize_pack_touched.argtypes = [vp, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp]
+    lib.qasg_step_touched.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp]
     lib.qasg_last_async_status.argtypes = [vp, vp]
     lib.qasg_launch_count.argtypes = [vp]
     lib.qasg_launch_count.restype = u64
@@ -215,6 +220,25 @@ class Context:
         _check(load().qasg_logreg_grad_csr(self._h, _ptr(rowptr), _ptr(colidx), _ptr(vals), _ptr(y), n_rows,
                                            d, M, _shards(shard_row0), _ptr(batch_rows), B, t, _ptr(x),
                                            _ptr(g), ld_g, _stream(stream)), "qasg_logreg_grad_csr")
+
+    def logreg_grad_csr_touched(self, rowptr, colidx, vals, y, n_rows, d, M, shard_row0, batch_rows, B, t, x, g,
+                                ld_g, touched, stream=None):
+        _check(load().qasg_logreg_grad_csr_touched(self._h, _ptr(rowptr), _ptr(colidx), _ptr(vals), _ptr(y),
+                                                   n_rows, d, M, _shards(shard_row0), _ptr(batch_rows), B, t,
+                                                   _ptr(x), _ptr(g), ld_g, _ptr(touched), _stream(stream)),
+               "qasg_logreg_grad_csr_touched")
+
+    def quantize_pack_touched(self, g, d, ld_g, M, t, params, touched, codes, scales, thresholds=None,
+                              counts=None, stream=None):
+        _check(load().qasg_quantize_pack_touched(self._h, _ptr(g), d, ld_g, M, t, ctypes.byref(params),
+                                                 _ptr(touched), _ptr(codes), _ptr(scales), _ptr(thresholds),
+                                                 _ptr(counts), _stream(stream)), "qasg_quantize_pack_touched")
+
+    def step_touched(self, rule, g, d, ld_g, M, t, params, touched, x, h, z=None, codes_out=None,
+                     scales_out=None, stream=None):
+        _check(load().qasg_step_touched(self._h, rule, _ptr(g), d, ld_g, M, t, ctypes.byref(params),
+                                        _ptr(touched), _ptr(x), _ptr(h), _ptr(z), _ptr(codes_out),
+                                        _ptr(scales_out), _stream(stream)), "qasg_step_touched")
 
     def last_async_status(self, stream=None):
         return int(load().qasg_last_async_status(self._h, _stream(stream)))

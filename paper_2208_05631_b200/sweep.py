@@ -135,7 +135,7 @@ def sweep_logreg(args):
     prob = inputs.logreg_dense_problem(n=n, d=d, M=M, seed=1)
     X, y = torch.from_numpy(prob["X"]).to(dev), torch.from_numpy(prob["y"]).to(dev)
     ctx = libqasg.Context(1 << 24, 16, device=0)
-    for rule, name in ((libqasg.RULE_CMD, "qcmd"), (libqasg.RULE_RDA, "qrda")):
+    for rule, name in (() if args.csr_only else ((libqasg.RULE_CMD, "qcmd"), (libqasg.RULE_RDA, "qrda"))):
         params = libqasg.make_params(1e-4, ETA, DELTA)
         x, h, z = (torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(3))
         g = torch.empty((M, d), dtype=torch.float32, device=dev)
@@ -170,6 +170,23 @@ def sweep_logreg(args):
                       "nnz": int(prob["rowptr"][-1]), "us_per_iteration": us, "us_per_graph_replay": graph_us,
                       "kernel_us": kernel_us,
                       "nnz_x": int((x != 0).sum().item())}), flush=True)
+    # the same iteration with the gradients held in sparse form (touched bits; g stays zero elsewhere)
+    x.zero_(), h.zero_(), z.zero_(), g.zero_()
+    bits = torch.zeros((M, d // 32), dtype=torch.int32, device=dev)
+    t[0] = 0
+
+    def it_touched():
+        t[0] += 1
+        ctx.logreg_grad_csr_touched(*dev_args, n, d, M, prob["shard_row0"], None, B, t[0], x, g, d, bits)
+        ctx.step_touched(libqasg.RULE_RDA, g, d, d, M, t[0], params, bits, x, h, z)
+    us, kernel_us = _timed_iterations(ctx, it_touched, 3, args.steps)
+    graph_us = _timed_graph(it_touched, 3, args.steps) if args.graph else None
+    words = bits.cpu().numpy().view("uint32").ravel()
+    touched = int(sum(bin(int(w)).count("1") for w in words[words != 0]))
+    print(json.dumps({"what": "logreg_csr_touched", "rule": "qrda", "n": n, "d": d, "M": M, "B": B,
+                      "nnz": int(prob["rowptr"][-1]), "touched_last_step": touched,
+                      "us_per_iteration": us, "us_per_graph_replay": graph_us, "kernel_us": kernel_us,
+                      "nnz_x": int((x != 0).sum().item())}), flush=True)
     assert ctx.last_async_status() == libqasg.OK
     ctx.close()
 
@@ -187,6 +204,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--csr-rows", type=int, default=1_000_000)
     ap.add_argument("--graph", action="store_true")
+    ap.add_argument("--csr-only", action="store_true")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "needs a CUDA device"
     if args.what == "step":
