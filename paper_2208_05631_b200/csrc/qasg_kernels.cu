@@ -71,8 +71,29 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
         const double total = chunk_sum.finish(geo.log2_group);
         if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
       };
+  // sparse rows: rows of a tile without a touched entry add +0.0 and are skipped, a warp without any
+  // contributes +0.0 without its butterfly; every other addition is the dense one
+  auto touched_body = [&](const float4 (&v)[kTileRows], uint32_t nibs, bool warp_any, uint32_t) {
+    double s = 0.0;
+    if (warp_any) {
+      if (nibs) {
+        double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+#pragma unroll
+        for (int r = 0; r < kTileRows; ++r)
+          if ((nibs >> (4 * r)) & 15u) {
+            cx += static_cast<double>(fabsf(v[r].x));
+            cy += static_cast<double>(fabsf(v[r].y));
+            cz += static_cast<double>(fabsf(v[r].z));
+            cw += static_cast<double>(fabsf(v[r].w));
+          }
+        s = (cx + cy) + (cz + cw);
+      }
+      s = warp_pair_tree(s);
+    }
+    chunk_sum.add_warp_sum(s);
+  };
   if (kTouched)
-    stream_touched_items(g, touched, geo, j, begin, body, end);
+    stream_touched_items(g, touched, geo, j, begin, touched_body, end);
   else
     stream_items<false>(g, nullptr, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
@@ -115,8 +136,17 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws, const ui
       }
     };
     if (kTouched)
-      walk_touched_tiles(row, reinterpret_cast<const uint8_t*>(touched + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5)),
-                         geo.d, geo.tiles, k0, k1, j, body);
+      walk_touched_tiles(row, touched + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5), geo.d, geo.tiles, k0, k1, j,
+                         [&](const float4 (&v)[kTileRows], uint32_t nibs, bool, uint32_t) {
+#pragma unroll
+                           for (int r = 0; r < kTileRows; ++r)
+                             if ((nibs >> (4 * r)) & 15u) {
+                               best = max(best, __float_as_uint(fabsf(v[r].x)));
+                               best = max(best, __float_as_uint(fabsf(v[r].y)));
+                               best = max(best, __float_as_uint(fabsf(v[r].z)));
+                               best = max(best, __float_as_uint(fabsf(v[r].w)));
+                             }
+                         });
     else
       walk_tiles(row, geo.d, k0, k1, j, body);
     best = __reduce_max_sync(0xffffffffu, best);
@@ -208,8 +238,41 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
           ws.part_cnt[p] = total;
         }
       };
+  // sparse rows: an entry that is not stored is +0.0, inside [-Delta, Delta]: code 0, nothing counted or
+  // summed.  A warp without a touched entry writes its 128 zero code bytes as 32 words.
+  auto touched_body = [&](const float4 (&v)[kTileRows], uint32_t nibs, bool warp_any, uint32_t k) {
+    if (!warp_any) {
+      store_zero_code_words(codes8, k, j >> 5, j & 31, row_words * 4);
+      chunk_sum.add_warp_sum(0.0);
+      return;
+    }
+    double s = 0.0;
+    uint32_t bytes[kTileRows] = {0u, 0u, 0u, 0u};
+    if (nibs) {
+      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+#pragma unroll
+      for (int r = 0; r < kTileRows; ++r)
+        if ((nibs >> (4 * r)) & 15u) {
+          const float4 t = v[r];
+          const float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
+          const float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
+          const float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
+          const float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+          const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;
+          cx += static_cast<double>(fabsf(t.x) * kx);
+          cy += static_cast<double>(fabsf(t.y) * ky);
+          cz += static_cast<double>(fabsf(t.z) * kz);
+          cw += static_cast<double>(fabsf(t.w) * kw);
+          cntf += (kx + ky) + (kz + kw);
+          bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
+        }
+      s = (cx + cy) + (cz + cw);
+    }
+    store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
+    chunk_sum.add_warp_sum(warp_pair_tree(s));
+  };
   if (kMode == 2)
-    stream_touched_items(g, bits, geo, j, begin, body, end);
+    stream_touched_items(g, bits, geo, j, begin, touched_body, end);
   else
     stream_items<kMasked>(g, bits, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
@@ -265,11 +328,29 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
     };
     if (kMode == 2) {
-      TileMask all;
+      // sparse rows: an entry that is not stored is kept with probability |0|/s = 0; its draw is not needed
+      walk_touched_tiles(row, bits + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5), geo.d, geo.tiles, k0, k1, j,
+                         [&](const float4 (&tile)[kTileRows], uint32_t nibs, bool warp_any, uint32_t k) {
+        if (!warp_any) {
+          store_zero_code_words(codes8, k, j >> 5, j & 31, row_words * 4);
+          return;
+        }
+        uint32_t bytes[kTileRows] = {0u, 0u, 0u, 0u};
 #pragma unroll
-      for (int r = 0; r < kTileRows; ++r) all.byte[r] = 0xffu;
-      walk_touched_tiles(row, ind8, geo.d, geo.tiles, k0, k1, j,
-                         [&](const float4 (&tile)[kTileRows], uint32_t k) { body(tile, all, k); });
+        for (int r = 0; r < kTileRows; ++r)
+          if ((nibs >> (4 * r)) & 15u) {
+            const float4 v = tile[r];
+            const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
+            const uint4 w = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), key0, key1);
+            const bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
+            const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
+            const bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
+            const bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
+            bytes[r] = pack4(split_code(v.x, kx), split_code(v.y, ky), split_code(v.z, kz), split_code(v.w, kw));
+            cnt += nonzero_codes(bytes[r]);
+          }
+        store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
+      });
     } else {
       walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, body);
     }

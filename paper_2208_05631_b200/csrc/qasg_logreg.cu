@@ -121,7 +121,8 @@ logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict_
   for (int64_t k = lo + lane; k < hi; k += 32) {
     const uint32_t col = static_cast<uint32_t>(__ldg(colidx + k));
     atomicAdd(row + col, c * __ldg(vals + k));
-    if (kTouched) atomicOr(bits + (col >> 5), 1u << (col & 31u));
+    // hot columns are hit by almost every row: look before the atomic, which same-address traffic serialises
+    if (kTouched && !(__ldcg(bits + (col >> 5)) & (1u << (col & 31u)))) atomicOr(bits + (col >> 5), 1u << (col & 31u));
   }
 }
 
