@@ -100,49 +100,96 @@ logreg_dense_colsum_kernel(const float* __restrict__ X, uint64_t d, uint32_t B, 
   }
 }
 
+// grid (ceil(B / 8), M): a CTA takes 8 minibatch rows of one worker, a warp per row.  Columns below
+// kHotCols are accumulated in shared memory first and reach g with one atomic per CTA and column:
+// with Zipf-like column frequencies nearly every row holds the first few columns, and same-address
+// atomics in L2 serialise.
+constexpr uint32_t kHotCols = 4096;
 template <bool kTouched>
 __global__ void __launch_bounds__(kThreads)
 logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ colidx,
-                  const float* __restrict__ vals, const float* __restrict__ y, uint32_t M, Shards sh,
+                  const float* __restrict__ vals, const float* __restrict__ y, uint64_t d, Shards sh,
                   const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t, const float* __restrict__ x,
                   float* __restrict__ g, uint64_t ld_g, uint32_t* __restrict__ touched, uint64_t touched_words) {
-  const uint32_t warp = (blockIdx.x * kThreads + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= M * B) return;
-  const uint32_t m = warp / B, b = warp - m * B;
-  const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
-  const int64_t lo = rowptr[r], hi = rowptr[r + 1];
-  float acc = 0.f;
-  for (int64_t k = lo + lane; k < hi; k += 32) acc = fmaf(__ldg(vals + k), __ldg(x + __ldg(colidx + k)), acc);
-#pragma unroll
-  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  const float c = logistic_coef(y[r], acc, 1.f / static_cast<float>(B));
+  __shared__ float hot[kHotCols];
+  __shared__ uint32_t hot_bits[kHotCols / 32];
+  const uint32_t m = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t b = blockIdx.x * (kThreads / 32) + warp;
+  for (uint32_t c = threadIdx.x; c < kHotCols; c += kThreads) hot[c] = 0.f;
+  if (threadIdx.x < kHotCols / 32) hot_bits[threadIdx.x] = 0u;
+  __syncthreads();
   float* row = g + static_cast<uint64_t>(m) * ld_g;
-  uint32_t* bits = kTouched ? touched + static_cast<uint64_t>(m) * touched_words : nullptr;
-  for (int64_t k = lo + lane; k < hi; k += 32) {
-    const uint32_t col = static_cast<uint32_t>(__ldg(colidx + k));
-    atomicAdd(row + col, c * __ldg(vals + k));
-    // hot columns are hit by almost every row: look before the atomic, which same-address traffic serialises
-    if (kTouched && !(__ldcg(bits + (col >> 5)) & (1u << (col & 31u)))) atomicOr(bits + (col >> 5), 1u << (col & 31u));
+  if (b < B) {
+    const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
+    const int64_t lo = rowptr[r], hi = rowptr[r + 1];
+    float acc = 0.f;
+    for (int64_t k = lo + lane; k < hi; k += 32) acc = fmaf(__ldg(vals + k), __ldg(x + __ldg(colidx + k)), acc);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+    const float c = logistic_coef(y[r], acc, 1.f / static_cast<float>(B));
+    uint32_t* bits = kTouched ? touched + static_cast<uint64_t>(m) * touched_words : nullptr;
+    for (int64_t k = lo + lane; k < hi; k += 32) {
+      const uint32_t col = static_cast<uint32_t>(__ldg(colidx + k));
+      const float add = c * __ldg(vals + k);
+      const uint32_t bit = 1u << (col & 31u);
+      if (col < kHotCols) {
+        atomicAdd(hot + col, add);
+        if (kTouched) atomicOr(hot_bits + (col >> 5), bit);
+      } else {
+        atomicAdd(row + col, add);
+        // look before the atomic: a set bit needs no second write
+        if (kTouched && !(__ldcg(bits + (col >> 5)) & bit)) atomicOr(bits + (col >> 5), bit);
+      }
+    }
+  }
+  __syncthreads();
+  const uint32_t hot_cols = d < kHotCols ? static_cast<uint32_t>(d) : kHotCols;
+  for (uint32_t c = threadIdx.x; c < hot_cols; c += kThreads) {
+    const float v = hot[c];
+    if (v != 0.f) atomicAdd(row + c, v);
+  }
+  if (kTouched && threadIdx.x < kHotCols / 32 && threadIdx.x < touched_words) {
+    uint32_t* word = touched + static_cast<uint64_t>(m) * touched_words + threadIdx.x;
+    const uint32_t mine = hot_bits[threadIdx.x];
+    if (mine & ~__ldcg(word)) atomicOr(word, mine);
   }
 }
 
-// One thread per word of touched bits: zeroes the entries of g the word marks, then the word.
+// Zeroes the entries of g the bits mark, then the bits.  The M rows of bits are one flat array; a
+// thread takes four words at a time (one 128-bit load; nearly all of them are zero).
+__device__ __forceinline__ void clear_marked(float* __restrict__ g, uint64_t ld_g, uint64_t touched_words, uint64_t d,
+                                             uint64_t w, uint32_t bits) {
+  const uint64_t m = w / touched_words, word = w - m * touched_words;
+  float* base = g + m * ld_g + word * 32;
+  while (bits) {
+    const int b = __ffs(bits) - 1;
+    if (word * 32 + b < d) base[b] = 0.f;  // a stray bit past d marks nothing
+    bits &= bits - 1;
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 touched_clear_kernel(float* __restrict__ g, uint64_t ld_g, uint32_t M, uint32_t* __restrict__ touched,
                      uint64_t touched_words, uint64_t d) {
-  const uint64_t total = static_cast<uint64_t>(M) * touched_words;
-  for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < total;
-       w += static_cast<uint64_t>(gridDim.x) * kThreads) {
-    uint32_t bits = touched[w];
-    if (!bits) continue;
-    const uint64_t m = w / touched_words, word = w - m * touched_words;
-    float* base = g + m * ld_g + word * 32;
-    while (bits) {
-      const int b = __ffs(bits) - 1;
-      if (word * 32 + b < d) base[b] = 0.f;  // a stray bit past d marks nothing
-      bits &= bits - 1;
+  const uint64_t total = static_cast<uint64_t>(M) * touched_words, quads = total >> 2;
+  const uint64_t tid = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+  uint4* t4 = reinterpret_cast<uint4*>(touched);
+  for (uint64_t q = tid; q < quads; q += stride) {
+    const uint4 v = t4[q];
+    if (!(v.x | v.y | v.z | v.w)) continue;
+    if (v.x) clear_marked(g, ld_g, touched_words, d, 4 * q, v.x);
+    if (v.y) clear_marked(g, ld_g, touched_words, d, 4 * q + 1, v.y);
+    if (v.z) clear_marked(g, ld_g, touched_words, d, 4 * q + 2, v.z);
+    if (v.w) clear_marked(g, ld_g, touched_words, d, 4 * q + 3, v.w);
+    t4[q] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  for (uint64_t w = 4 * quads + tid; w < total; w += stride) {
+    const uint32_t bits = touched[w];
+    if (bits) {
+      clear_marked(g, ld_g, touched_words, d, w, bits);
+      touched[w] = 0u;
     }
-    touched[w] = 0u;
   }
 }
 
@@ -171,14 +218,13 @@ int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float*
                       const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
                       uint64_t ld_g, const LaunchShape&, cudaStream_t stream, uint32_t* touched) {
   const Shards sh = make_shards(shard_row0_host, M);
-  const uint64_t warps = static_cast<uint64_t>(M) * B;
-  const unsigned grid = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
+  const dim3 grid((B + kThreads / 32 - 1) / (kThreads / 32), M);
   if (touched) {
-    logreg_csr_kernel<true><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, M, sh, batch_rows, B, t, x, g,
+    logreg_csr_kernel<true><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, d, sh, batch_rows, B, t, x, g,
                                                           ld_g, touched, (d + 31) >> 5);
   } else {
     cudaMemset2DAsync(g, ld_g * sizeof(float), 0, d * sizeof(float), M, stream);
-    logreg_csr_kernel<false><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, M, sh, batch_rows, B, t, x, g,
+    logreg_csr_kernel<false><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, d, sh, batch_rows, B, t, x, g,
                                                            ld_g, nullptr, 0);
   }
   return 1;
@@ -187,8 +233,8 @@ int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float*
 int launch_touched_clear(float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint32_t* touched,
                          const LaunchShape& shape, cudaStream_t stream) {
   const uint64_t words = (d + 31) >> 5;
-  const uint64_t ctas = (static_cast<uint64_t>(M) * words + kThreads - 1) / kThreads;
-  const uint64_t cap = static_cast<uint64_t>(shape.sm_count) * 32;
+  const uint64_t ctas = (static_cast<uint64_t>(M) * words / 4 + kThreads) / kThreads;
+  const uint64_t cap = static_cast<uint64_t>(shape.sm_count) * 8;
   touched_clear_kernel<<<static_cast<unsigned>(ctas < cap ? ctas : cap), kThreads, 0, stream>>>(g, ld_g, M, touched,
                                                                                               words, d);
   return 1;
