@@ -109,6 +109,109 @@ def threshold_quantize(v, coef=0.75):
 
 
 # ----------------------------------------------------------------------------------
+# Exact optimal threshold (Section 3.4: rank the components, try each as the threshold)
+# ----------------------------------------------------------------------------------
+SCAN_WARP = 32
+SCAN_BLOCK = SCAN_WARP * SCAN_WARP   # 1024
+
+
+def _doubling_scan(x):
+    """Inclusive prefix sums along the last axis by recursive doubling: at step s = 1, 2, 4, ...
+    every element i >= s becomes x[i - s] + x[i], all at once."""
+    x = np.array(x, dtype=F64)
+    s = 1
+    while s < x.shape[-1]:
+        y = x.copy()
+        y[..., s:] = x[..., :-s] + x[..., s:]
+        x = y
+        s *= 2
+    return x
+
+
+def _block_scan(x):
+    """Inclusive prefix sums of blocks of 1024 (last axis): doubling scan inside each run of 32,
+    doubling scan of the 32 run totals, then (sum of the runs before) + (value inside the run)."""
+    lead = x.shape[:-1]
+    runs = _doubling_scan(np.asarray(x, dtype=F64).reshape(lead + (SCAN_WARP, SCAN_WARP)))
+    totals = _doubling_scan(runs[..., -1])
+    before = np.concatenate([np.zeros(lead + (1,), dtype=F64), totals[..., :-1]], axis=-1)
+    return (before[..., None] + runs).reshape(lead + (SCAN_BLOCK,))
+
+
+def canonical_prefix(a):
+    """Inclusive prefix sums P_i = a_0 + ... + a_i of a non-negative vector in fp64, in one fixed
+    order (like `canonical_sum`, a convention of this library so that every implementation gets the
+    same bits): blocks of 1024 elements scanned by `_block_scan`; the block totals of each group of
+    1024 blocks scanned the same way; the group totals added one after the other;
+    P_i = (sum of the groups before + sum of the blocks before inside the group) + value in the block."""
+    a = np.asarray(a, dtype=F64).ravel()
+    n = a.size
+    blocks = -(-n // SCAN_BLOCK)
+    groups = -(-blocks // SCAN_BLOCK)
+    buf = np.zeros(groups * SCAN_BLOCK * SCAN_BLOCK, dtype=F64)
+    buf[:n] = a
+    inner = _block_scan(buf.reshape(groups, SCAN_BLOCK, SCAN_BLOCK))          # [g, b, i]
+    block_scan = _block_scan(inner[..., -1])                                   # [g, b] inclusive over blocks
+    blocks_before = np.concatenate([np.zeros((groups, 1)), block_scan[:, :-1]], axis=1)
+    groups_before = np.zeros(groups, dtype=F64)
+    acc = F64(0.0)
+    for gi in range(groups):
+        groups_before[gi] = acc
+        acc = acc + block_scan[gi, -1]
+    base = groups_before[:, None] + blocks_before
+    return (base[..., None] + inner).reshape(-1)[:n]
+
+
+def optimal_threshold(v):
+    """Delta* = argmax_Delta (sum_{I_Delta} |v_i|)^2 / |I_Delta|, I_Delta = {i : |v_i| > Delta}
+    (Section 3.4), by the paper's procedure: rank the |v_i| and try every component as the threshold.
+
+    With a_0 >= a_1 >= ... the ranked magnitudes, the candidate sets are the k largest for every k
+    with a_{k-1} > a_k (a strict drop: equal components fall on the same side of any threshold) and
+    a_{k-1} > 0, plus k = d when a_{d-1} > 0.  The objective of k is F_k = (P_{k-1} * P_{k-1}) / k in
+    fp64 with P the canonical prefix sums; the smallest k among equal maxima wins.  The threshold
+    returned is the largest component outside the set, Delta* = a_k (0 when k = d or nothing is
+    non-zero), so that Q_{Delta*} with its strict comparisons selects exactly those k.
+    Returns (Delta* fp32, k int)."""
+    a = np.sort(np.abs(np.asarray(v, dtype=F32).ravel()))[::-1]
+    d = a.size
+    prefix = canonical_prefix(a.astype(F64))
+    objective = (prefix * prefix) / np.arange(1, d + 1, dtype=F64)
+    drop = np.ones(d, dtype=bool)
+    drop[:-1] = a[:-1] > a[1:]
+    valid = drop & (a > 0)
+    if not valid.any():
+        return F32(0.0), 0
+    i = int(np.argmax(np.where(valid, objective, -1.0)))     # first maximum
+    return (a[i + 1] if i + 1 < d else F32(0.0)), i + 1
+
+
+def quantize_at_threshold(v, delta):
+    """Q_Delta(v) for a given fp32 Delta: codes by the strict fp32 comparisons of Section 3.4 and
+    s*_Delta = mean of |v_i| over I_Delta (canonical sum).  Returns (tern, s fp32, |I_Delta|)."""
+    v = np.asarray(v, dtype=F32).ravel()
+    delta = F32(delta)
+    pos = v > delta
+    neg = v < -delta
+    tern = pos.astype(np.int8) - neg.astype(np.int8)
+    selected = pos | neg
+    n = int(np.count_nonzero(selected))
+    if n == 0:
+        return tern, F32(0.0), 0
+    picked = canonical_sum(np.where(selected, np.abs(v), F32(0.0)))
+    return tern, F32(picked / F64(n)), n
+
+
+def optimal_threshold_quantize(v):
+    """Q_{Delta*}(v): the threshold quantizer at the exact optimal threshold.
+    Returns (tern, s fp32, Delta* fp32, |I_{Delta*}|)."""
+    delta, k = optimal_threshold(v)
+    tern, scale, n = quantize_at_threshold(v, delta)
+    assert n == k
+    return tern, scale, delta, n
+
+
+# ----------------------------------------------------------------------------------
 # Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
 # 1, 2, 3", SC'11) and the stochastic ternary quantizer
 # ----------------------------------------------------------------------------------

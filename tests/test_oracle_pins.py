@@ -539,3 +539,82 @@ def test_touched_step_is_the_dense_step_of_the_stored_entries():
                 assert a["quant"]["thresholds"][m] == np.float32(0.75 * exact / d)
     with pytest.raises(ValueError):
         O.densify_touched(vals, touched[:, :-1])
+
+
+# ------------------------------------------------------------------ exact optimal threshold
+def test_canonical_prefix_is_a_prefix_sum():
+    rng = np.random.default_rng(51)
+    # exact on integers (every partial sum representable), across block, group and group-sequence levels
+    for d in (1, 31, 33, 1023, 1025, 5000, (1 << 20) + 4321, (1 << 21) + 77):
+        a = rng.integers(0, 1 << 16, size=d).astype(np.float64)
+        assert np.array_equal(O.canonical_prefix(a), np.cumsum(a))
+    a = np.abs(rng.standard_normal(70_001)) * 10.0 ** rng.integers(-5, 5, size=70_001)
+    got = O.canonical_prefix(a)
+    want = np.array([math.fsum(a[: i + 1]) for i in range(0, 70_001, 997)])
+    assert np.all(np.abs(got[::997] - want) <= 64 * 2.0 ** -53 * want)
+    assert np.all(np.diff(got) >= 0)
+
+
+def _best_ternary_error(v):
+    """Eq. of the quantization objective by exhaustive search: min over tern in {-1,0,1}^d and s >= 0
+    of ||v - s*tern||^2 (for a given tern the best s is max(0, <v, tern>/|tern|_0))."""
+    import itertools
+    v = v.astype(np.float64)
+    best = float((v * v).sum())
+    for tern in itertools.product((-1.0, 0.0, 1.0), repeat=v.size):
+        t = np.array(tern)
+        nnz = np.count_nonzero(t)
+        if nnz == 0:
+            continue
+        s = max(0.0, float(v @ t) / nnz)
+        best = min(best, float(((v - s * t) ** 2).sum()))
+    return best
+
+
+def test_optimal_threshold_attains_the_minimum_over_all_ternary_vectors():
+    rng = np.random.default_rng(52)
+    for d in (1, 2, 3, 5, 7):
+        for _ in range(6):
+            v = rng.standard_normal(d).astype(np.float32)
+            if d > 2 and rng.random() < 0.3:
+                v[1] = v[0]                                   # a tie
+            tern, s, delta, n = O.optimal_threshold_quantize(v)
+            s_exact = np.abs(v.astype(np.float64))[tern != 0].sum() / n
+            err = float(((v.astype(np.float64) - s_exact * tern) ** 2).sum())
+            assert err <= _best_ternary_error(v) * (1 + 1e-12) + 1e-300
+            assert float(s) == pytest.approx(s_exact, rel=1e-6)
+            assert n == int((np.abs(v) > delta).sum())
+            assert delta == 0 or delta in np.abs(v)           # a component, as the paper's procedure has it
+
+
+def test_optimal_threshold_beats_every_component_taken_as_threshold():
+    rng = np.random.default_rng(53)
+    for d, scale in ((50, 1.0), (1000, 1e-3), (4097, 30.0)):
+        v = (rng.standard_normal(d) * scale).astype(np.float32)
+        v[rng.integers(0, d, size=d // 10)] = 0.0
+        v[5] = v[6] = v[7]
+        delta, k = O.optimal_threshold(v)
+        a = np.abs(v).astype(np.float64)
+
+        def objective(thr):
+            sel = a[a > thr]
+            return math.fsum(sel) ** 2 / sel.size if sel.size else 0.0
+        best = max(objective(float(c)) for c in np.unique(np.concatenate([a, [0.0]])))
+        assert objective(float(delta)) >= best * (1 - 1e-13)
+        assert k == int((a > float(delta)).sum()) and k > 0
+    assert O.optimal_threshold(np.zeros(9, dtype=np.float32)) == (np.float32(0.0), 0)
+    # all equal and non-zero: everything is kept, the threshold falls to 0
+    assert O.optimal_threshold(np.full(9, -2.5, dtype=np.float32)) == (np.float32(0.0), 9)
+
+
+def test_optimal_threshold_for_gaussian_data_is_about_0p6_sigma():
+    # Section 3.5 quotes Delta* ~ 0.6 sigma for N(0, sigma^2); the 0.75 * E|v| rule approximates it.
+    rng = np.random.default_rng(54)
+    v = (rng.standard_normal(300_000) * 2.0).astype(np.float32)
+    delta, k = O.optimal_threshold(v)
+    assert 0.55 * 2.0 < float(delta) < 0.67 * 2.0
+    _, _, approx, _ = O.threshold_quantize(v)
+    assert abs(float(approx) - float(delta)) < 0.06 * 2.0
+    tern, s, d2, n = O.optimal_threshold_quantize(v)
+    got = (np.abs(v.astype(np.float64))[tern != 0].sum()) ** 2 / n
+    assert got == pytest.approx(_optimal_threshold_objective(v), rel=1e-12)
