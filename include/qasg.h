@@ -278,6 +278,24 @@ qasg_status qasg_step_touched(qasg_ctx* ctx, qasg_rule rule, const float* g, uin
                               float* x, float* h, float* z, uint32_t* codes_out, float* scales_out,
                               void* stream);
 
+/* The threshold quantizer at the exact optimal threshold of Section 3.4 instead of the 0.75 * mean|g|
+ * rule of Section 3.5: per worker, the magnitudes are ranked (radix sort), every component is taken as
+ * the candidate threshold, and the one that maximises (sum_{I_Delta} |g_i|)^2 / |I_Delta| is kept
+ * (candidates are the strict drops of the ranked magnitudes, equal maxima resolve to the smaller set,
+ * Delta* is the largest component outside the chosen set, 0 if everything non-zero is kept).  Codes,
+ * scales (mean kept magnitude) and counts (|I_Delta*|) then as for qasg_quantize_pack.  O(d log d) work
+ * and 12 passes over the row: an accuracy reference for the rule, not a per-step path.
+ *   params        quantizer must be QASG_Q_THRESHOLD; thr_coef is not used.
+ *   scratch       device, 256-byte aligned, at least qasg_optimal_scratch_bytes(d) bytes (about 8.3 d),
+ *                 used for one worker after the other; contents undefined afterwards.
+ *   d             below 2^31 (qasg_optimal_scratch_bytes returns 0 beyond).
+ * Non-finite gradients: status NONFINITE, outputs unspecified. */
+uint64_t qasg_optimal_scratch_bytes(uint64_t d);
+qasg_status qasg_quantize_pack_optimal(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                                       const qasg_params* params, uint32_t* codes, float* scales,
+                                       float* thresholds, uint64_t* counts, void* scratch,
+                                       uint64_t scratch_bytes, void* stream);
+
 /* The threshold quantizer of qasg_quantize_pack for callers that cannot allocate device
  * memory.  (The paper has no counterpart: this entry point exists for the sake of its
  * callers, not of the method.)

@@ -33,7 +33,7 @@ enum KernelId {
   kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
   kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kAvgAbsSum, kAvgAbsMax,
   kAvgThresholdCodes, kAvgStochasticCodes, kSelectStats, kIndicatorOr, kTouchedClear, kLogregCsrTouched,
-  kKernelIdCount
+  kOptimalThreshold, kKernelIdCount
 };
 static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
 
@@ -410,6 +410,36 @@ qasg_status qasg_step_touched(qasg_ctx* ctx, qasg_rule rule, const float* g, uin
   return leave();
 }
 
+uint64_t qasg_optimal_scratch_bytes(uint64_t d) { return (d >= 1 && d < (1ull << 31)) ? optimal_scratch_bytes(d) : 0; }
+
+qasg_status qasg_quantize_pack_optimal(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                                       const qasg_params* params, uint32_t* codes, float* scales,
+                                       float* thresholds, uint64_t* counts, void* scratch, uint64_t scratch_bytes,
+                                       void* stream) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, false);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (!codes || !scales || !scratch || params->quantizer != QASG_Q_THRESHOLD || d >= (1ull << 31))
+    return QASG_ERR_INVALID_ARG;
+  if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(scratch) & 255u)) return QASG_ERR_ALIGNMENT;
+  if (scratch_bytes < optimal_scratch_bytes(d)) return QASG_ERR_WORKSPACE;
+  if ((st = enter(ctx)) != QASG_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  for (uint32_t m = 0; m < M; ++m) {  // one row after the other through the same scratch
+    Launch l(ctx, kOptimalThreshold, s);
+    l += launch_optimal_threshold(g + static_cast<uint64_t>(m) * ld_g, d, scratch, ctx->ws.thresholds + m,
+                                  thresholds ? thresholds + m : nullptr, nullptr, ctx->ws.status, s);
+  }
+  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
+  {
+    Launch l(ctx, kThresholdCodes, s);
+    l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, reinterpret_cast<unsigned long long*>(counts),
+                                ctx->shape, s);
+  }
+  return leave();
+}
+
 qasg_status qasg_requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                             uint64_t t, const qasg_params* params, uint32_t* qcodes, float* qscale,
                             float* qthreshold, uint64_t* qcount, void* stream) {
@@ -676,7 +706,7 @@ const char* qasg_kernel_name(int id) {
       "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
       "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr", "avg_abs_sum",
       "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes", "select_stats", "indicator_or",
-      "touched_clear", "logreg_csr_touched"};
+      "touched_clear", "logreg_csr_touched", "optimal_threshold"};
   return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
 }
 

@@ -124,6 +124,13 @@ int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float*
 int launch_touched_clear(float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint32_t* touched,
                          const LaunchShape& shape, cudaStream_t stream);
 
+// Exact optimal threshold of one row (rank, prefix sums, first maximum of (sum of the k largest)^2 / k).
+// scratch: optimal_scratch_bytes(d) bytes of device memory, 256-byte aligned; d < 2^31.
+// Writes Delta* to ws_threshold (and threshold_out, kept_out = k if not null).
+uint64_t optimal_scratch_bytes(uint64_t d);
+int launch_optimal_threshold(const float* row, uint64_t d, void* scratch, float* ws_threshold, float* threshold_out,
+                             unsigned long long* kept_out, unsigned int* status, cudaStream_t stream);
+
 void query_launch_shape(LaunchShape* shape);
 
 }  // namespace qasg

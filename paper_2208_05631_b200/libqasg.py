@@ -28,6 +28,7 @@ EXPORTS = [
     "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static", "qasg_requantize", "qasg_step_double",
     "qasg_select_quantize_pack", "qasg_indicator_or", "qasg_step_select",
     "qasg_logreg_grad_csr_touched", "qasg_quantize_pack_touched", "qasg_step_touched",
+    "qasg_optimal_scratch_bytes", "qasg_quantize_pack_optimal",
 ]
 STATIC_MAX_WORKERS = 16
 KERNEL_COUNT = 24
@@ -88,6 +89,9 @@ def load():
                                                  u64, vp, vp, u64, vp, vp]
     lib.qasg_quantize_pack_touched.argtypes = [vp, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp]
     lib.qasg_step_touched.argtypes = [vp, i32, vp, u64, u64, u32, u64, pp, vp, vp, vp, vp, vp, vp, vp]
+    lib.qasg_optimal_scratch_bytes.argtypes = [u64]
+    lib.qasg_optimal_scratch_bytes.restype = u64
+    lib.qasg_quantize_pack_optimal.argtypes = [vp, vp, u64, u64, u32, pp, vp, vp, vp, vp, vp, u64, vp]
     lib.qasg_last_async_status.argtypes = [vp, vp]
     lib.qasg_launch_count.argtypes = [vp]
     lib.qasg_launch_count.restype = u64
@@ -240,6 +244,14 @@ class Context:
                                         _ptr(touched), _ptr(x), _ptr(h), _ptr(z), _ptr(codes_out),
                                         _ptr(scales_out), _stream(stream)), "qasg_step_touched")
 
+    def quantize_pack_optimal(self, g, d, ld_g, M, params, codes, scales, scratch, thresholds=None, counts=None,
+                              stream=None):
+        """scratch: a device tensor of at least optimal_scratch_bytes(d) bytes."""
+        _check(load().qasg_quantize_pack_optimal(self._h, _ptr(g), d, ld_g, M, ctypes.byref(params), _ptr(codes),
+                                                 _ptr(scales), _ptr(thresholds), _ptr(counts), _ptr(scratch),
+                                                 scratch.numel() * scratch.element_size(), _stream(stream)),
+               "qasg_quantize_pack_optimal")
+
     def last_async_status(self, stream=None):
         return int(load().qasg_last_async_status(self._h, _stream(stream)))
 
@@ -256,6 +268,10 @@ class Context:
 
     def launch_count(self):
         return int(load().qasg_launch_count(self._h))
+
+
+def optimal_scratch_bytes(d):
+    return int(load().qasg_optimal_scratch_bytes(d))
 
 
 def quantize_pack_static(device, g, d, ld_g, M, thr_coef, codes, scales, thresholds=None, counts=None,
