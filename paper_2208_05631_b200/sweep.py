@@ -2,7 +2,8 @@
 
   python -m paper_2208_05631_b200.sweep step   [--quantizer threshold|stochastic] [--double-quant] [--select]
                                                [--min-log2-d 20] [--max-log2-d 28] [--workers 2,4,8,16,32]
-  python -m paper_2208_05631_b200.sweep logreg [--steps 50] [--graph]
+  python -m paper_2208_05631_b200.sweep logreg [--steps 50] [--graph] [--csr-only]
+  python -m paper_2208_05631_b200.sweep optimal [--min-log2-d 20] [--max-log2-d 28] [--workers 8]
 
 `step`   - the fused step over d in {2^20 .. 2^28} x M in {2, 4, 8, 16, 32} simulated workers,
            N(0,1) gradients, both update rules (the paper uses 2-4 workers; this is the scaling
@@ -11,6 +12,10 @@
 `logreg` - the two L1-logistic-regression workloads: gradient kernel + fused step per iteration.
            dense: X 65536 x 4096, 8 workers, minibatch 512; sparse: 10^6 x 2^24 CSR, ~80 non-zeros
            per row, 16 workers, minibatch 1024.
+
+`optimal` - the threshold quantizer with the 0.75 * mean|g| rule against the exact optimal threshold
+           (sort + prefix sums): time of each and the relative quantization error each reaches, on
+           N(0,1) and on Student-t(3) gradients.
 
 `--graph` captures one iteration (fixed step index) in a CUDA graph and replays it: every call of the
 library only enqueues kernels on the given stream, so a launch-bound loop can be replayed without
@@ -191,9 +196,49 @@ def sweep_logreg(args):
     ctx.close()
 
 
+def sweep_optimal(args):
+    """The 0.75 * mean|g| rule against the exact optimal threshold: time of each quantizer and the
+    quantization error ||g - s*tern||^2 / ||g||^2 = 1 - n s^2 / ||g||^2 each one reaches."""
+    dev = torch.device("cuda", 0)
+    M = int(args.workers.split(",")[0])
+    for log2_d in range(args.min_log2_d, args.max_log2_d + 1, 2):
+        d = 1 << log2_d
+        ctx = libqasg.Context(d, M, device=0)
+        scratch = torch.empty(libqasg.optimal_scratch_bytes(d), dtype=torch.uint8, device=dev)
+        params = libqasg.make_params(LAM, ETA, DELTA)
+        flush = torch.zeros(64 << 20, dtype=torch.float32, device=dev)      # 256 MB > L2
+        for name, gen in (("normal", inputs.normal_gradients), ("student_t3", inputs.student_t_gradients)):
+            g = gen(d, M, seed=4, device=dev)
+            sq = (g.double() ** 2).sum(dim=1)
+            codes = torch.empty((M, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+            out = {}
+            for which in ("rule", "optimal"):
+                scales = torch.zeros(M, dtype=torch.float32, device=dev)
+                thr = torch.zeros(M, dtype=torch.float32, device=dev)
+                cnt = torch.zeros(M, dtype=torch.int64, device=dev)
+
+                def run():
+                    if which == "rule":
+                        ctx.quantize_pack(g, d, d, M, 1, params, codes, scales, thr, cnt)
+                    else:
+                        ctx.quantize_pack_optimal(g, d, d, M, params, codes, scales, scratch, thr, cnt)
+                run()
+                ms_median, _ = _time_calls(run, args.reps, flush)
+                err = 1.0 - cnt.double() * scales.double() ** 2 / sq
+                out[which] = {"ms_median": ms_median,
+                              "threshold_over_mean_abs": (thr.double() / g.abs().double().mean(dim=1)).tolist(),
+                              "kept_fraction": (cnt.double() / d).tolist(),
+                              "relative_sq_error": err.tolist()}
+            print(json.dumps({"what": "optimal_vs_rule", "input": name, "d": d, "M": M, **out}), flush=True)
+            del g
+        assert ctx.last_async_status() == libqasg.OK
+        ctx.close()
+        del scratch
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["step", "logreg"])
+    ap.add_argument("what", choices=["step", "logreg", "optimal"])
     ap.add_argument("--quantizer", default="threshold", choices=["threshold", "stochastic"])
     ap.add_argument("--double-quant", action="store_true")
     ap.add_argument("--select", action="store_true")
@@ -207,7 +252,9 @@ def main():
     ap.add_argument("--csr-only", action="store_true")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "needs a CUDA device"
-    if args.what == "step":
+    if args.what == "optimal":
+        sweep_optimal(args)
+    elif args.what == "step":
         sweep_step(args)
     else:
         sweep_logreg(args)
