@@ -897,8 +897,9 @@ __host__ __device__ inline size_t select_smem_bytes(uint32_t M) {
   return static_cast<size_t>(M) * (kSelectDoublesPerWorker * sizeof(double) + 2 * sizeof(uint32_t));
 }
 
+// QRDA keeps two state tiles of z in registers next to the two gradient tiles: two CTAs per SM, not three.
 template <int kRule, bool kStochastic>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, kRule == 0 ? 3 : 2)
 select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __restrict__ x,
                     const float* __restrict__ hz, SelectScalars sc, float coef, Workspace ws,
                     uint32_t* __restrict__ indicators, float* __restrict__ thresholds_out,
@@ -919,18 +920,28 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
     for (uint32_t m = j; m < 2 * M; m += kThreads) sm_cnt[m] = 0u;  // counts and maxima
     __syncthreads();
     uint32_t pending = 0, pushed = 0;
+    // The chunk is one stream of gradient tiles, (tile k, worker 0..M-1), (tile k+1, worker 0..M-1), ...:
+    // the next one is always in flight, and the state of tile k+1 is requested while the last worker of
+    // tile k is processed.  Of x only "non-zero" is kept (one bit per coordinate).
+    float4 ga[kTileRows], gb[kTileRows], xn[kTileRows], zc[kTileRows], zn[kTileRows];
+    bool a_cur = true;
+    auto whole_tile = [&](uint32_t k) { return static_cast<uint64_t>(k + 1) * kTile <= geo.d; };
+    load_state_tile(x, geo.d, k0, j, whole_tile(k0), xn);
+    if (kRule == 1) load_state_tile(hz, geo.d, k0, j, whole_tile(k0), zn);
+    load_tile(g, static_cast<uint64_t>(k0) * kTile, geo.d, j, ga);
     for (uint32_t k = k0; k < k1; ++k) {
       const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
-      const bool whole = tile_base + kTile <= geo.d;
-      float4 xv[kTileRows], hv[kTileRows];
-      load_state_tile(x, geo.d, k, j, whole, xv);
-      if (kRule == 1) {
-        load_state_tile(hz, geo.d, k, j, whole, hv);
-      } else {  // the QCMD test reads no accumulator
+      uint32_t xmask = 0u;  // bit 4r + q: x != 0 at coordinate q of the thread's float4 of row r
 #pragma unroll
-        for (int r = 0; r < kTileRows; ++r) hv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int r = 0; r < kTileRows; ++r) {
+        xmask |= (xn[r].x != 0.f ? 1u : 0u) << (4 * r);
+        xmask |= (xn[r].y != 0.f ? 2u : 0u) << (4 * r);
+        xmask |= (xn[r].z != 0.f ? 4u : 0u) << (4 * r);
+        xmask |= (xn[r].w != 0.f ? 8u : 0u) << (4 * r);
+        if (kRule == 1) zc[r] = zn[r];
       }
-      // one worker's share of this tile: indicator bits, selected |g| into the fixed-order sum
+      // One worker's share of this tile: indicator bits, selected |g| into the fixed-order sum.
+      // Coordinates at or past d read as x = z = g = +0.0 and are never selected (lambda >= 0).
       auto worker_tile = [&](const float4 (&gv)[kTileRows], uint32_t m) {
         uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words);
         double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
@@ -939,11 +950,18 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
 #pragma unroll
         for (int r = 0; r < kTileRows; ++r) {
           const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
-          const bool bx = (whole || i0 < geo.d) && selects<kRule>(gv[r].x, xv[r].x, hv[r].x, sc);
-          const bool by = (whole || i0 + 1 < geo.d) && selects<kRule>(gv[r].y, xv[r].y, hv[r].y, sc);
-          const bool bz = (whole || i0 + 2 < geo.d) && selects<kRule>(gv[r].z, xv[r].z, hv[r].z, sc);
-          const bool bw = (whole || i0 + 3 < geo.d) && selects<kRule>(gv[r].w, xv[r].w, hv[r].w, sc);
-          const float sx = bx ? 1.f : 0.f, sy = by ? 1.f : 0.f, sz = bz ? 1.f : 0.f, sw = bw ? 1.f : 0.f;
+          bool bx, by, bz, bw;
+          if (kRule == 0) {
+            bx = fabsf(gv[r].x) > sc.lambda, by = fabsf(gv[r].y) > sc.lambda;
+            bz = fabsf(gv[r].z) > sc.lambda, bw = fabsf(gv[r].w) > sc.lambda;
+          } else {
+            bx = fabsf(__fadd_rn(zc[r].x, gv[r].x)) > sc.lambda_t, by = fabsf(__fadd_rn(zc[r].y, gv[r].y)) > sc.lambda_t;
+            bz = fabsf(__fadd_rn(zc[r].z, gv[r].z)) > sc.lambda_t, bw = fabsf(__fadd_rn(zc[r].w, gv[r].w)) > sc.lambda_t;
+          }
+          const uint32_t nib = ((xmask >> (4 * r)) & 15u) | static_cast<uint32_t>(bx) | (static_cast<uint32_t>(by) << 1) |
+                               (static_cast<uint32_t>(bz) << 2) | (static_cast<uint32_t>(bw) << 3);
+          const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
+          const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
           if (!kStochastic) {
             cx += static_cast<double>(fabsf(gv[r].x) * sx);
             cy += static_cast<double>(fabsf(gv[r].y) * sy);
@@ -957,8 +975,6 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
           }
           cntf += (sx + sy) + (sz + sw);
           // two adjacent threads share an indicator byte; the even one writes it (zeros past d)
-          const uint32_t nib = static_cast<uint32_t>(bx) | (static_cast<uint32_t>(by) << 1) |
-                               (static_cast<uint32_t>(bz) << 2) | (static_cast<uint32_t>(bw) << 3);
           const uint32_t upper = __shfl_down_sync(0xffffffffu, nib, 1);
           if ((j & 1) == 0 && (i0 >> 3) < ind_words * 4) ind8[i0 >> 3] = static_cast<uint8_t>(nib | (upper << 4));
         }
@@ -972,17 +988,24 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
         const uint32_t cnt = __reduce_add_sync(0xffffffffu, static_cast<uint32_t>(cntf));
         if (lane == 0 && cnt) atomicAdd(&sm_cnt[m], cnt);
       };
-      // walk the workers with the next worker's tile in flight
-      float4 ga[kTileRows], gb[kTileRows];
-      load_tile(g, tile_base, geo.d, j, ga);
-      uint32_t m = 0;
-      while (true) {
-        if (m + 1 < M) load_tile(g + static_cast<uint64_t>(m + 1) * geo.ld, tile_base, geo.d, j, gb);
-        worker_tile(ga, m);
-        if (++m >= M) break;
-        if (m + 1 < M) load_tile(g + static_cast<uint64_t>(m + 1) * geo.ld, tile_base, geo.d, j, ga);
-        worker_tile(gb, m);
-        if (++m >= M) break;
+      for (uint32_t m = 0; m < M; ++m) {
+        auto prefetch = [&](float4 (&nxt)[kTileRows]) {
+          if (m + 1 < M) {
+            load_tile(g + static_cast<uint64_t>(m + 1) * geo.ld, tile_base, geo.d, j, nxt);
+          } else if (k + 1 < k1) {
+            load_tile(g, tile_base + kTile, geo.d, j, nxt);
+            load_state_tile(x, geo.d, k + 1, j, whole_tile(k + 1), xn);
+            if (kRule == 1) load_state_tile(hz, geo.d, k + 1, j, whole_tile(k + 1), zn);
+          }
+        };
+        if (a_cur) {
+          prefetch(gb);
+          worker_tile(ga, m);
+        } else {
+          prefetch(ga);
+          worker_tile(gb, m);
+        }
+        a_cur = !a_cur;
       }
       ++pending;
       if (!kStochastic && (pending == kSelectBatch || k + 1 == k1)) {
@@ -1142,7 +1165,7 @@ int launch_select_stats(int rule, bool stochastic, const float* g, const Geometr
                         uint32_t* indicators, float* thresholds_out, unsigned long long* selected_out,
                         const LaunchShape& shape, cudaStream_t stream) {
   const size_t smem = select_smem_bytes(geo.M);
-  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * 3;
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * (rule == 0 ? 3 : 2);
   const unsigned grid = static_cast<unsigned>(geo.chunks < resident ? geo.chunks : resident);
 #define QASG_SELECT(R, S)                                                                                    \
   do {                                                                                                       \
