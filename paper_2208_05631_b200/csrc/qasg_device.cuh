@@ -161,29 +161,33 @@ __device__ __forceinline__ void walk_tiles(const float* __restrict__ row, uint64
   }
 }
 
-// The indicator bytes a thread needs for its four rows of tile k (two threads share a byte).
+// The indicator bits of tile k as a warp needs them (its 128 columns of the 4 rows = 16 words): lane
+// l < 16 holds the word of row l>>2, quarter l&3, the other lanes 0; a thread's nibble of row r comes
+// out of the holder's word by one shuffle (all lanes of the warp must call nibble together).
 struct TileMask {
-  uint32_t byte[kTileRows];
-  __device__ __forceinline__ uint32_t nibble(int r, int j) const { return (byte[r] >> (4 * (j & 1))) & 15u; }
-};
-__device__ __forceinline__ void load_tile_mask(const uint8_t* __restrict__ ind8, uint64_t d, uint32_t k, int j,
-                                               TileMask& mask) {
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) {
-    const uint64_t i0 = static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j;
-    mask.byte[r] = i0 < d ? static_cast<uint32_t>(__ldg(ind8 + (i0 >> 3))) : 0u;
+  uint32_t word;
+  __device__ __forceinline__ uint32_t nibble(int r, int j) const {
+    const int lane = j & 31;
+    const uint32_t w = __shfl_sync(0xffffffffu, word, r * 4 + (lane >> 3));
+    return (w >> (4 * (lane & 7))) & 15u;
   }
+};
+// words: the worker's row of indicator words (bits at or past d are 0 there).
+__device__ __forceinline__ void load_tile_mask(const uint32_t* __restrict__ words, uint64_t d, uint32_t k, int j,
+                                               TileMask& mask) {
+  const int lane = j & 31, warp = j >> 5;
+  const uint64_t idx = static_cast<uint64_t>(k) * (kTile / 32) + (lane >> 2) * (kTileCols / 32) + 4 * warp + (lane & 3);
+  mask.word = (lane < 16 && idx * 32 < d) ? __ldg(words + idx) : 0u;
 }
 
 // walk_tiles with the tile's indicator bytes travelling along: body(tile_values, mask, k).
 // Without a mask (kMasked false) no byte is loaded and every nibble reads as selected.
 template <bool kMasked, class Body>
-__device__ __forceinline__ void walk_tiles_masked(const float* __restrict__ row, const uint8_t* __restrict__ ind8,
+__device__ __forceinline__ void walk_tiles_masked(const float* __restrict__ row, const uint32_t* __restrict__ ind8,
                                                   uint64_t d, uint32_t k0, uint32_t k1, int j, Body&& body) {
   float4 a[kTileRows], b[kTileRows];
   TileMask ma, mb;
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
+  ma.word = mb.word = 0xffffffffu;
   load_tile(row, static_cast<uint64_t>(k0) * kTile, d, j, a);
   if (kMasked) load_tile_mask(ind8, d, k0, j, ma);
   uint32_t k = k0;
@@ -233,12 +237,11 @@ __device__ __forceinline__ void stream_items(const float* __restrict__ g, const 
   uint32_t k = cur.k0;
   float4 a[kTileRows], b[kTileRows];
   TileMask ma, mb;
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) ma.byte[r] = mb.byte[r] = 0xffu;
+  ma.word = mb.word = 0xffffffffu;
   auto load = [&](const ItemPos& p, uint32_t kk, float4 (&v)[kTileRows], TileMask& mk) {
     load_tile(g + static_cast<uint64_t>(p.m) * geo.ld, static_cast<uint64_t>(kk) * kTile, geo.d, j, v);
     if (kMasked)
-      load_tile_mask(reinterpret_cast<const uint8_t*>(indicators + static_cast<uint64_t>(p.m) * ind_words), geo.d, kk, j, mk);
+      load_tile_mask(indicators + static_cast<uint64_t>(p.m) * ind_words, geo.d, kk, j, mk);
   };
   load(cur, k, a, ma);
   begin(cur.m, cur.c);

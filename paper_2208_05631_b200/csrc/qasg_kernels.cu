@@ -300,8 +300,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
     const float scale = ws.scales[m];
-    const uint8_t* ind8 = kMode ? reinterpret_cast<const uint8_t*>(bits + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5))
-                                : nullptr;
+    const uint32_t* ind8 = kMode ? bits + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5) : nullptr;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
