@@ -114,13 +114,30 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
                    uint64_t* counts, cudaStream_t stream, const uint32_t* touched = nullptr) {
   const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
+  if (touched) {  // rows held in sparse form: one warp per tile
+    const bool stochastic = p->quantizer != QASG_Q_THRESHOLD;
+    if (!stochastic) {
+      Launch l(ctx, kAbsSum, stream);
+      l += launch_touched_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, touched, ctx->shape, stream);
+    } else {
+      Launch l(ctx, kAbsMax, stream);
+      l += launch_touched_abs_max(g, geo, ctx->ws, touched, ctx->shape, stream);
+    }
+    {
+      Launch l(ctx, stochastic ? kStochasticCodes : kThresholdCodes, stream);
+      l += launch_touched_codes(stochastic, g, geo, p->seed, t, ctx->ws, codes, scales, counts_out, touched, ctx->shape,
+                                stream);
+    }
+    if (stochastic && thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
+    return;
+  }
   if (p->quantizer == QASG_Q_THRESHOLD) {
-    { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream, nullptr, touched); }
-    { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream, nullptr, touched); }
+    { Launch l(ctx, kAbsSum, stream); l += launch_abs_sum(g, geo, p->thr_coef, ctx->ws, thresholds, ctx->shape, stream); }
+    { Launch l(ctx, kThresholdCodes, stream); l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, counts_out, ctx->shape, stream); }
   } else {
-    { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream, touched); }
+    { Launch l(ctx, kAbsMax, stream); l += launch_abs_max(g, geo, ctx->ws, ctx->shape, stream); }
     { Launch l(ctx, kStochasticCodes, stream); l += launch_stochastic_codes(g, geo, p->seed, t, 0u, ctx->ws, codes, scales, counts_out,
-                                             ctx->shape, stream, nullptr, touched); }
+                                             ctx->shape, stream); }
     if (thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
   }
 }

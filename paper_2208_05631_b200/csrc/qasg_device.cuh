@@ -271,116 +271,6 @@ __device__ __forceinline__ void stream_items(const float* __restrict__ g, const 
   }
 }
 
-// ------------------------------------------------------------------ gradients held in sparse form
-// A worker's row stores only the entries its `touched` bits mark (bit i&31 of word i>>5); every other
-// entry is +0.0 by definition and its memory is never read.  The tile geometry and every sum stay those
-// of the dense row (adding +0.0 changes no bit of an fp64 sum of non-negative terms), so the results
-// are those of the dense kernels on the densified row, while the loads shrink to the touched sectors
-// and a warp whose 4 x 128 coordinates of a tile hold nothing skips the arithmetic altogether.
-
-// The 16 words of touched bits a warp needs for tile k (its 128 columns of the 4 rows): lane l < 16
-// holds the word of row l>>2, quarter l&3; the other lanes hold 0.  Bits at or past d are dropped.
-__device__ __forceinline__ uint32_t load_touched_words(const uint32_t* __restrict__ trow, uint64_t d, uint32_t k,
-                                                       int warp, int lane, bool ragged) {
-  uint32_t w = 0u;
-  if (lane < 16) {
-    const uint64_t idx = static_cast<uint64_t>(k) * (kTile / 32) + (lane >> 2) * (kTileCols / 32) + 4 * warp + (lane & 3);
-    if (!ragged) {
-      w = __ldg(trow + idx);
-    } else if (idx * 32 < d) {
-      w = __ldg(trow + idx);
-      if (d - idx * 32 < 32) w &= (1u << (d - idx * 32)) - 1u;
-    }
-  }
-  return w;
-}
-
-// The thread's nibbles of touched bits for its four rows (row r in bits 4r..4r+3), from the warp's words.
-__device__ __forceinline__ uint32_t thread_nibbles(uint32_t w, int lane) {
-  uint32_t n = 0u;
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) {
-    const uint32_t ww = __shfl_sync(0xffffffffu, w, r * 4 + (lane >> 3));
-    n |= ((ww >> (4 * (lane & 7))) & 15u) << (4 * r);
-  }
-  return n;
-}
-
-// The thread's four float4 of tile k.  A row is loaded only where its nibble is non-zero (untouched
-// lanes forced to +0.0); rows with an empty nibble read as +0.0.
-__device__ __forceinline__ void load_touched_values(const float* __restrict__ row, uint32_t k, int j, uint32_t nibs,
-                                                    float4 (&v)[kTileRows]) {
-#pragma unroll
-  for (int r = 0; r < kTileRows; ++r) {
-    const uint32_t nib = (nibs >> (4 * r)) & 15u;
-    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (nib) {  // some coordinate below d is marked: the float4 lies inside the row (ld % 4 == 0, ld >= d)
-      t = load_f4(row + static_cast<uint64_t>(k) * kTile + r * kTileCols + 4 * j);
-      if (!(nib & 1u)) t.x = 0.f;
-      if (!(nib & 2u)) t.y = 0.f;
-      if (!(nib & 4u)) t.z = 0.f;
-      if (!(nib & 8u)) t.w = 0.f;
-    }
-    v[r] = t;
-  }
-}
-
-// body(values, nibbles, warp_any, k) for the tiles k0 <= k < k1 of one row.  `values` are valid only in
-// threads whose `nibbles` are non-zero (else they are stale and must not be read); warp_any is uniform
-// in the warp: some lane has a nibble.  The words of bits run two tiles ahead of the arithmetic and
-// the values they admit one tile ahead, so neither load is waited for in steady state.
-template <class Body>
-__device__ __forceinline__ void walk_touched_tiles(const float* __restrict__ row, const uint32_t* __restrict__ trow,
-                                                   uint64_t d, uint32_t tiles, uint32_t k0, uint32_t k1, int j,
-                                                   Body&& body) {
-  const int warp = j >> 5, lane = j & 31;
-  const uint32_t ragged_tile = (d % kTile) ? tiles - 1 : 0xffffffffu;
-  float4 a[kTileRows], b[kTileRows];
-  uint32_t nibs_a = 0u, nibs_b = 0u, w_next, w_after = 0u;
-  bool any_a = false, any_b = false;
-  auto fetch_values = [&](uint32_t kk, uint32_t w, float4 (&v)[kTileRows], uint32_t& nibs, bool& any) {
-    any = __any_sync(0xffffffffu, w != 0u);
-    nibs = 0u;
-    if (any) {
-      nibs = thread_nibbles(w, lane);
-      if (nibs) load_touched_values(row, kk, j, nibs, v);
-    }
-  };
-  w_next = load_touched_words(trow, d, k0, warp, lane, k0 == ragged_tile);
-  if (k0 + 1 < k1) w_after = load_touched_words(trow, d, k0 + 1, warp, lane, k0 + 1 == ragged_tile);
-  fetch_values(k0, w_next, a, nibs_a, any_a);
-  w_next = w_after;
-  uint32_t k = k0;
-  while (true) {
-    if (k + 2 < k1) w_after = load_touched_words(trow, d, k + 2, warp, lane, k + 2 == ragged_tile);
-    if (k + 1 < k1) fetch_values(k + 1, w_next, b, nibs_b, any_b);
-    body(a, nibs_a, any_a, k);
-    w_next = w_after;  // after the arithmetic: by now the words have arrived
-    if (++k >= k1) break;
-    if (k + 2 < k1) w_after = load_touched_words(trow, d, k + 2, warp, lane, k + 2 == ragged_tile);
-    if (k + 1 < k1) fetch_values(k + 1, w_next, a, nibs_a, any_a);
-    body(b, nibs_b, any_b, k);
-    w_next = w_after;
-    if (++k >= k1) break;
-  }
-}
-
-// The items of a launch (as in stream_items) for touched rows: begin(m, c), body as above, end(m, c, n_tiles).
-template <class Begin, class Body, class End>
-__device__ __forceinline__ void stream_touched_items(const float* __restrict__ g, const uint32_t* __restrict__ touched,
-                                                     const Geometry& geo, int j, Begin&& begin, Body&& body,
-                                                     End&& end) {
-  const uint32_t n_items = geo.M * geo.chunks;
-  const uint64_t words = (geo.d + 31) >> 5;
-  for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const ItemPos p = item_pos(geo, item);
-    begin(p.m, p.c);
-    walk_touched_tiles(g + static_cast<uint64_t>(p.m) * geo.ld, touched + static_cast<uint64_t>(p.m) * words, geo.d,
-                       geo.tiles, p.k0, p.k1, j, body);
-    end(p.m, p.c, p.k1 - p.k0);
-  }
-}
-
 // ------------------------------------------------------------------ pass B helpers
 // Code byte of four coordinates, built on the FMA pipe.  pos/neg are 1.0f or 0.0f per
 // coordinate (code 1 = +1, code 2 = -1); the byte value pos0 + 2 neg0 + 4 pos1 + ... + 128 neg3
@@ -427,14 +317,6 @@ __device__ __forceinline__ void store_code_bytes(uint8_t* __restrict__ codes8, u
     for (int r = 0; r < kTileRows; ++r)
       if (b0 + r * (kTileCols / 4) < row_bytes) __stcs(codes8 + b0 + r * (kTileCols / 4), static_cast<uint8_t>(bytes[r]));
   }
-}
-
-// The same bytes for a warp whose codes of tile k are all 0: its 4 x 32 code bytes go out as one
-// 32-bit word per lane (row lane>>3, word lane&7).  The code row is a whole number of words.
-__device__ __forceinline__ void store_zero_code_words(uint8_t* __restrict__ codes8, uint32_t k, int warp, int lane,
-                                                      uint64_t row_bytes) {
-  const uint64_t off = static_cast<uint64_t>(k) * (kTile / 4) + (lane >> 3) * (kTileCols / 4) + 32 * warp + 4 * (lane & 7);
-  if (off < row_bytes) __stcs(reinterpret_cast<uint32_t*>(codes8 + off), 0u);
 }
 
 // Sums per-thread counts over the CTA; the result is valid in thread 0.

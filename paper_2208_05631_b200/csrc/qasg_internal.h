@@ -66,23 +66,19 @@ struct StepScalars {
 
 // Each launcher enqueues on `stream` and returns the number of kernels it launched.
 // denom (device, [M]) replaces d in Delta = coef * sum / d when the sum runs over selected coordinates.
-// touched ([M][ceil(d/32)] words, bit i&31 of word i>>5): the rows of g are held in sparse form, only the
-// marked entries are stored (and read), every other entry is +0.0.
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
                    float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
-                   const unsigned long long* denom = nullptr, const uint32_t* touched = nullptr);
+                   const unsigned long long* denom = nullptr);
 int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
-                   const LaunchShape& shape, cudaStream_t stream, const uint32_t* touched = nullptr);
+                   const LaunchShape& shape, cudaStream_t stream);
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
-                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators = nullptr,
-                           const uint32_t* touched = nullptr);
+                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators = nullptr);
 // stream_base is added to the worker index in Philox counter word 1 (0 for workers, 1<<16 for the server row).
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
                             uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
-                            cudaStream_t stream, const uint32_t* indicators = nullptr,
-                            const uint32_t* touched = nullptr);
+                            cudaStream_t stream, const uint32_t* indicators = nullptr);
 // Sparse selection: indicators [M][ceil(d/32)] words, bit i&31 of word i>>5.
 int launch_select_stats(int rule, bool stochastic, const float* g, const Geometry& geo, const float* x,
                         const float* hz, const SelectScalars& sc, float coef, const Workspace& ws,
@@ -123,6 +119,17 @@ int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float*
 // bits a previous gradient left: zeroes the marked entries of g, then the bits.
 int launch_touched_clear(float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint32_t* touched,
                          const LaunchShape& shape, cudaStream_t stream);
+
+// Passes A and B for rows held in sparse form, one warp per tile (qasg_touched.cu): the results of the
+// dense launchers on the row with +0.0 wherever a touched bit is 0.
+// touched: [M][ceil(d/32)] words, bit i&31 of word i>>5; only the marked entries are stored (and read).
+int launch_touched_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws, float* thresholds_out,
+                           const uint32_t* touched, const LaunchShape& shape, cudaStream_t stream);
+int launch_touched_abs_max(const float* g, const Geometry& geo, const Workspace& ws, const uint32_t* touched,
+                           const LaunchShape& shape, cudaStream_t stream);
+int launch_touched_codes(bool stochastic, const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
+                         const Workspace& ws, uint32_t* codes, float* scales_out, unsigned long long* counts_out,
+                         const uint32_t* touched, const LaunchShape& shape, cudaStream_t stream);
 
 // Exact optimal threshold of one row (rank, prefix sums, first maximum of (sum of the k largest)^2 / k).
 // scratch: optimal_scratch_bytes(d) bytes of device memory, 256-byte aligned; d < 2^31.

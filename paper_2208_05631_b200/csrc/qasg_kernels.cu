@@ -45,12 +45,9 @@ Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks,
 }
 
 // ------------------------------------------------------------------ pass A: sum |g|
-// kTouched: the rows are held in sparse form, `touched` marks their stored entries.
-template <bool kTouched>
 __global__ void __launch_bounds__(kThreads, 4)
 abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
-               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom,
-               const uint32_t* __restrict__ touched) {
+               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom) {
   __shared__ ChunkSumStorage sm_sum;
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -71,31 +68,7 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
         const double total = chunk_sum.finish(geo.log2_group);
         if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
       };
-  // sparse rows: rows of a tile without a touched entry add +0.0 and are skipped, a warp without any
-  // contributes +0.0 without its butterfly; every other addition is the dense one
-  auto touched_body = [&](const float4 (&v)[kTileRows], uint32_t nibs, bool warp_any, uint32_t) {
-    double s = 0.0;
-    if (warp_any) {
-      if (nibs) {
-        double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
-#pragma unroll
-        for (int r = 0; r < kTileRows; ++r)
-          if ((nibs >> (4 * r)) & 15u) {
-            cx += static_cast<double>(fabsf(v[r].x));
-            cy += static_cast<double>(fabsf(v[r].y));
-            cz += static_cast<double>(fabsf(v[r].z));
-            cw += static_cast<double>(fabsf(v[r].w));
-          }
-        s = (cx + cy) + (cz + cw);
-      }
-      s = warp_pair_tree(s);
-    }
-    chunk_sum.add_warp_sum(s);
-  };
-  if (kTouched)
-    stream_touched_items(g, touched, geo, j, begin, touched_body, end);
-  else
-    stream_items<false>(g, nullptr, geo, j, begin, body, end);
+  stream_items<false>(g, nullptr, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   const int warp = j >> 5, lane = j & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
@@ -113,9 +86,8 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
 }
 
 // ------------------------------------------------------------------ pass A': max |g|
-template <bool kTouched>
 __global__ void __launch_bounds__(kThreads)
-abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws, const uint32_t* __restrict__ touched) {
+abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
   __shared__ uint32_t sm_warp[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -135,20 +107,7 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws, const ui
         best = max(best, __float_as_uint(fabsf(v[r].w)));
       }
     };
-    if (kTouched)
-      walk_touched_tiles(row, touched + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5), geo.d, geo.tiles, k0, k1, j,
-                         [&](const float4 (&v)[kTileRows], uint32_t nibs, bool, uint32_t) {
-#pragma unroll
-                           for (int r = 0; r < kTileRows; ++r)
-                             if ((nibs >> (4 * r)) & 15u) {
-                               best = max(best, __float_as_uint(fabsf(v[r].x)));
-                               best = max(best, __float_as_uint(fabsf(v[r].y)));
-                               best = max(best, __float_as_uint(fabsf(v[r].z)));
-                               best = max(best, __float_as_uint(fabsf(v[r].w)));
-                             }
-                         });
-    else
-      walk_tiles(row, geo.d, k0, k1, j, body);
+    walk_tiles(row, geo.d, k0, k1, j, body);
     best = __reduce_max_sync(0xffffffffu, best);
     __syncthreads();  // the previous item's readers are done with sm_warp
     if ((j & 31) == 0) sm_warp[j >> 5] = best;
@@ -177,14 +136,12 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws, const ui
 }
 
 // ------------------------------------------------------------------ pass B: Q_Delta codes
-// kMode 0: dense rows.  1: only coordinates whose indicator bit is set are candidates (sparse selection,
-// Q(S(g, I))); `bits` are the indicators.  2: rows held in sparse form; `bits` mark the stored entries.
-template <int kMode>
+// kMasked: only coordinates whose indicator bit is set are candidates (sparse selection, Q(S(g, I))).
+template <bool kMasked>
 __global__ void __launch_bounds__(kThreads, 4)
 threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
                        uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ bits) {
-  constexpr bool kMasked = kMode == 1;
+                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
   __shared__ ChunkSumStorage sm_sum;
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
@@ -238,55 +195,18 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
           ws.part_cnt[p] = total;
         }
       };
-  // sparse rows: an entry that is not stored is +0.0, inside [-Delta, Delta]: code 0, nothing counted or
-  // summed.  A warp without a touched entry writes its 128 zero code bytes as 32 words.
-  auto touched_body = [&](const float4 (&v)[kTileRows], uint32_t nibs, bool warp_any, uint32_t k) {
-    if (!warp_any) {
-      store_zero_code_words(codes8, k, j >> 5, j & 31, row_words * 4);
-      chunk_sum.add_warp_sum(0.0);
-      return;
-    }
-    double s = 0.0;
-    uint32_t bytes[kTileRows] = {0u, 0u, 0u, 0u};
-    if (nibs) {
-      double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
-#pragma unroll
-      for (int r = 0; r < kTileRows; ++r)
-        if ((nibs >> (4 * r)) & 15u) {
-          const float4 t = v[r];
-          const float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
-          const float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
-          const float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
-          const float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
-          const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;
-          cx += static_cast<double>(fabsf(t.x) * kx);
-          cy += static_cast<double>(fabsf(t.y) * ky);
-          cz += static_cast<double>(fabsf(t.z) * kz);
-          cw += static_cast<double>(fabsf(t.w) * kw);
-          cntf += (kx + ky) + (kz + kw);
-          bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
-        }
-      s = (cx + cy) + (cz + cw);
-    }
-    store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
-    chunk_sum.add_warp_sum(warp_pair_tree(s));
-  };
-  if (kMode == 2)
-    stream_touched_items(g, bits, geo, j, begin, touched_body, end);
-  else
-    stream_items<kMasked>(g, bits, geo, j, begin, body, end);
+  stream_items<kMasked>(g, indicators, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   finish_codes<true>(geo, ws, scales_out, counts_out);
   if (j == 0) *ws.ticket = 0u;
 }
 
 // ------------------------------------------------------------------ pass B': stochastic codes
-template <int kMode>  // as for threshold_codes_kernel
+template <bool kMasked>
 __global__ void __launch_bounds__(kThreads)
 stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
                         uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ bits) {
-  constexpr bool kMasked = kMode == 1;
+                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
@@ -300,7 +220,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
     const float scale = ws.scales[m];
-    const uint32_t* ind8 = kMode ? bits + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5) : nullptr;
+    const uint32_t* ind_row = kMasked ? indicators + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5) : nullptr;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
     uint32_t cnt = 0;
@@ -326,33 +246,8 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
       }
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
     };
-    if (kMode == 2) {
-      // sparse rows: an entry that is not stored is kept with probability |0|/s = 0; its draw is not needed
-      walk_touched_tiles(row, bits + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5), geo.d, geo.tiles, k0, k1, j,
-                         [&](const float4 (&tile)[kTileRows], uint32_t nibs, bool warp_any, uint32_t k) {
-        if (!warp_any) {
-          store_zero_code_words(codes8, k, j >> 5, j & 31, row_words * 4);
-          return;
-        }
-        uint32_t bytes[kTileRows] = {0u, 0u, 0u, 0u};
-#pragma unroll
-        for (int r = 0; r < kTileRows; ++r)
-          if ((nibs >> (4 * r)) & 15u) {
-            const float4 v = tile[r];
-            const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
-            const uint4 w = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), key0, key1);
-            const bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
-            const bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
-            const bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
-            const bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
-            bytes[r] = pack4(split_code(v.x, kx), split_code(v.y, ky), split_code(v.z, kz), split_code(v.w, kw));
-            cnt += nonzero_codes(bytes[r]);
-          }
-        store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
-      });
-    } else {
-      walk_tiles_masked<kMasked>(row, ind8, geo.d, k0, k1, j, body);
-    }
+
+    walk_tiles_masked<kMasked>(row, ind_row, geo.d, k0, k1, j, body);
     const unsigned long long total = block_count(cnt, sm_cnt);
     if (j == 0) ws.part_cnt[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
   }
@@ -1108,53 +1003,38 @@ static unsigned update_grid(uint64_t d, const LaunchShape& shape) {
 
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
                    float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
-                   const unsigned long long* denom, const uint32_t* touched) {
-  if (touched)
-    abs_sum_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom,
-                                                                          touched);
-  else
-    abs_sum_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom,
-                                                                           nullptr);
+                   const unsigned long long* denom) {
+  abs_sum_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom);
   return 1;
 }
 
 int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
-                   const LaunchShape& shape, cudaStream_t stream, const uint32_t* touched) {
-  if (touched)
-    abs_max_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, touched);
-  else
-    abs_max_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, nullptr);
+                   const LaunchShape& shape, cudaStream_t stream) {
+  abs_max_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws);
   return 1;
 }
 
 int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace& ws,
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
-                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators,
-                           const uint32_t* touched) {
-  if (touched)
-    threshold_codes_kernel<2><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                               counts_out, touched);
-  else if (indicators)
-    threshold_codes_kernel<1><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                               counts_out, indicators);
+                           const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators) {
+  if (indicators)
+    threshold_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                                  counts_out, indicators);
   else
-    threshold_codes_kernel<0><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                               counts_out, nullptr);
+    threshold_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
+                                                                                   counts_out, nullptr);
   return 1;
 }
 
 int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, uint64_t t,
                             uint32_t stream_base, const Workspace& ws, uint32_t* codes, float* scales_out,
                             unsigned long long* counts_out, const LaunchShape& shape,
-                            cudaStream_t stream, const uint32_t* indicators, const uint32_t* touched) {
-  if (touched)
-    stochastic_codes_kernel<2><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
-        g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, touched);
-  else if (indicators)
-    stochastic_codes_kernel<1><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+                            cudaStream_t stream, const uint32_t* indicators) {
+  if (indicators)
+    stochastic_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
         g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, indicators);
   else
-    stochastic_codes_kernel<0><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
+    stochastic_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
         g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, nullptr);
   return 1;
 }
