@@ -361,8 +361,9 @@ touched_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, u
 // As many CTAs as are resident at once (the items differ a lot in cost: no second wave behind a slow one).
 template <class Kernel>
 unsigned touched_grid(Kernel kernel, const Geometry& geo, const LaunchShape& shape) {
-  int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+  static int per_sm = 0;  // one instantiation per kernel: asked once (every GPU of a process is the same model)
+  if (per_sm < 1 && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1))
+    per_sm = 1;
   const uint64_t items = static_cast<uint64_t>(geo.M) * geo.chunks;
   const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * per_sm;
   return static_cast<unsigned>(items < resident ? items : resident);
