@@ -112,3 +112,66 @@ def test_more_than_2_to_31_coordinates():
     assert np.array_equal(got[: half // 16], O.pack_codes(tern[:half]))
     assert np.array_equal(got[half // 16:], O.pack_codes(tern[half:]))
     ctx.close()
+
+
+def test_sparse_form_at_the_size_of_the_sparse_logistic_workload():
+    """d = 2^24, 16 workers, minibatch 1024 rows of ~61 entries (the sparse-feature workload), gradients
+    held in sparse form: touched bits exact, gradient values within tolerance, then one QRDA step fed
+    with the oracle's gradient: thresholds, scales and all code rows exact, iterates on a sample."""
+    from oracle import logreg_oracle as L
+    from tests.test_gpu_logreg import G_ATOL, G_RTOL
+    if not _enough_memory():
+        pytest.skip("needs 40 GB of device memory and 24 GB of host memory")
+    dev = U.dev()
+    d, n, m_workers, batch, t = 1 << 24, 1 << 16, 16, 1024, 3
+    lam, eta, delta = 1e-5, 0.1, 1e-8
+    prob = inputs.logreg_csr_problem(n=n, d=d, M=m_workers, nnz_per_row=80, seed=3)
+    rng = np.random.default_rng(8)
+    x0 = (rng.standard_normal(d) * 0.1 * (rng.random(d) < 0.01)).astype(np.float32)
+    h0 = (rng.random(d) * 1e-4).astype(np.float32)
+    z0 = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    ctx = libqasg.Context(d, m_workers, device=0)
+    dev_args = [U.to_dev(prob[k]) for k in ("rowptr", "colidx", "vals", "y")]
+    g = torch.zeros((m_workers, d), dtype=torch.float32, device=dev)
+    bits = torch.zeros((m_workers, d // 32), dtype=torch.int32, device=dev)
+    ctx.logreg_grad_csr_touched(*dev_args, n, d, m_workers, prob["shard_row0"], None, batch, t, U.to_dev(x0), g, d, bits)
+
+    touched = L.touched_columns(prob["rowptr"], prob["colidx"], prob["shard_row0"], batch, t, d)
+    assert np.array_equal(bits.cpu().numpy().view(np.uint32), np.stack([O.pack_bits(r) for r in touched]))
+    g64 = L.grad_workers_csr(prob["rowptr"], prob["colidx"], prob["vals"], prob["y"], prob["shard_row0"], batch, t,
+                             x0.astype(np.float64), d)
+    got = g.cpu().numpy()
+    assert not got[~touched].any()
+    where = np.nonzero(touched)
+    err = np.abs(got[where].astype(np.float64) - g64[where])
+    assert (err <= G_ATOL * np.abs(g64).max() + G_RTOL * np.abs(g64[where])).all()
+    assert 200_000 < where[0].size < 1_000_000
+
+    g32 = np.where(touched, g64.astype(np.float32), np.float32(np.nan))
+    del g64, got
+    params = libqasg.make_params(lam, eta, delta)
+    codes = torch.zeros((m_workers, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+    scales = torch.zeros(m_workers, dtype=torch.float32, device=dev)
+    x, h, z = U.to_dev(x0), U.to_dev(h0), U.to_dev(z0)
+    g.copy_(torch.from_numpy(g32))
+    ctx.step_touched(libqasg.RULE_RDA, g, d, d, m_workers, t, params, bits, x, h, z, codes_out=codes, scales_out=scales)
+    assert ctx.last_async_status() == libqasg.OK
+
+    idx = np.unique(np.concatenate([rng.integers(0, d, size=1 << 18), np.arange(0, 8200), np.arange(d - 4100, d)]))
+    terns = np.zeros((m_workers, idx.size), dtype=np.int8)
+    ref_scales = np.zeros(m_workers, dtype=np.float32)
+    dense = O.densify_touched(g32, touched)
+    for m in range(m_workers):
+        tern, s, thr, cnt = O.threshold_quantize(dense[m])
+        assert cnt > 0
+        assert np.array_equal(U.codes_np(codes[m]), O.pack_codes(tern)), "codes of worker %d" % m
+        assert np.float32(s).view(np.uint32) == scales.cpu().numpy()[m].view(np.uint32), "scale of worker %d" % m
+        terns[m], ref_scales[m] = tern[idx], s
+    q = O.decode_average(terns, ref_scales)
+    x_ref, h_ref, z_ref, a = O.rda_step(q, h0[idx], z0[idx], t, lam, eta, delta)
+    idx_t = torch.from_numpy(idx).to(dev)
+    U.assert_close(x[idx_t], x_ref, "x")
+    U.assert_close(h[idx_t], h_ref, "h")
+    U.assert_close(z[idx_t], z_ref, "z", atol=U.ATOL + 2.0 ** -23 * (np.abs(z0[idx]) + np.abs(q)))
+    U.assert_zero_pattern(x[idx_t], x_ref, a, lam)
+    ctx.close()
