@@ -50,9 +50,9 @@ def bytes_per_coord(M):
 # capture summarised in profiles/step_kernels_d2p24_M8_ncu_full.md (d = 2^24; passes A and B stream,
 # so their traffic grows in proportion to d).  Valid only for the kernel source it was taken from.
 NCU_TRAFFIC = {
-    "kernels_sha256": "57b05eeff5d7e7a99ad8c8ef3f28ee6da94e240b6c8c7e1f202b8c9342abb4a5",
+    "kernels_sha256": "206f79a8b0e52d6d7c801b5258a6214599e3ddb408b8d8cdab5f08dc45f2091a",
     "M": 8,
-    "bytes_per_coord": {"abs_sum": 541030144 / 2 ** 24, "threshold_codes": 568138752 / 2 ** 24},
+    "bytes_per_coord": {"abs_sum": 540481024 / 2 ** 24, "threshold_codes": 568381696 / 2 ** 24},
 }
 
 
