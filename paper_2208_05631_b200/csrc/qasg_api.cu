@@ -33,7 +33,7 @@ enum KernelId {
   kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
   kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kAvgAbsSum, kAvgAbsMax,
   kAvgThresholdCodes, kAvgStochasticCodes, kSelectStats, kIndicatorOr, kTouchedClear, kLogregCsrTouched,
-  kOptimalThreshold, kSmallStep, kKernelIdCount
+  kOptimalThreshold, kKernelIdCount
 };
 static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
 
@@ -380,12 +380,6 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
   if (!codes) return QASG_ERR_WORKSPACE;
   if ((st = enter(ctx)) != QASG_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (d <= kSmallStepMaxD && params->quantizer == QASG_Q_THRESHOLD) {  // a few tiles: everything in one launch
-    Launch l(ctx, kSmallStep, s);
-    l += launch_small_step(rule, g, d, ld_g, M, params->thr_coef, ctx->ws, codes, scales_out, x, h, z,
-                           scalars(params, t), s);
-    return leave();
-  }
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
   { Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s); l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
                                         ctx->ws.status, ctx->shape, s); }
@@ -729,7 +723,7 @@ const char* qasg_kernel_name(int id) {
       "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
       "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr", "avg_abs_sum",
       "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes", "select_stats", "indicator_or",
-      "touched_clear", "logreg_csr_touched", "optimal_threshold", "small_step"};
+      "touched_clear", "logreg_csr_touched", "optimal_threshold"};
   return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
 }
 

@@ -383,42 +383,4 @@ __device__ __forceinline__ float philox_uniform(uint32_t word) {
   return static_cast<float>(word >> 8) * 5.9604644775390625e-08f;  // 2^-24, exact
 }
 
-// ------------------------------------------------------------------ the two updates, one coordinate
-// Square root and reciprocal from the special-function unit: at most 2 ulp off (relative
-// error below 2.4e-7), two orders of magnitude inside the tolerance on the iterates, for a
-// fraction of the instructions of the correctly rounded forms.  Subnormals are kept.
-__device__ __forceinline__ float sqrt_sfu(float a) {
-  float r;
-  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
-  return r;
-}
-__device__ __forceinline__ float rcp_sfu(float a) {
-  float r;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
-  return r;
-}
-
-// Eq. H_t and Eq. QCMD for one coordinate.
-__device__ __forceinline__ void cmd_update(float q, float& x, float& h, const StepScalars& sc) {
-  const float hn = fmaf(q, q, h);
-  const float big_h = sc.delta + sqrt_sfu(hn);
-  const float rate = sc.eta * rcp_sfu(big_h);
-  const float u = fmaf(-rate, q, x);
-  const float mag = fabsf(u) - sc.lambda * rate;
-  x = mag > 0.f ? copysignf(mag, u) : 0.f;
-  h = hn;
-}
-
-// Eq. H_t and Eq. QRDA for one coordinate.  sc.t holds t, sc.inv_t its reciprocal.
-__device__ __forceinline__ void rda_update(float q, float& x, float& h, float& z, const StepScalars& sc) {
-  const float hn = fmaf(q, q, h);
-  const float zn = z + q;
-  const float big_h = sc.delta + sqrt_sfu(hn);
-  const float a = fmaf(fabsf(zn), sc.inv_t, -sc.lambda);
-  const float coef = (sc.t * sc.eta) * rcp_sfu(big_h);
-  x = a > 0.f ? -copysignf(coef * a, zn) : 0.f;
-  h = hn;
-  z = zn;
-}
-
 }  // namespace qasg

@@ -120,13 +120,6 @@ int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float*
 int launch_touched_clear(float* g, uint64_t d, uint64_t ld_g, uint32_t M, uint32_t* touched,
                          const LaunchShape& shape, cudaStream_t stream);
 
-// The fused step with the threshold quantizer in one launch (one CTA per worker, the last one updates):
-// for dimensions of a few tiles, where three launches are all latency.  rule 0 = QCMD, 1 = QRDA.
-constexpr uint64_t kSmallStepMaxD = 4 * kTile;
-int launch_small_step(int rule, const float* g, uint64_t d, uint64_t ld, uint32_t M, float coef, const Workspace& ws,
-                      uint32_t* codes, float* scales_out, float* x, float* h, float* z, const StepScalars& sc,
-                      cudaStream_t stream);
-
 // Passes A and B for rows held in sparse form, one warp per tile (qasg_touched.cu): the results of the
 // dense launchers on the row with +0.0 wherever a touched bit is 0.
 // touched: [M][ceil(d/32)] words, bit i&31 of word i>>5; only the marked entries are stored (and read).
