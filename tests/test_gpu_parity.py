@@ -250,6 +250,33 @@ def test_fused_step_worker_counts(ctx, M, rule):
     U.assert_zero_pattern(x, ref["x"], ref["a"], LAM)
 
 
+@pytest.mark.parametrize("d,M", [(4097, 3), (70_003, 8), (30_000, 13)])
+@pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
+def test_fused_step_gives_the_bits_of_the_unfused_sequence(ctx, d, M, rule):
+    """qasg_step against quantize_pack -> decode_average -> cmd_step / rda_step: same arithmetic, other kernels."""
+    t = 7
+    g = inputs.optimizer_only_gradients(d, M, t, seed=d + M) * np.float32(0.02)
+    x0, h0, z0 = (v.numpy() for v in inputs.random_state(d, seed=M))
+    params = libqasg.make_params(LAM, ETA, DELTA)
+    g_dev, ld = U.grad_to_dev(g)
+    x, h, z = U.to_dev(x0), U.to_dev(h0), U.to_dev(z0)
+    codes, scales = U.new_codes(M, d), torch.zeros(M, dtype=torch.float32, device=U.dev())
+    ctx.step(rule, g_dev, d, ld, M, t, params, x, h, z, codes_out=codes, scales_out=scales)
+    codes2, scales2 = U.new_codes(M, d), torch.zeros(M, dtype=torch.float32, device=U.dev())
+    ctx.quantize_pack(g_dev, d, ld, M, t, params, codes2, scales2)
+    gbar = torch.zeros((d + 3) // 4 * 4, dtype=torch.float32, device=U.dev())
+    ctx.decode_average(codes2, scales2, d, M, gbar)
+    x2, h2, z2 = U.to_dev(x0), U.to_dev(h0), U.to_dev(z0)
+    if rule == libqasg.RULE_CMD:
+        ctx.cmd_step(gbar, x2, h2, d, t, params)
+    else:
+        ctx.rda_step(gbar, x2, h2, z2, d, t, params)
+    assert np.array_equal(U.codes_np(codes), U.codes_np(codes2))
+    assert np.array_equal(U.f32_bits(scales), U.f32_bits(scales2))
+    for a, b in ((x, x2), (h, h2), (z, z2)):
+        assert np.array_equal(U.f32_bits(a), U.f32_bits(b))
+
+
 def test_step_host_matches_step(ctx):
     d, M, t = 50_003, 4, 5
     g = inputs.optimizer_only_gradients(d, M, t, seed=1)
