@@ -168,13 +168,22 @@ __device__ __forceinline__ void stream_touched_tiles(const uint32_t* __restrict_
         for (int r = 0; r < kTileRows; ++r) w[r] = wn[r];
       }
       __syncthreads();
-      if (j == 0)
-        for (uint32_t t = 0; t < batch; ++t) tile_push(st->stack, pushed + t, st->tile_sums[t]);
-      pushed += batch;
+      // The batch is an aligned block of up to 64 tiles, i.e. a complete subtree of the pairwise tree over
+      // tiles (missing tiles count +0.0): one warp sums it - adjacent pairs inside a lane, then the lane
+      // butterfly - and one value per batch goes onto the stack.  (A serial push of every tile by one
+      // thread, with the CTA waiting, cost more than the tiles themselves.)
+      if (warp == 0) {
+        const double a = 2u * lane < batch ? st->tile_sums[2 * lane] : 0.0;
+        const double b = 2u * lane + 1 < batch ? st->tile_sums[2 * lane + 1] : 0.0;
+        const double batch_sum = warp_pair_tree(a + b);
+        if (lane == 0) tile_push(st->stack, pushed, batch_sum);
+      }
+      ++pushed;
       __syncthreads();
     }
     double total = 0.0;
-    if (j == 0) total = tile_fold(st->stack, pushed, geo.log2_group);
+    // the stack holds batches: log2(batches per chunk) levels
+    if (j == 0) total = tile_fold(st->stack, pushed, geo.log2_group > 6 ? geo.log2_group - 6 : 0);
     end(p.m, p.c, total);
   }
 }

@@ -4,6 +4,7 @@
                                                [--min-log2-d 20] [--max-log2-d 28] [--workers 2,4,8,16,32]
   python -m paper_2208_05631_b200.sweep logreg [--steps 50] [--graph] [--csr-only]
   python -m paper_2208_05631_b200.sweep optimal [--min-log2-d 20] [--max-log2-d 28] [--workers 8]
+  python -m paper_2208_05631_b200.sweep touched [--steps 50]
 
 `step`   - the fused step over d in {2^20 .. 2^28} x M in {2, 4, 8, 16, 32} simulated workers,
            N(0,1) gradients, both update rules (the paper uses 2-4 workers; this is the scaling
@@ -16,6 +17,9 @@
 `optimal` - the threshold quantizer with the 0.75 * mean|g| rule against the exact optimal threshold
            (sort + prefix sums): time of each and the relative quantization error each reaches, on
            N(0,1) and on Student-t(3) gradients.
+
+`touched` - passes A and B on rows held in sparse form for synthetic patterns of stored entries (d = 2^24,
+           16 workers): none, uniform, Zipf-like, full head tiles; replayed from a CUDA graph (both kernels).
 
 `--graph` captures one iteration (fixed step index) in a CUDA graph and replays it: every call of the
 library only enqueues kernels on the given stream, so a launch-bound loop can be replayed without
@@ -236,9 +240,60 @@ def sweep_optimal(args):
         del scratch
 
 
+def _bits_from_columns(columns, d, dev):
+    """columns: one int64 tensor of column ids per worker -> touched words int32 [M, d/32]."""
+    rows = []
+    for cols in columns:
+        cols = torch.unique(cols)
+        acc = torch.zeros(d // 32, dtype=torch.int64, device=dev)
+        acc.index_put_(((cols >> 5),), torch.ones_like(cols) << (cols & 31), accumulate=True)   # distinct bits: sum == or
+        rows.append(torch.where(acc >= 2 ** 31, acc - 2 ** 32, acc).to(torch.int32))
+    return torch.stack(rows)
+
+
+def sweep_touched(args):
+    """Passes A and B on rows held in sparse form, for synthetic patterns of stored entries (d = 2^24, M = 16):
+    how the time depends on the number of entries and on where they sit."""
+    dev = torch.device("cuda", 0)
+    d, M = 1 << 24, 16
+    ctx = libqasg.Context(d, M, device=0)
+    params = libqasg.make_params(1e-5, ETA, DELTA)
+    g = torch.randn((M, d), device=dev) * 0.01
+    codes = torch.empty((M, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+    scales = torch.zeros(M, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1)
+    cdf = torch.cumsum(torch.arange(1, d + 1, device=dev, dtype=torch.float64) ** -1.1, 0)
+    cdf = cdf / cdf[-1].clone()
+
+    def uniform(n):
+        return [torch.randint(0, d, (n,), device=dev, generator=gen) for _ in range(M)]
+
+    def zipf(n):
+        return [torch.searchsorted(cdf, torch.rand(n, device=dev, dtype=torch.float64, generator=gen)).clamp(max=d - 1)
+                for _ in range(M)]
+    cases = [("no entry", [torch.zeros(0, dtype=torch.int64, device=dev)] * M),
+             ("25 000 uniform draws per worker", uniform(25_000)),
+             ("250 000 uniform draws per worker", uniform(250_000)),
+             ("62 000 Zipf(1.1) draws per worker", zipf(62_000)),
+             ("the first tile full", [torch.arange(0, 4096, device=dev)] * M),
+             ("the first 16 tiles full", [torch.arange(0, 16 * 4096, device=dev)] * M)]
+    for name, columns in cases:
+        bits = _bits_from_columns(columns, d, dev)
+
+        def run():
+            ctx.quantize_pack_touched(g, d, d, M, 1, params, bits, codes, scales)
+        graph_us = _timed_graph(run, 3, args.steps)
+        entries = int(sum(torch.unique(c).numel() for c in columns))
+        print(json.dumps({"what": "touched_passes_A_B", "pattern": name, "d": d, "M": M, "stored_entries": entries,
+                          "us_per_graph_replay": graph_us}), flush=True)
+    assert ctx.last_async_status() == libqasg.OK
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["step", "logreg", "optimal"])
+    ap.add_argument("what", choices=["step", "logreg", "optimal", "touched"])
     ap.add_argument("--quantizer", default="threshold", choices=["threshold", "stochastic"])
     ap.add_argument("--double-quant", action="store_true")
     ap.add_argument("--select", action="store_true")
@@ -254,6 +309,8 @@ def main():
     assert torch.cuda.is_available(), "needs a CUDA device"
     if args.what == "optimal":
         sweep_optimal(args)
+    elif args.what == "touched":
+        sweep_touched(args)
     elif args.what == "step":
         sweep_step(args)
     else:
