@@ -5,11 +5,13 @@
 // word of touched bits per row, so a tile without entries costs four coalesced word loads and a vote, and a
 // stored entry costs one scalar load.  The sums are those of the dense kernels bit for bit, because the
 // tree is the same and adding +0.0 changes nothing: column sums down the rows, a pairwise tree over a
-// lane's 32 columns (levels 0-4), the lane butterfly (levels 5-9), the pairwise stack over tiles, chunk
-// partials combined by the last CTA.  A lane with more than two touched columns (the head of a row whose
-// column frequencies are Zipf-like is full) fetches its rows with 128-bit loads, all in flight together,
-// and keeps its 32 column sums in local memory.  Rows that are full throughout are better served by the
-// dense entry points.
+// lane's 32 columns (levels 0-4), the lane butterfly (levels 5-9), a pairwise tree over the tiles of a
+// chunk (one warp per batch of up to 64 tiles, a pairwise stack over the batches), chunk partials combined
+// by the last CTA.  A lane takes one of three paths by the number of its touched columns: one or two (the
+// usual case: all loads issued together, a + b is the tree), up to twelve (column after column, the next
+// column's loads ahead), more (the head of a row whose column frequencies are Zipf-like is full: 128-bit
+// loads of all four rows in flight together, values and column sums in local memory).  Rows that are full
+// throughout are better served by the dense entry points.
 #include "qasg_device.cuh"
 
 namespace qasg {
@@ -17,7 +19,7 @@ namespace qasg {
 namespace {
 
 constexpr int kWarps = kThreads / 32;
-constexpr int kTouchedBatch = 64;  // tiles per CTA-wide meeting (kWarps tiles in flight at a time)
+constexpr int kTouchedBatch = 64;  // tiles between two meetings of the CTA (a warp takes every eighth of them)
 
 struct TouchedStorage {
   double tile_sums[kTouchedBatch];
