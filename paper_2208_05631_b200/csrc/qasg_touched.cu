@@ -11,7 +11,9 @@
 // usual case: all loads issued together, a + b is the tree), up to twelve (column after column, the next
 // column's loads ahead), more (the head of a row whose column frequencies are Zipf-like is full: 128-bit
 // loads of all four rows in flight together, values and column sums in local memory).  Rows that are full
-// throughout are better served by the dense entry points.
+// throughout are better served by the dense entry points.  A tile with more than kCrowdedTile entries is walked
+// in the dense layout instead (crowded_tile below).  (Capping the registers to keep five CTAs per SM made the
+// crowded path spill and every pattern slower.)
 #include "qasg_device.cuh"
 
 namespace qasg {
@@ -137,6 +139,57 @@ __device__ __forceinline__ double lane_columns(const float* __restrict__ row, ui
   return lane_tree(col);
 }
 
+// A crowded tile (more than kCrowdedTile entries), still by one warp, in the dense kernels' layout: eight
+// slices of 128 columns; in slice q lane l takes the float4 at columns 128q + 4l .. + 3 of each row whose
+// nibble of bits is non-zero (untouched lanes forced to +0.0).  slice(values, nibbles, q) returns the
+// thread's share (cx + cy) + (cz + cw) of the slice; the lane butterfly makes it the sum of the slice's 128
+// columns (levels 0-6 of the tree) and the eight slices are combined pairwise (levels 7-9).
+constexpr uint32_t kCrowdedTile = 256;
+
+__device__ __forceinline__ uint32_t tile_entries(const uint32_t (&w)[kTileRows]) {
+  return __reduce_add_sync(0xffffffffu, (__popc(w[0]) + __popc(w[1])) + (__popc(w[2]) + __popc(w[3])));
+}
+
+template <class Slice>
+__device__ __forceinline__ double crowded_tile(const float* __restrict__ row, uint64_t tile_base, int lane,
+                                               const uint32_t (&w)[kTileRows], Slice&& slice) {
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, total = 0.0;  // pairwise stack over the slices
+#pragma unroll 1
+  for (int q = 0; q < 8; ++q) {
+    uint32_t nibs = 0u;
+    float4 v[kTileRows];
+#pragma unroll
+    for (int r = 0; r < kTileRows; ++r) {
+      const uint32_t word = __shfl_sync(0xffffffffu, w[r], 4 * q + (lane >> 3));
+      const uint32_t nib = (word >> (4 * (lane & 7))) & 15u;
+      nibs |= nib << (4 * r);
+      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (nib) {  // some coordinate below d is marked: the float4 lies inside the row
+        t = load_f4(row + tile_base + r * kTileCols + 128 * q + 4 * lane);
+        if (!(nib & 1u)) t.x = 0.f;
+        if (!(nib & 2u)) t.y = 0.f;
+        if (!(nib & 4u)) t.z = 0.f;
+        if (!(nib & 8u)) t.w = 0.f;
+      }
+      v[r] = t;
+    }
+    double x = warp_pair_tree(slice(v, nibs, q));
+    if (q & 1) {
+      x = s0 + x;
+      if (q & 2) {
+        x = s1 + x;
+        if (q & 4) total = s2 + x;
+        else s2 = x;
+      } else {
+        s1 = x;
+      }
+    } else {
+      s0 = x;
+    }
+  }
+  return total;
+}
+
 // The tiles of the CTA's items, one warp per tile, in batches of kTouchedBatch tiles:
 //   begin(m, c)                    all threads, before an item
 //   tile(m, k, words) -> double    one warp, a tile with entries: its sum (valid in every lane)
@@ -200,8 +253,21 @@ touched_abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Wo
   stream_touched_tiles(
       touched, geo, &st, [](uint32_t, uint32_t) {},
       [&](uint32_t m, uint32_t k, const uint32_t (&w)[kTileRows]) -> double {
-        const double s = lane_columns(g + static_cast<uint64_t>(m) * geo.ld, static_cast<uint64_t>(k) * kTile, lane, w,
-                                      [](int, int, float v) { return fabsf(v); });
+        const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+        if (tile_entries(w) > kCrowdedTile)
+          return crowded_tile(row, static_cast<uint64_t>(k) * kTile, lane, w,
+                              [](const float4 (&v)[kTileRows], uint32_t, int) -> double {
+                                double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
+#pragma unroll
+                                for (int r = 1; r < kTileRows; ++r) {
+                                  cx += static_cast<double>(fabsf(v[r].x));
+                                  cy += static_cast<double>(fabsf(v[r].y));
+                                  cz += static_cast<double>(fabsf(v[r].z));
+                                  cw += static_cast<double>(fabsf(v[r].w));
+                                }
+                                return (cx + cy) + (cz + cw);
+                              });
+        const double s = lane_columns(row, static_cast<uint64_t>(k) * kTile, lane, w, [](int, int, float v) { return fabsf(v); });
         return warp_pair_tree(s);
       },
       [](uint32_t, uint32_t) {},
@@ -233,11 +299,25 @@ touched_abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws, 
   stream_touched_tiles(
       touched, geo, &st, [&](uint32_t, uint32_t) { best = 0u; },
       [&](uint32_t m, uint32_t k, const uint32_t (&w)[kTileRows]) -> double {
-        lane_columns(g + static_cast<uint64_t>(m) * geo.ld, static_cast<uint64_t>(k) * kTile, lane, w,
-                     [&](int, int, float v) {
-                       best = max(best, __float_as_uint(fabsf(v)));
-                       return 0.f;
-                     });
+        const float* row = g + static_cast<uint64_t>(m) * geo.ld;
+        if (tile_entries(w) > kCrowdedTile) {
+          crowded_tile(row, static_cast<uint64_t>(k) * kTile, lane, w,
+                       [&](const float4 (&v)[kTileRows], uint32_t, int) -> double {
+#pragma unroll
+                         for (int r = 0; r < kTileRows; ++r) {  // untouched lanes are +0.0 and change no maximum
+                           best = max(best, __float_as_uint(fabsf(v[r].x)));
+                           best = max(best, __float_as_uint(fabsf(v[r].y)));
+                           best = max(best, __float_as_uint(fabsf(v[r].z)));
+                           best = max(best, __float_as_uint(fabsf(v[r].w)));
+                         }
+                         return 0.0;
+                       });
+          return 0.0;
+        }
+        lane_columns(row, static_cast<uint64_t>(k) * kTile, lane, w, [&](int, int, float v) {
+          best = max(best, __float_as_uint(fabsf(v)));
+          return 0.f;
+        });
         return 0.0;
       },
       [](uint32_t, uint32_t) {},
@@ -323,9 +403,49 @@ touched_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, u
         cnt = 0;
       },
       [&](uint32_t m, uint32_t k, const uint32_t (&w)[kTileRows]) -> double {
+        const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
+        if (tile_entries(w) > kCrowdedTile) {
+          uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
+          const double s = crowded_tile(
+              g + static_cast<uint64_t>(m) * geo.ld, tile_base, lane, w,
+              [&](const float4 (&v)[kTileRows], uint32_t nibs, int q) -> double {
+                double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
+#pragma unroll
+                for (int r = 0; r < kTileRows; ++r) {
+                  const float4 t = v[r];
+                  uint32_t byte = 0u;
+                  if ((nibs >> (4 * r)) & 15u) {
+                    if (!kStochastic) {
+                      const float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
+                      const float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
+                      const float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
+                      const float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+                      cx += static_cast<double>(fabsf(t.x) * (px + nx));
+                      cy += static_cast<double>(fabsf(t.y) * (py + ny));
+                      cz += static_cast<double>(fabsf(t.z) * (pz + nz));
+                      cw += static_cast<double>(fabsf(t.w) * (pw + nw));
+                      byte = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
+                    } else {
+                      // the float4 at columns 128q + 4*lane is Philox block (coordinate >> 2)
+                      const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + 32 * q + lane;
+                      const uint4 x = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), key0, key1);
+                      const bool kx = philox_uniform(x.x) < __fdiv_rn(fabsf(t.x), scale);
+                      const bool ky = philox_uniform(x.y) < __fdiv_rn(fabsf(t.y), scale);
+                      const bool kz = philox_uniform(x.z) < __fdiv_rn(fabsf(t.z), scale);
+                      const bool kw = philox_uniform(x.w) < __fdiv_rn(fabsf(t.w), scale);
+                      byte = pack4(split_code(t.x, kx), split_code(t.y, ky), split_code(t.z, kz), split_code(t.w, kw));
+                    }
+                    cnt += nonzero_codes(byte);
+                  }
+                  const uint64_t off = static_cast<uint64_t>(k) * (kTile / 4) + r * (kTileCols / 4) + 32 * q + lane;
+                  if (off < row_words * 4) __stcs(codes8 + off, static_cast<uint8_t>(byte));
+                }
+                return (cx + cy) + (cz + cw);
+              });
+          return kStochastic ? 0.0 : s;
+        }
         LaneCodes lc;
         lc.clear();
-        const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
         const double s = lane_columns(
             g + static_cast<uint64_t>(m) * geo.ld, tile_base, lane, w, [&](int r, int c, float v) {
               uint32_t code;
