@@ -144,7 +144,7 @@ __device__ __forceinline__ double lane_columns(const float* __restrict__ row, ui
 // nibble of bits is non-zero (untouched lanes forced to +0.0).  slice(values, nibbles, q) returns the
 // thread's share (cx + cy) + (cz + cw) of the slice; the lane butterfly makes it the sum of the slice's 128
 // columns (levels 0-6 of the tree) and the eight slices are combined pairwise (levels 7-9).
-constexpr uint32_t kCrowdedTile = 256;
+constexpr uint32_t kCrowdedTile = 128;
 
 __device__ __forceinline__ uint32_t tile_entries(const uint32_t (&w)[kTileRows]) {
   return __reduce_add_sync(0xffffffffu, (__popc(w[0]) + __popc(w[1])) + (__popc(w[2]) + __popc(w[3])));
