@@ -15,6 +15,15 @@ Conventions the paper leaves open (each is this library's documented reading):
   theorems assume) draws from Philox4x32-10 keyed by (seed, t, m, i).
 * Scalars lambda, eta, delta and the threshold coefficient are fp32 at the library
   boundary; they are promoted exactly to fp64 here.
+
+Parity unpinned (the paper fixes none of these, so no outside value can pin them):
+the order of additions inside `canonical_sum` and `canonical_prefix` (their last fp64
+bits), the bit layout of `pack_codes`, and the way `philox_draws` maps (seed, t, m, i)
+to counter and key words.  What the tests pin instead: both sums as sums (exact where
+the partial sums are representable, within the pairwise error bound of the exactly
+rounded sum otherwise; the fp32 threshold equal to the exactly rounded definition on
+the seeded cases), the Philox block function by its published known-answer vectors,
+and pack/unpack as inverse maps.
 """
 import numpy as np
 
