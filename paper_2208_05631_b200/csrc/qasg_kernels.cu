@@ -203,7 +203,7 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
 
 // ------------------------------------------------------------------ pass B': stochastic codes
 template <bool kMasked>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
                         uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
                         unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
