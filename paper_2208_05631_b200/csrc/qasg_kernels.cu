@@ -461,6 +461,199 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
   if (bad) atomicOr(status, kFlagBadCode);
 }
 
+// ------------------------------------------------------------------ pass C for 13 workers and more
+// With many workers the byte-per-worker decode above is bound by integer instructions (address
+// arithmetic for one byte load per worker and four coordinates, the 2-bit transposition, the
+// field extraction), not by HBM.  Here a thread owns eight consecutive coordinates, so one
+// 16-bit load per worker brings its codes, and the lookup index is formed differently: the four
+// bytes gathered from a group of four workers are masked down to one 2-bit field each, and one
+// 32-bit multiplication sums them with the weights (1, 3, 9, 27) into the radix-3 index
+//   idx = c0 + 3 c1 + 9 c2 + 27 c3  in 0..80      (code values 0, 1, 2).  The table of a worker group then has 81 entries instead of 256, so 16
+// lane copies (no bank conflict for 64-bit lookups) fit for every worker count: 10 KB per group.
+// The partial sums are the same doubles, added in the same order, as in decode_update_kernel.
+// A code value 3 has no radix-3 digit: the fields are tested before they are used, and a thread that
+// meets one clears them first (code 3 decodes to 0).
+constexpr int kWideThreads = 512;
+constexpr int kLut3Entries = 81;
+constexpr int kLut3Lanes = 16;
+
+__device__ __forceinline__ void build_decode_lut3(double* lut, const float* __restrict__ scales, uint32_t M) {
+  const uint32_t groups = (M + 3) >> 2;
+  for (uint32_t e = threadIdx.x; e < groups * kLut3Entries * kLut3Lanes; e += blockDim.x) {
+    const uint32_t entry = e / kLut3Lanes;
+    const uint32_t grp = entry / kLut3Entries;
+    uint32_t idx = entry - grp * kLut3Entries;
+    double acc = 0.0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t m = grp * 4 + k;
+      const uint32_t c = idx % 3u;
+      idx /= 3u;
+      if (m < M && c != 0u) {
+        const double sv = static_cast<double>(scales[m]);
+        acc += (c == 1u) ? sv : -sv;
+      }
+    }
+    lut[e] = acc;
+  }
+  __syncthreads();
+}
+
+// Entry idx of the lane's copy of the table at shared-memory address table_lane: 32-bit address
+// arithmetic, one multiply-add.
+__device__ __forceinline__ double lut3_entry(uint32_t table_lane, uint32_t idx) {
+  double v;
+  asm("ld.shared.f64 %0, [%1];" : "=d"(v) : "r"(idx * (kLut3Lanes * 8u) + table_lane));
+  return v;
+}
+
+// Loads the 16 code bits that each of the batch's workers m0 .. m0 + 4 kG4 - 1 holds for the eight
+// coordinates of oct o, and adds their decoded values to q (Eq. SynQ_t before the division by M).
+// lut_lane is the shared-memory address of the lane's copy of the batch's first table.  kLast: the batch holds the last
+// worker group, the only one that can be short of workers.  Returns true if a code value 3 was met.
+template <int kG4, bool kLast>
+__device__ __forceinline__ bool decode_batch(const uint16_t* __restrict__ codes16, uint64_t row_halves,
+                                             uint64_t o, uint32_t m0, uint32_t M, uint32_t lut_lane,
+                                             double (&q)[8]) {
+  uint32_t c[4 * kG4];
+  const uint16_t* p = codes16 + static_cast<uint64_t>(m0) * row_halves + o;
+#pragma unroll
+  for (int m = 0; m < 4 * kG4; ++m)
+    c[m] = (!kLast || m < 4 * (kG4 - 1) || m0 + m < M) ? __ldg(p + m * row_halves) : 0u;
+  uint32_t lo[kG4], hi[kG4], threes = 0;
+#pragma unroll
+  for (int G = 0; G < kG4; ++G) {
+    // byte k of lo (hi) = worker 4G+k's codes of coordinates 0..3 (4..7)
+    const uint32_t ab = __byte_perm(c[4 * G], c[4 * G + 1], 0x5140);
+    const uint32_t cd = __byte_perm(c[4 * G + 2], c[4 * G + 3], 0x5140);
+    lo[G] = __byte_perm(ab, cd, 0x5410);
+    hi[G] = __byte_perm(ab, cd, 0x7632);
+    threes |= (lo[G] & (lo[G] >> 1)) | (hi[G] & (hi[G] >> 1));
+  }
+  const bool bad = (threes & 0x55555555u) != 0u;
+  if (bad) {  // rare: clear the fields that hold 3 before they are used as digits
+#pragma unroll
+    for (int G = 0; G < kG4; ++G) {
+      lo[G] &= ~((lo[G] & (lo[G] >> 1) & 0x55555555u) * 3u);
+      hi[G] &= ~((hi[G] & (hi[G] >> 1) & 0x55555555u) * 3u);
+    }
+  }
+  // A word masked down to one field per byte holds four digits; in its product with the weights the
+  // top byte collects byte0 + 3 byte1 + 9 byte2 + 27 byte3 <= 80: the other partial products fall
+  // below bit 24, in disjoint fields, or leave the 32 bits.
+  constexpr uint32_t kRadix3 = 0x0103091Bu;
+#pragma unroll
+  for (int G = 0; G < kG4; ++G) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t il = (((lo[G] >> (2 * j)) & 0x03030303u) * kRadix3) >> 24;
+      const uint32_t ih = (((hi[G] >> (2 * j)) & 0x03030303u) * kRadix3) >> 24;
+      q[j] += lut3_entry(lut_lane + G * (kLut3Entries * kLut3Lanes * 8), il);
+      q[4 + j] += lut3_entry(lut_lane + G * (kLut3Entries * kLut3Lanes * 8), ih);
+    }
+  }
+  return bad;
+}
+
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
+// Two CTAs of kWideThreads threads per SM.  The workers are decoded in batches of 16 (their code bits
+// are the only loads in flight then); the state of the eight coordinates is requested into L2 first and
+// loaded once the average is known, so that it does not hold registers during the decode.
+template <int kRule, int kM4>
+__global__ void __launch_bounds__(kWideThreads, 2)
+decode_update_wide_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ scales, uint64_t d,
+                          uint32_t M, double inv_m, float* __restrict__ x, float* __restrict__ h,
+                          float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
+  extern __shared__ double sm_lut[];
+  build_decode_lut3(sm_lut, scales, M);
+  const uint32_t lut_lane =
+      static_cast<uint32_t>(__cvta_generic_to_shared(sm_lut + (threadIdx.x & (kLut3Lanes - 1))));
+  const uint16_t* codes16 = reinterpret_cast<const uint16_t*>(codes);
+  const uint64_t row_halves = ((d + 15) >> 4) * 2;
+  const uint64_t octs = (d + 7) >> 3, full = d >> 3;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kWideThreads;
+  constexpr int kBatch = 4;                         // worker groups per batch
+  constexpr int kWholeBatches = (kM4 - 1) / kBatch;  // batches before the last one
+  bool bad = false;
+  for (uint64_t o = static_cast<uint64_t>(blockIdx.x) * kWideThreads + threadIdx.x; o < octs; o += stride) {
+    const bool whole = o < full;
+    float* ap = (kRule == 0 ? x : z) + 8 * o;  // x for QCMD (read and written), z for QRDA
+    if (kRule != 2 && whole) {
+      prefetch_l2(h + 8 * o);
+      prefetch_l2(ap);
+    }
+    double q[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = 0.0;
+#pragma unroll
+    for (int b = 0; b < kWholeBatches; ++b)
+      bad |= decode_batch<kBatch, false>(codes16, row_halves, o, 4 * kBatch * b, M,
+                                         lut_lane + b * (kBatch * kLut3Entries * kLut3Lanes * 8), q);
+    bad |= decode_batch<kM4 - kBatch * kWholeBatches, true>(
+        codes16, row_halves, o, 4 * kBatch * kWholeBatches, M,
+        lut_lane + kWholeBatches * (kBatch * kLut3Entries * kLut3Lanes * 8), q);
+    float qf[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qf[i] = static_cast<float>(q[i] * inv_m);
+    if (whole) {
+      if (kRule == 2) {
+        *reinterpret_cast<float4*>(x + 8 * o) = make_float4(qf[0], qf[1], qf[2], qf[3]);
+        *reinterpret_cast<float4*>(x + 8 * o + 4) = make_float4(qf[4], qf[5], qf[6], qf[7]);
+        continue;
+      }
+      float4 h0 = *reinterpret_cast<const float4*>(h + 8 * o);
+      float4 h1 = *reinterpret_cast<const float4*>(h + 8 * o + 4);
+      float4 a0 = *reinterpret_cast<const float4*>(ap);
+      float4 a1 = *reinterpret_cast<const float4*>(ap + 4);
+      if (kRule == 0) {
+        cmd_update(qf[0], a0.x, h0.x, sc), cmd_update(qf[1], a0.y, h0.y, sc);
+        cmd_update(qf[2], a0.z, h0.z, sc), cmd_update(qf[3], a0.w, h0.w, sc);
+        cmd_update(qf[4], a1.x, h1.x, sc), cmd_update(qf[5], a1.y, h1.y, sc);
+        cmd_update(qf[6], a1.z, h1.z, sc), cmd_update(qf[7], a1.w, h1.w, sc);
+        *reinterpret_cast<float4*>(x + 8 * o) = a0;
+        *reinterpret_cast<float4*>(x + 8 * o + 4) = a1;
+      } else {
+        float4 x0, x1;
+        rda_update(qf[0], x0.x, h0.x, a0.x, sc), rda_update(qf[1], x0.y, h0.y, a0.y, sc);
+        rda_update(qf[2], x0.z, h0.z, a0.z, sc), rda_update(qf[3], x0.w, h0.w, a0.w, sc);
+        rda_update(qf[4], x1.x, h1.x, a1.x, sc), rda_update(qf[5], x1.y, h1.y, a1.y, sc);
+        rda_update(qf[6], x1.z, h1.z, a1.z, sc), rda_update(qf[7], x1.w, h1.w, a1.w, sc);
+        *reinterpret_cast<float4*>(z + 8 * o) = a0;
+        *reinterpret_cast<float4*>(z + 8 * o + 4) = a1;
+        *reinterpret_cast<float4*>(x + 8 * o) = x0;
+        *reinterpret_cast<float4*>(x + 8 * o + 4) = x1;
+      }
+      *reinterpret_cast<float4*>(h + 8 * o) = h0;
+      *reinterpret_cast<float4*>(h + 8 * o + 4) = h1;
+    } else {  // ragged tail: d % 8 coordinates
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint64_t i = 8 * o + e;
+        if (i >= d) break;
+        const float qi = qf[e];
+        if (kRule == 2) {
+          x[i] = qi;
+          continue;
+        }
+        float xi = (kRule == 0) ? x[i] : 0.f, hi = h[i];
+        if (kRule == 0) {
+          cmd_update(qi, xi, hi, sc);
+        } else {
+          float zi = z[i];
+          rda_update(qi, xi, hi, zi, sc);
+          z[i] = zi;
+        }
+        x[i] = xi;
+        h[i] = hi;
+      }
+    }
+  }
+  if (bad) atomicOr(status, kFlagBadCode);
+}
+
 // ------------------------------------------------------------------ pass C, update from a dense q
 template <int kRule>
 __global__ void __launch_bounds__(kThreads)
@@ -1097,6 +1290,30 @@ static void launch_decode_update_as(const uint32_t* codes, const float* scales, 
                                                                         status);
 }
 
+template <int kRule, int kM4>
+static void launch_decode_update_wide_as(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
+                                         float* x, float* h, float* z, const StepScalars& sc,
+                                         unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
+  auto kernel = decode_update_wide_kernel<kRule, kM4>;
+  const size_t lut_bytes = static_cast<size_t>(kM4) * kLut3Entries * kLut3Lanes * sizeof(double);
+  static thread_local int ctas_per_sm[64] = {0};  // per device, resolved on first use
+  int dev = 0;
+  cudaGetDevice(&dev);
+  int& resident = ctas_per_sm[dev & 63];
+  if (resident == 0) {
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(lut_bytes));
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kWideThreads, lut_bytes);
+    if (resident < 1) resident = 1;
+  }
+  const uint64_t octs = (d + 7) >> 3;
+  uint64_t grid = (octs + kWideThreads - 1) / kWideThreads;
+  const uint64_t max_grid = static_cast<uint64_t>(shape.sm_count) * resident;
+  if (grid > max_grid) grid = max_grid;
+  const double inv_m = 1.0 / static_cast<double>(M);
+  kernel<<<static_cast<unsigned>(grid), kWideThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc,
+                                                                           status);
+}
+
 template <int kRule>
 static void launch_decode_update_rule(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
                                       float* x, float* h, float* z, const StepScalars& sc,
@@ -1107,16 +1324,19 @@ static void launch_decode_update_rule(const uint32_t* codes, const float* scales
   case m4: launch_decode_update_as<kRule, m4, 16, 512, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_LANES(m4, lanes) \
   case m4: launch_decode_update_as<kRule, m4, lanes, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+#define QASG_WIDE(m4) \
+  case m4: launch_decode_update_wide_as<kRule, m4>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_SHARED(m4) \
   case m4: launch_decode_update_as<kRule, m4, 1, kThreads, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
   switch ((M + 3) / 4) {
     QASG_LANE(1) QASG_LANE(2) QASG_LANE(3)
     // 16 copies (32 KB per worker group) keep the two half-warps of a 64-bit lookup apart; 8 copies
     // leave two lanes per copy
-    QASG_LANES(4, 16) QASG_LANES(5, 16) QASG_LANES(6, 16) QASG_LANES(7, 16)
-    QASG_LANES(8, 8) QASG_LANES(9, 8) QASG_LANES(10, 8) QASG_LANES(11, 8) QASG_LANES(12, 8) QASG_LANES(13, 8)
+    QASG_WIDE(4) QASG_WIDE(5) QASG_WIDE(6) QASG_WIDE(7) QASG_WIDE(8)
+    QASG_LANES(9, 8) QASG_LANES(10, 8) QASG_LANES(11, 8) QASG_LANES(12, 8) QASG_LANES(13, 8)
     QASG_SHARED(14) QASG_SHARED(15) QASG_SHARED(16)
   }
+#undef QASG_WIDE
 #undef QASG_LANE
 #undef QASG_LANES
 #undef QASG_SHARED

@@ -115,7 +115,8 @@ def test_stochastic_codes_bit_exact(ctx, d, t, seed):
 
 
 # ------------------------------------------------------------------ decode + average
-@pytest.mark.parametrize("d,M", [(1, 1), (18, 3), (4099, 8), (100_001, 33)])
+@pytest.mark.parametrize("d,M", [(1, 1), (18, 3), (4099, 8), (100_001, 33),
+                                 (1, 13), (7, 16), (8, 17), (4103, 20), (70_005, 29), (100_001, 32)])
 def test_decode_average(ctx, d, M):
     g = inputs.optimizer_only_gradients(d, M, t=2, seed=5)
     ref = O.quantize_workers(g, O.QUANT_THRESHOLD)
@@ -136,6 +137,26 @@ def test_invalid_code_is_reported_and_decodes_to_zero(ctx):
     assert ctx.last_async_status() == libqasg.ERR_BAD_CODE
     out = gbar.cpu().numpy()
     assert out[0] == 0.0 and out[1] == 1.0 and not out[2:].any()
+
+
+@pytest.mark.parametrize("M", [13, 16, 29, 32])
+def test_invalid_codes_among_many_workers(ctx, M):
+    """13 to 32 workers are decoded eight coordinates at a time through radix-3 tables, where a code
+    value 3 is not a digit: it must still decode to 0, be reported, and leave every other worker's
+    and coordinate's contribution as it is."""
+    d = 8 * 512 * 3 + 5
+    rng = np.random.default_rng(M)
+    tern = rng.integers(-1, 2, size=(M, d)).astype(np.int8)
+    scales = (1.0 + rng.random(M)).astype(np.float32)
+    words = np.stack([O.pack_codes(tern[m]) for m in range(M)])
+    hit = [(0, 0), (M - 1, 9), (M // 2, 4100), (3, d - 1), (M - 2, d - 1)]   # (worker, coordinate)
+    for m, i in hit:
+        words[m, i >> 4] |= np.uint32(3) << np.uint32(2 * (i & 15))
+        tern[m, i] = 0
+    gbar = torch.full((d,), 7.0, dtype=torch.float32, device=U.dev())
+    ctx.decode_average(U.to_dev(words.view(np.int32)), U.to_dev(scales), d, M, gbar)
+    assert ctx.last_async_status() == libqasg.ERR_BAD_CODE
+    U.assert_close(gbar, O.decode_average(tern, scales), "gbar")
 
 
 # ------------------------------------------------------------------ dense updates
