@@ -5,6 +5,7 @@
 //           stochastic_codes_kernel             unbiased ternary codes from Philox draws
 //   pass C  decode_update_kernel                decode + average + accumulator + QCMD/QRDA (or the
 //                                               average alone), dense_update_kernel: update from a dense q
+//           decode_update_wide_kernel           the same for 13 to 32 workers, eight coordinates per thread
 //   server  avg_abs_sum/avg_abs_max/avg_codes   double quantization: Q applied to the average
 //   select  select_stats, indicator_or          sparse selection: indicators, statistics over the selected
 //
@@ -512,14 +513,17 @@ __device__ __forceinline__ double lut3_entry(uint32_t table_lane, uint32_t idx) 
 // lut_lane is the shared-memory address of the lane's copy of the batch's first table.  kLast: the batch holds the last
 // worker group, the only one that can be short of workers.  Returns true if a code value 3 was met.
 template <int kG4, bool kLast>
-__device__ __forceinline__ bool decode_batch(const uint16_t* __restrict__ codes16, uint64_t row_halves,
+__device__ __forceinline__ bool decode_batch(const uint8_t* __restrict__ codes8, uint32_t row_bytes,
                                              uint64_t o, uint32_t m0, uint32_t M, uint32_t lut_lane,
                                              double (&q)[8]) {
   uint32_t c[4 * kG4];
-  const uint16_t* p = codes16 + static_cast<uint64_t>(m0) * row_halves + o;
+  // row_bytes fits 32 bits (the launcher checks), so a worker's address is one widening multiply-add
+  const uint8_t* p = codes8 + static_cast<uint64_t>(m0) * row_bytes + 2 * o;
 #pragma unroll
   for (int m = 0; m < 4 * kG4; ++m)
-    c[m] = (!kLast || m < 4 * (kG4 - 1) || m0 + m < M) ? __ldg(p + m * row_halves) : 0u;
+    c[m] = (!kLast || m < 4 * (kG4 - 1) || m0 + m < M)
+               ? __ldg(reinterpret_cast<const uint16_t*>(p + static_cast<uint64_t>(row_bytes) * static_cast<uint32_t>(m)))
+               : 0u;
   uint32_t lo[kG4], hi[kG4], threes = 0;
 #pragma unroll
   for (int G = 0; G < kG4; ++G) {
@@ -571,8 +575,8 @@ decode_update_wide_kernel(const uint32_t* __restrict__ codes, const float* __res
   build_decode_lut3(sm_lut, scales, M);
   const uint32_t lut_lane =
       static_cast<uint32_t>(__cvta_generic_to_shared(sm_lut + (threadIdx.x & (kLut3Lanes - 1))));
-  const uint16_t* codes16 = reinterpret_cast<const uint16_t*>(codes);
-  const uint64_t row_halves = ((d + 15) >> 4) * 2;
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  const uint32_t row_bytes = static_cast<uint32_t>(((d + 15) >> 4) * 4);
   const uint64_t octs = (d + 7) >> 3, full = d >> 3;
   const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kWideThreads;
   constexpr int kBatch = 4;                         // worker groups per batch
@@ -590,10 +594,10 @@ decode_update_wide_kernel(const uint32_t* __restrict__ codes, const float* __res
     for (int i = 0; i < 8; ++i) q[i] = 0.0;
 #pragma unroll
     for (int b = 0; b < kWholeBatches; ++b)
-      bad |= decode_batch<kBatch, false>(codes16, row_halves, o, 4 * kBatch * b, M,
+      bad |= decode_batch<kBatch, false>(codes8, row_bytes, o, 4 * kBatch * b, M,
                                          lut_lane + b * (kBatch * kLut3Entries * kLut3Lanes * 8), q);
     bad |= decode_batch<kM4 - kBatch * kWholeBatches, true>(
-        codes16, row_halves, o, 4 * kBatch * kWholeBatches, M,
+        codes8, row_bytes, o, 4 * kBatch * kWholeBatches, M,
         lut_lane + kWholeBatches * (kBatch * kLut3Entries * kLut3Lanes * 8), q);
     float qf[8];
 #pragma unroll
@@ -1325,9 +1329,14 @@ static void launch_decode_update_rule(const uint32_t* codes, const float* scales
 #define QASG_LANES(m4, lanes) \
   case m4: launch_decode_update_as<kRule, m4, lanes, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_WIDE(m4) \
-  case m4: launch_decode_update_wide_as<kRule, m4>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+  case m4: \
+    if (wide) launch_decode_update_wide_as<kRule, m4>(codes, scales, d, M, x, h, z, sc, status, shape, stream); \
+    else launch_decode_update_as<kRule, m4, 8, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); \
+    break;
 #define QASG_SHARED(m4) \
   case m4: launch_decode_update_as<kRule, m4, 1, kThreads, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
+  // the eight-coordinate kernel addresses a worker's code row with a 32-bit byte count
+  const bool wide = ((d + 15) >> 4) * 4 <= 0xFFFFFFFFull;
   switch ((M + 3) / 4) {
     QASG_LANE(1) QASG_LANE(2) QASG_LANE(3)
     // 16 copies (32 KB per worker group) keep the two half-warps of a 64-bit lookup apart; 8 copies
