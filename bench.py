@@ -50,9 +50,9 @@ def bytes_per_coord(M):
 # capture summarised in profiles/step_kernels_d2p24_M8_ncu_full.md (d = 2^24; passes A and B stream,
 # so their traffic grows in proportion to d).  Valid only for the kernel source it was taken from.
 NCU_TRAFFIC = {
-    "kernels_sha256": "ca3ad323ae2e7f2698a4a37e086f946eedf920c11fd18c6a9413e7dd3e39d5ec",
+    "kernels_sha256": "15c39fbd299dd161025ec37617c0e0ae9bcdeef5e5b886510ff02a86c5f49841",
     "M": 8,
-    "bytes_per_coord": {"abs_sum": 540500736 / 2 ** 24, "threshold_codes": 567868928 / 2 ** 24},
+    "bytes_per_coord": {"abs_sum": 541067520 / 2 ** 24, "threshold_codes": 568647424 / 2 ** 24},
 }
 
 

@@ -5,7 +5,7 @@
 //           stochastic_codes_kernel             unbiased ternary codes from Philox draws
 //   pass C  decode_update_kernel                decode + average + accumulator + QCMD/QRDA (or the
 //                                               average alone), dense_update_kernel: update from a dense q
-//           decode_update_wide_kernel           the same for 13 to 32 workers, eight coordinates per thread
+//           decode_update_wide_kernel           the same with eight coordinates per thread (13 to 32 workers, some fewer)
 //   server  avg_abs_sum/avg_abs_max/avg_codes   double quantization: Q applied to the average
 //   select  select_stats, indicator_or          sparse selection: indicators, statistics over the selected
 //
@@ -462,7 +462,8 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
   if (bad) atomicOr(status, kFlagBadCode);
 }
 
-// ------------------------------------------------------------------ pass C for 13 workers and more
+// ------------------------------------------------------------------ pass C, eight coordinates per thread
+// Serves 13 to 32 workers, and fewer where it was measured faster (the launcher says which).
 // With many workers the byte-per-worker decode above is bound by integer instructions (address
 // arithmetic for one byte load per worker and four coordinates, the 2-bit transposition, the
 // field extraction), not by HBM.  Here a thread owns eight consecutive coordinates, so one
@@ -1324,8 +1325,6 @@ static void launch_decode_update_rule(const uint32_t* codes, const float* scales
                                       unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
   constexpr int kG = kRule == 1 ? 1 : 2;  // groups per thread with per-lane tables (measured best)
   // up to 12 workers: 16 copies of the tables (conflict-free for 64-bit lookups), two CTAs of 512 threads per SM
-#define QASG_LANE(m4) \
-  case m4: launch_decode_update_as<kRule, m4, 16, 512, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_LANES(m4, lanes) \
   case m4: launch_decode_update_as<kRule, m4, lanes, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
 #define QASG_WIDE(m4) \
@@ -1333,20 +1332,31 @@ static void launch_decode_update_rule(const uint32_t* codes, const float* scales
     if (wide) launch_decode_update_wide_as<kRule, m4>(codes, scales, d, M, x, h, z, sc, status, shape, stream); \
     else launch_decode_update_as<kRule, m4, 8, 1024, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); \
     break;
+#define QASG_EITHER(m4, prefer_wide) \
+  case m4: \
+    if constexpr (prefer_wide) { \
+      if (wide) { \
+        launch_decode_update_wide_as<kRule, m4>(codes, scales, d, M, x, h, z, sc, status, shape, stream); \
+        break; \
+      } \
+    } \
+    launch_decode_update_as<kRule, m4, 16, 512, kG>(codes, scales, d, M, x, h, z, sc, status, shape, stream); \
+    break;
 #define QASG_SHARED(m4) \
   case m4: launch_decode_update_as<kRule, m4, 1, kThreads, 1>(codes, scales, d, M, x, h, z, sc, status, shape, stream); break;
   // the eight-coordinate kernel addresses a worker's code row with a 32-bit byte count
   const bool wide = ((d + 15) >> 4) * 4 <= 0xFFFFFFFFull;
   switch ((M + 3) / 4) {
-    QASG_LANE(1) QASG_LANE(2) QASG_LANE(3)
-    // 16 copies (32 KB per worker group) keep the two half-warps of a 64-bit lookup apart; 8 copies
-    // leave two lanes per copy
+    // measured at d = 2^28: the eight-coordinate kernel also wins for QCMD from 4 workers on and for QRDA from 9 on
+    // (QRDA moves more state per coordinate and loses by loading it after the decode when the decode is short)
+    QASG_EITHER(1, kRule == 0) QASG_EITHER(2, kRule == 0) QASG_EITHER(3, kRule != 2)
     QASG_WIDE(4) QASG_WIDE(5) QASG_WIDE(6) QASG_WIDE(7) QASG_WIDE(8)
+    // 33 workers and more: 8 copies of the 256-entry tables (two lanes per copy), then one shared copy
     QASG_LANES(9, 8) QASG_LANES(10, 8) QASG_LANES(11, 8) QASG_LANES(12, 8) QASG_LANES(13, 8)
     QASG_SHARED(14) QASG_SHARED(15) QASG_SHARED(16)
   }
 #undef QASG_WIDE
-#undef QASG_LANE
+#undef QASG_EITHER
 #undef QASG_LANES
 #undef QASG_SHARED
 }
