@@ -494,6 +494,47 @@ def test_selected_quantizer_is_q_on_the_selected_subvector():
     assert np.array_equal(full[0], ref[0]) and full[1:4] == ref[1:]
 
 
+def test_selected_stochastic_quantizer_is_the_unbiased_quantizer_of_the_selected_subvector():
+    # Section 3.2 / 3.4: Q(S(v, I)) with the unbiased ternary Q.  The scale is the maximum over the
+    # SELECTED components (here the two largest magnitudes are not selected), unselected components
+    # code 0, and on the selected ones the codes are those of the quantizer applied to the compacted
+    # sub-vector with the same draws.
+    rng = np.random.default_rng(35)
+    d = 4000
+    v = rng.standard_normal(d).astype(np.float32)
+    sel = rng.random(d) < 0.4
+    big = np.argsort(-np.abs(v))[:2]
+    sel[big] = False
+    assert np.abs(v[sel]).max() < np.abs(v[big]).min()
+    u = rng.random(d).astype(np.float32)
+    tern, s = O.ternary_stochastic_quantize_selected(v, u, sel)
+    assert s == np.abs(v[sel]).max() and s < np.abs(v).max()
+    assert not tern[~sel].any()
+    want = (u[sel] < np.abs(v[sel]) / s).astype(np.int8) * np.sign(v[sel]).astype(np.int8)
+    assert np.array_equal(tern[sel], want)
+    sub_tern, sub_s = O.ternary_stochastic_quantize(v[sel], u[sel])
+    assert sub_s == s and np.array_equal(tern[sel], sub_tern)
+    # nothing selected: nothing is sent
+    none, s0 = O.ternary_stochastic_quantize_selected(v, u, np.zeros(d, bool))
+    assert s0 == 0 and not none.any()
+    # Monte Carlo over Philox draws: unbiased on the selected components, identically 0 elsewhere
+    g = np.array([0.9, -0.05, 3.0, 0.0, -1.2, 0.61, -7.0, -0.33], dtype=np.float32)
+    pick = np.array([1, 1, 0, 1, 1, 0, 0, 1], dtype=bool)
+    trials = 200_000
+    t = np.arange(1, trials + 1, dtype=np.uint64)[:, None]
+    _, draws = O.philox_draws(seed=5, t=t, m=1, idx=np.arange(g.size, dtype=np.uint64)[None, :])
+    total = np.zeros(g.size)
+    for row in draws:
+        tr, sr = O.ternary_stochastic_quantize_selected(g, row, pick)
+        total += float(sr) * tr
+    mean = total / trials
+    smax = float(np.abs(g[pick]).max())
+    p = np.where(pick, np.abs(g.astype(np.float64)) / smax, 0.0)
+    sigma = smax * np.sqrt(p * (1 - p) / trials)
+    assert (np.abs(mean - np.where(pick, g, 0.0)) <= 5 * sigma + 1e-12).all()
+    assert not mean[~pick].any()
+
+
 def test_indicator_words_or_and_sparse_bit_budget():
     rng = np.random.default_rng(34)
     d, M = 1000, 4
