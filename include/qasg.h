@@ -39,9 +39,10 @@ typedef enum {
   QASG_ERR_ALIGNMENT = 2,   /* pointer or leading dimension not aligned as required   */
   QASG_ERR_WORKSPACE = 3,   /* d or M beyond what the context was created for         */
   QASG_ERR_CUDA = 4,        /* a CUDA runtime call failed                             */
-  QASG_ERR_TIMEOUT = 5,     /* reserved: a bounded device-side wait ran out           */
+  QASG_ERR_TIMEOUT = 5,     /* (async) a bounded device-side wait ran out             */
   QASG_ERR_NONFINITE = 6,   /* (async) a gradient held NaN or Inf                     */
-  QASG_ERR_BAD_CODE = 7     /* (async) a packed code word held the unused value 3     */
+  QASG_ERR_BAD_CODE = 7,    /* (async) a packed code word held the unused value 3     */
+  QASG_ERR_BAD_INDEX = 8    /* (async) a row or column index of sparse data out of range */
 } qasg_status;
 
 /* The quantization function Q(.) applied to each worker's gradient. */
@@ -55,7 +56,11 @@ typedef enum {
    * Randomness: Philox4x32-10 (Salmon et al., SC'11), key (seed lo, seed hi), counter
    * (i>>2, m, t lo, t hi), coordinate i uses output word i&3, u = (word>>8) * 2^-24,
    * non-zero iff u < |v_i|/s in fp32. */
-  QASG_Q_TERNARY_STOCH = 1
+  QASG_Q_TERNARY_STOCH = 1,
+  /* No quantization: the 32-bit CMD adagrad / RDA adagrad the paper compares with
+   * (Section 5.1 "Baselines"; Eq. CMD adagrad, Eq. RDA adagrad).  Accepted by qasg_step
+   * and qasg_step_host only: q_t is the plain mean of the M fp32 gradients. */
+  QASG_Q_NONE = 2
 } qasg_quantizer;
 
 typedef enum {
@@ -85,6 +90,29 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
                         uint32_t flags);
 /* Frees the workspace.  The caller must have synchronized the streams it used. */
 qasg_status qasg_destroy(qasg_ctx* ctx);
+
+/* Options of a context (qasg_set_option).  Defaults suit a B200 (126 MB of L2).
+ *
+ * qasg_quantize_pack and qasg_step read every gradient row twice: once for the threshold of
+ * Section 3.5 (a sum over the whole row), once to cut the codes.  Rows of at most
+ * QASG_OPT_STREAM_ROW_BYTES bytes (4*d) are quantized by ONE cooperative launch that codes a row
+ * while it is still in the L2 cache, QASG_OPT_STREAM_LAG rows after it was summed, so that the
+ * gradients cross device memory once; its CTAs wait for one another through words in the
+ * context's workspace, every wait bounded by QASG_OPT_WAIT_POLLS polls (about 0.2 us each), after
+ * which the call gives up and qasg_last_async_status reports QASG_ERR_TIMEOUT (the outputs of that
+ * call are then incomplete).  Longer rows go through two launches (all sums, then all codes).  Both
+ * ways give the same bits. */
+typedef enum {
+  QASG_OPT_STREAM_ROW_BYTES = 0, /* 0 = always two launches; default 64 MiB                    */
+  QASG_OPT_STREAM_LAG = 1,       /* 0, 1, 2, ...; 0xFFFFFFFF = chosen from the row size (default) */
+  QASG_OPT_WAIT_POLLS = 2        /* 1 .. 2^31; default 2^22 (about a second)                   */
+} qasg_option;
+qasg_status qasg_set_option(qasg_ctx* ctx, qasg_option option, uint64_t value);
+
+/* Runs the bounded device-side wait on a word that nothing sets, with a bound of max_polls polls:
+ * the kernel returns by itself and the next qasg_last_async_status reports QASG_ERR_TIMEOUT.  This
+ * is how the give-up path of the waits is exercised without hanging anything. */
+qasg_status qasg_wait_selftest(qasg_ctx* ctx, uint32_t max_polls, void* stream);
 
 /* Number of 32-bit code words one worker's d codes occupy: ceil(d/16)
  * (Section 3.5 "Encode": 2 bits per coordinate). */
@@ -135,7 +163,12 @@ qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, flo
  * M/4 code bytes are written and read once, and h, x (z) cross memory once.
  *   rule        QASG_RULE_CMD (z may be NULL) or QASG_RULE_RDA (z required).
  *   codes_out   device uint32 [M][code_words(d)] or NULL to use the context's scratch.
- *   scales_out  device fp32 [M] or NULL. */
+ *   scales_out  device fp32 [M] or NULL.
+ * With params->quantizer = QASG_Q_NONE nothing is quantized: one pass reads the M gradients
+ * of a coordinate once, sums them in fp64 in worker order, q_i = fp32(sum * (1/M)), and applies
+ * the same accumulator and update (4M + 16 or 20 bytes per coordinate); codes_out and
+ * scales_out are not touched, thr_coef and seed are not used.  A non-finite mean is reported
+ * as QASG_ERR_NONFINITE and still enters the state, as it would in plain AdaGrad. */
 qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
                       uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h,
                       float* z, uint32_t* codes_out, float* scales_out, void* stream);
@@ -235,9 +268,15 @@ qasg_status qasg_logreg_grad_dense(qasg_ctx* ctx, const float* X, const float* y
                                    uint32_t B, uint64_t t, const float* x, float* g,
                                    uint64_t ld_g, void* stream);
 
-/* Same for a CSR matrix: rowptr device int64 [n_rows+1], colidx device int32 [nnz]
- * (0 <= colidx < d), vals device fp32 [nnz].  g rows are zeroed, then accumulated with
- * atomic adds (the summation order inside one coordinate is not fixed). */
+/* Same for a CSR matrix: rowptr device int64 [n_rows+1] (rowptr[n_rows] = nnz), colidx device
+ * int32 [nnz] (0 <= colidx < d), vals device fp32 [nnz].  g rows are zeroed, then accumulated
+ * with atomic adds: the summation order inside one coordinate is not fixed, so the last bits of
+ * g, and with them the codes of coordinates that sit within rounding of Delta_m, can differ from
+ * run to run.  The indices are checked on the device: a minibatch row id >= n_rows, a row whose
+ * rowptr pair is not 0 <= lo <= hi <= rowptr[n_rows], or an entry with a column outside [0, d)
+ * is skipped (it adds nothing and no memory outside the arguments is touched) and
+ * qasg_last_async_status reports QASG_ERR_BAD_INDEX.  The dense entry point checks batch_rows
+ * the same way. */
 qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
                                  const float* vals, const float* y, uint64_t n_rows,
                                  uint64_t d, uint32_t M, const uint64_t* shard_row0,
@@ -332,7 +371,8 @@ qasg_status qasg_quantize_pack_static(int device, const float* g, uint64_t d, ui
                                       float* thresholds, uint64_t* counts, void* stream);
 
 /* Waits for `stream`, then returns and clears the conditions kernels recorded since
- * the last call: QASG_ERR_NONFINITE, QASG_ERR_BAD_CODE, QASG_ERR_CUDA, else QASG_OK. */
+ * the last call: QASG_ERR_TIMEOUT, QASG_ERR_NONFINITE, QASG_ERR_BAD_CODE, QASG_ERR_BAD_INDEX,
+ * QASG_ERR_CUDA, else QASG_OK (the first of these that applies). */
 qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream);
 
 /* Number of kernels this context has launched since it was created. */

@@ -273,18 +273,25 @@ def philox_draws(seed, t, m, idx, domain=0):
     return word, u
 
 
-def ternary_stochastic_quantize(v, u):
+def ternary_stochastic_quantize(v, u, scale=None):
     """Unbiased ternary quantizer with the max-norm scaler (the comparison quantizer
     of Section 3.4 / related work: levels {-1, 0, 1} times a scaler).
 
     s = max_i |v_i|;  tern_i = sign(v_i) with probability |v_i| / s, else 0, realised
     as  u_i < |v_i| / s  with the fp32 division and the given uniforms u in [0, 1).
     Returns (tern int8[d], s fp32).  s = 0 gives all zeros.
+
+    scale: when v is a slice of a longer vector, the scaler of that whole vector (its
+    maximum magnitude, which the caller has taken); the slice's codes are then the
+    corresponding slice of the whole vector's codes.
     """
     v = np.asarray(v, dtype=F32).ravel()
     u = np.asarray(u, dtype=F32).ravel()
     absv = np.abs(v)
-    s = F32(absv.max()) if v.size else F32(0.0)
+    if scale is None:
+        s = F32(absv.max()) if v.size else F32(0.0)
+    else:
+        s = F32(scale)
     if not s > 0:
         return np.zeros(v.size, dtype=np.int8), F32(0.0)
     prob = absv / s

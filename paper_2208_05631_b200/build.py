@@ -7,7 +7,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "lib", "libqasg.so")
-SOURCES = ["qasg_api.cu", "qasg_kernels.cu", "qasg_logreg.cu", "qasg_static.cu", "qasg_optimal.cu", "qasg_touched.cu"]
+SOURCES = ["qasg_api.cu", "qasg_kernels.cu", "qasg_logreg.cu", "qasg_static.cu", "qasg_optimal.cu", "qasg_touched.cu",
+           "qasg_stream.cu"]
 HEADERS = [os.path.join(CSRC, "qasg_internal.h"), os.path.join(CSRC, "qasg_device.cuh"),
            os.path.join(os.path.dirname(HERE), "include", "qasg.h")]
 

@@ -21,6 +21,10 @@ struct qasg_ctx {
   uint32_t* ind_scratch;    // [M_max + 1][ceil(d_max/32)] or NULL: workers' indicators, then their OR
   unsigned long long* ksyn; // [1] number of bits of the synchronous indicator
   float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
+  StreamSync* sync;         // words the CTAs of the one-launch quantizer wait on
+  uint64_t stream_row_bytes;  // rows up to this size are quantized by the one-launch kernel
+  uint32_t stream_lag;      // kAutoLag: chosen from the row size
+  uint32_t wait_polls;
   uint64_t launches;
   bool profiling;
   std::vector<cudaEvent_t> events;  // pairs (start, stop), reused between profiles
@@ -33,7 +37,7 @@ enum KernelId {
   kAbsSum = 0, kAbsMax, kThresholdCodes, kStochasticCodes, kDecodeUpdateCmd, kDecodeUpdateRda,
   kDecodeAverage, kDenseUpdateCmd, kDenseUpdateRda, kLogregDense, kLogregCsr, kAvgAbsSum, kAvgAbsMax,
   kAvgThresholdCodes, kAvgStochasticCodes, kSelectStats, kIndicatorOr, kTouchedClear, kLogregCsrTouched,
-  kOptimalThreshold, kKernelIdCount
+  kOptimalThreshold, kMeanUpdateCmd, kMeanUpdateRda, kStreamThreshold, kStreamStochastic, kKernelIdCount
 };
 static_assert(kKernelIdCount <= QASG_KERNEL_COUNT, "kernel id table");
 
@@ -64,20 +68,30 @@ struct Launch {
 };
 
 constexpr uint64_t kMaxD = 1ull << 34;
+constexpr uint32_t kAutoLag = 0xFFFFFFFFu;
+constexpr uint64_t kDefaultStreamRowBytes = 64ull << 20;
+// A row is coded `lag` rows after it was summed; in between the rows summed and coded meanwhile pass
+// through L2.  One row of lag hides the wait for a worker's threshold; it is taken while three rows fit.
+constexpr uint64_t kLagOneRowBytes = 24ull << 20;
+// Code rows small enough to stay in L2 until pass C reads them are written with ordinary stores.
+constexpr uint64_t kKeepCodesBytes = 32ull << 20;
 constexpr uint64_t kLogregEntries = 1ull << 20;  // M * B of one gradient call
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-qasg_status check_params(const qasg_params* p, bool need_update) {
+qasg_status check_params_update(const qasg_params* p) {
+  if (!(p->lambda >= 0.f) || !isfinite(p->lambda)) return QASG_ERR_INVALID_ARG;
+  if (!(p->eta > 0.f) || !isfinite(p->eta)) return QASG_ERR_INVALID_ARG;
+  if (!(p->delta > 0.f) || !isfinite(p->delta)) return QASG_ERR_INVALID_ARG;
+  return QASG_OK;
+}
+
+qasg_status check_params(const qasg_params* p, bool need_update, bool allow_none = false) {
   if (!p || p->struct_size != sizeof(qasg_params)) return QASG_ERR_INVALID_ARG;
+  if (p->quantizer == QASG_Q_NONE) return allow_none && need_update ? check_params_update(p) : QASG_ERR_INVALID_ARG;
   if (p->quantizer != QASG_Q_THRESHOLD && p->quantizer != QASG_Q_TERNARY_STOCH) return QASG_ERR_INVALID_ARG;
   if (!(p->thr_coef > 0.f) || !isfinite(p->thr_coef)) return QASG_ERR_INVALID_ARG;
-  if (need_update) {
-    if (!(p->lambda >= 0.f) || !isfinite(p->lambda)) return QASG_ERR_INVALID_ARG;
-    if (!(p->eta > 0.f) || !isfinite(p->eta)) return QASG_ERR_INVALID_ARG;
-    if (!(p->delta > 0.f) || !isfinite(p->delta)) return QASG_ERR_INVALID_ARG;
-  }
-  return QASG_OK;
+  return need_update ? check_params_update(p) : QASG_OK;
 }
 
 qasg_status check_shape(const qasg_ctx* ctx, uint64_t d, uint32_t M) {
@@ -129,6 +143,22 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
                                 stream);
     }
     if (stochastic && thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
+    return;
+  }
+  if (d * sizeof(float) <= ctx->stream_row_bytes) {  // one launch, each row coded out of L2
+    const bool stochastic = p->quantizer != QASG_Q_THRESHOLD;
+    StreamParams sp;
+    sp.coef = p->thr_coef;
+    sp.lag = ctx->stream_lag != kAutoLag ? ctx->stream_lag : (d * sizeof(float) <= kLagOneRowBytes ? 1u : 0u);
+    if (sp.lag > M) sp.lag = M;
+    sp.max_polls = ctx->wait_polls;
+    sp.stream_base = 0u;
+    sp.seed = p->seed;
+    sp.t = t;
+    const bool keep_codes = static_cast<uint64_t>(M) * qasg_code_words(d) * 4 <= kKeepCodesBytes;
+    Launch l(ctx, stochastic ? kStreamStochastic : kStreamThreshold, stream);
+    l += launch_quantize_stream(stochastic, keep_codes, g, geo, sp, ctx->ws, ctx->sync, codes, scales, thresholds,
+                                counts_out, ctx->shape, stream);
     return;
   }
   if (p->quantizer == QASG_Q_THRESHOLD) {
@@ -217,6 +247,23 @@ qasg_status check_gradient(const float* g, uint64_t d, uint64_t ld_g) {
   return QASG_OK;
 }
 
+// Everything qasg_step checks before it enqueues anything (shared with qasg_step_host, which must not
+// start a copy for a call that will be refused).
+qasg_status check_step(const qasg_ctx* ctx, int rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
+                       uint64_t t, const qasg_params* params, const float* x, const float* h, const float* z,
+                       const uint32_t* codes_out) {
+  qasg_status st = check_shape(ctx, d, M);
+  if (st == QASG_OK) st = check_params(params, true, true);
+  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  if (st != QASG_OK) return st;
+  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
+  if (!x || !h || t < 1 || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(h) || (z && !aligned16(z)) || (codes_out && !aligned16(codes_out)))
+    return QASG_ERR_ALIGNMENT;
+  if (params->quantizer != QASG_Q_NONE && !codes_out && !ctx->code_scratch) return QASG_ERR_WORKSPACE;
+  return QASG_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -234,6 +281,9 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ctx->M_max = M_max;
   ctx->launches = 0;
   ctx->profiling = false;
+  ctx->stream_row_bytes = kDefaultStreamRowBytes;
+  ctx->stream_lag = kAutoLag;
+  ctx->wait_polls = 1u << 22;
   query_launch_shape(&ctx->shape);
   const size_t slots = static_cast<size_t>(M_max) * kMaxChunks;
   bool ok = true;
@@ -248,6 +298,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ok &= cudaMalloc(&ctx->ws.ticket, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->ws.status, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->logreg_ws, kLogregEntries * 2 * sizeof(float)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->sync, sizeof(StreamSync)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.part_sum, kRowChunks * sizeof(double)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.part_max, kRowChunks * sizeof(uint32_t)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.part_cnt, kRowChunks * sizeof(unsigned long long)) == cudaSuccess;
@@ -266,6 +317,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   if (ok) {
     ok &= cudaMemset(ctx->ws.ticket, 0, 64) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.status, 0, 64) == cudaSuccess;
+    ok &= cudaMemset(ctx->sync, 0, sizeof(StreamSync)) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.thresholds, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.scales, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
     ok &= cudaMemset(ctx->wsq.thresholds, 0, 64) == cudaSuccess;
@@ -292,6 +344,7 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->ws.ticket);
   cudaFree(ctx->ws.status);
   cudaFree(ctx->logreg_ws);
+  cudaFree(ctx->sync);
   cudaFree(ctx->code_scratch);
   cudaFree(ctx->qcode_scratch);
   cudaFree(ctx->gbar_scratch);
@@ -311,6 +364,32 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
 }
 
 uint64_t qasg_code_words(uint64_t d) { return (d + 15) >> 4; }
+
+qasg_status qasg_set_option(qasg_ctx* ctx, qasg_option option, uint64_t value) {
+  if (!ctx) return QASG_ERR_INVALID_ARG;
+  switch (option) {
+    case QASG_OPT_STREAM_ROW_BYTES:
+      ctx->stream_row_bytes = value;
+      return QASG_OK;
+    case QASG_OPT_STREAM_LAG:
+      if (value != kAutoLag && value > static_cast<uint64_t>(kMaxWorkers)) return QASG_ERR_INVALID_ARG;
+      ctx->stream_lag = static_cast<uint32_t>(value);
+      return QASG_OK;
+    case QASG_OPT_WAIT_POLLS:
+      if (value < 1 || value > (1ull << 31)) return QASG_ERR_INVALID_ARG;
+      ctx->wait_polls = static_cast<uint32_t>(value);
+      return QASG_OK;
+  }
+  return QASG_ERR_INVALID_ARG;
+}
+
+qasg_status qasg_wait_selftest(qasg_ctx* ctx, uint32_t max_polls, void* stream) {
+  if (!ctx || max_polls < 1 || max_polls > (1u << 24)) return QASG_ERR_INVALID_ARG;
+  qasg_status st = enter(ctx);
+  if (st != QASG_OK) return st;
+  ctx->launches += launch_wait_selftest(ctx->sync, ctx->ws.status, max_polls, static_cast<cudaStream_t>(stream));
+  return leave();
+}
 
 qasg_status qasg_quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
                                uint64_t t, const qasg_params* params, uint32_t* codes, float* scales,
@@ -368,18 +447,16 @@ qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, flo
 qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
                       uint64_t t, const qasg_params* params, float* x, float* h, float* z,
                       uint32_t* codes_out, float* scales_out, void* stream) {
-  qasg_status st = check_shape(ctx, d, M);
-  if (st == QASG_OK) st = check_params(params, true);
-  if (st == QASG_OK) st = check_gradient(g, d, ld_g);
+  qasg_status st = check_step(ctx, rule, g, d, ld_g, M, t, params, x, h, z, codes_out);
   if (st != QASG_OK) return st;
-  if (rule != QASG_RULE_CMD && rule != QASG_RULE_RDA) return QASG_ERR_INVALID_ARG;
-  if (!x || !h || t < 1 || (rule == QASG_RULE_RDA && !z)) return QASG_ERR_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(h) || (z && !aligned16(z)) || (codes_out && !aligned16(codes_out)))
-    return QASG_ERR_ALIGNMENT;
-  uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
-  if (!codes) return QASG_ERR_WORKSPACE;
   if ((st = enter(ctx)) != QASG_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (params->quantizer == QASG_Q_NONE) {
+    Launch l(ctx, rule == QASG_RULE_CMD ? kMeanUpdateCmd : kMeanUpdateRda, s);
+    l += launch_mean_update(rule, g, d, ld_g, M, x, h, z, scalars(params, t), ctx->ws.status, ctx->shape, s);
+    return leave();
+  }
+  uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
   { Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s); l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
                                         ctx->ws.status, ctx->shape, s); }
@@ -579,11 +656,10 @@ qasg_status qasg_step_host(qasg_ctx* ctx, qasg_rule rule, const float* g_host, u
                            uint32_t M, uint64_t t, const qasg_params* params, float* x_host, float* h_host,
                            float* z_host, float* g_dev, float* x_dev, float* h_dev, float* z_dev,
                            void* stream) {
-  qasg_status st = check_shape(ctx, d, M);
+  // every check of qasg_step on the staging buffers comes first: a refused call copies nothing
+  qasg_status st = check_step(ctx, rule, g_dev, d, ld_g, M, t, params, x_dev, h_dev, z_dev, nullptr);
   if (st != QASG_OK) return st;
-  if (!g_host || !x_host || !h_host || !g_dev || !x_dev || !h_dev) return QASG_ERR_INVALID_ARG;
-  if (rule == QASG_RULE_RDA && (!z_host || !z_dev)) return QASG_ERR_INVALID_ARG;
-  if (ld_g < d) return QASG_ERR_INVALID_ARG;
+  if (!g_host || !x_host || !h_host || (rule == QASG_RULE_RDA && !z_host)) return QASG_ERR_INVALID_ARG;
   if ((st = enter(ctx)) != QASG_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t vec = d * sizeof(float);
@@ -633,8 +709,8 @@ qasg_status qasg_logreg_grad_dense(qasg_ctx* ctx, const float* X, const float* y
   if (!X) return QASG_ERR_INVALID_ARG;
   if ((d & 3u) || !aligned16(X)) return QASG_ERR_ALIGNMENT;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  { Launch l(ctx, kLogregDense, static_cast<cudaStream_t>(stream)); l += launch_logreg_dense(X, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->logreg_ws,
-                                       ctx->shape, static_cast<cudaStream_t>(stream)); }
+  { Launch l(ctx, kLogregDense, static_cast<cudaStream_t>(stream)); l += launch_logreg_dense(X, y, n_rows, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->logreg_ws,
+                                       ctx->ws.status, ctx->shape, static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -646,8 +722,8 @@ qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int
   if (st != QASG_OK) return st;
   if (!rowptr || !colidx || !vals) return QASG_ERR_INVALID_ARG;
   if ((st = enter(ctx)) != QASG_OK) return st;
-  { Launch l(ctx, kLogregCsr, static_cast<cudaStream_t>(stream)); l += launch_logreg_csr(rowptr, colidx, vals, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
-                                     ctx->shape, static_cast<cudaStream_t>(stream)); }
+  { Launch l(ctx, kLogregCsr, static_cast<cudaStream_t>(stream)); l += launch_logreg_csr(rowptr, colidx, vals, y, n_rows, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
+                                     ctx->ws.status, ctx->shape, static_cast<cudaStream_t>(stream)); }
   return leave();
 }
 
@@ -665,7 +741,8 @@ qasg_status qasg_logreg_grad_csr_touched(qasg_ctx* ctx, const int64_t* rowptr, c
   { Launch l(ctx, kTouchedClear, s); l += launch_touched_clear(g, d, ld_g, M, touched, ctx->shape, s); }
   {
     Launch l(ctx, kLogregCsrTouched, s);
-    l += launch_logreg_csr(rowptr, colidx, vals, y, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->shape, s,
+    l += launch_logreg_csr(rowptr, colidx, vals, y, n_rows, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
+                           ctx->ws.status, ctx->shape, s,
                            touched);
   }
   return leave();
@@ -682,8 +759,14 @@ qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream) {
     cudaGetLastError();
     return QASG_ERR_CUDA;
   }
+  if (flags & kFlagTimeout) {  // a call gave up half-way: its tickets and abort word are left set
+    cudaMemsetAsync(ctx->sync, 0, sizeof(StreamSync), s);
+    cudaStreamSynchronize(s);
+    return QASG_ERR_TIMEOUT;
+  }
   if (flags & kFlagNonFinite) return QASG_ERR_NONFINITE;
   if (flags & kFlagBadCode) return QASG_ERR_BAD_CODE;
+  if (flags & kFlagBadIndex) return QASG_ERR_BAD_INDEX;
   return QASG_OK;
 }
 
@@ -723,7 +806,8 @@ const char* qasg_kernel_name(int id) {
       "abs_sum", "abs_max", "threshold_codes", "stochastic_codes", "decode_update_cmd", "decode_update_rda",
       "decode_average", "dense_update_cmd", "dense_update_rda", "logreg_dense", "logreg_csr", "avg_abs_sum",
       "avg_abs_max", "avg_threshold_codes", "avg_stochastic_codes", "select_stats", "indicator_or",
-      "touched_clear", "logreg_csr_touched", "optimal_threshold"};
+      "touched_clear", "logreg_csr_touched", "optimal_threshold", "mean_update_cmd", "mean_update_rda",
+      "quantize_stream_threshold", "quantize_stream_stochastic"};
   return (id >= 0 && id < kKernelIdCount) ? names[id] : "";
 }
 
@@ -737,6 +821,7 @@ const char* qasg_status_string(qasg_status s) {
     case QASG_ERR_TIMEOUT: return "device-side wait timed out";
     case QASG_ERR_NONFINITE: return "non-finite gradient";
     case QASG_ERR_BAD_CODE: return "invalid code value in packed words";
+    case QASG_ERR_BAD_INDEX: return "row or column index out of range";
   }
   return "unknown status";
 }

@@ -21,7 +21,7 @@ constexpr int kMaxWorkers = 64;
 // The server row (the averaged gradient, re-quantized) is one long row: it may use more chunks.
 constexpr int kRowChunks = 8 * kMaxChunks;
 
-enum : unsigned { kFlagNonFinite = 1u, kFlagBadCode = 2u };
+enum : unsigned { kFlagNonFinite = 1u, kFlagBadCode = 2u, kFlagBadIndex = 4u, kFlagTimeout = 8u };
 
 struct Geometry {
   uint64_t d;       // coordinates per worker
@@ -47,6 +47,25 @@ struct Workspace {
   unsigned long long* selected;  // [M_max] coordinates the worker's indicator selects (sparse selection)
   unsigned int* ticket;          // grid-completion counter, zero between launches
   unsigned int* status;          // OR of kFlag*
+};
+
+// Words the CTAs of the one-launch quantizer (qasg_stream.cu) synchronise through.  All of them are back
+// at zero when a call completes (the CTA that ends a worker's last item resets that worker's words), so a
+// captured launch can be replayed; a call that gave up leaves them set and the host clears them.
+struct StreamSync {
+  unsigned int ticket_a[kMaxWorkers];  // sum items of worker m completed in this call
+  unsigned int ticket_b[kMaxWorkers];  // code items of worker m completed in this call
+  unsigned int ready[kMaxWorkers];     // 1 once worker m's threshold (or scaler) of this call is published
+  unsigned int abort;                  // non-zero once a wait ran out: every later wait returns at once
+  unsigned int probe, probe_abort;     // the wait self-test's own words (nothing ever sets probe)
+};
+
+struct StreamParams {
+  float coef;            // threshold coefficient (0.75)
+  uint32_t lag;          // rows between a worker's sum and its codes, 0 <= lag <= M
+  uint32_t max_polls;    // bound of every wait
+  uint32_t stream_base;  // Philox counter word 1 = stream_base + worker
+  uint64_t seed, t;
 };
 
 struct LaunchShape {
@@ -104,16 +123,22 @@ int launch_avg_codes(bool stochastic, const uint32_t* codes, const float* scales
                      cudaStream_t stream);
 int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h, float* z,
                         const StepScalars& sc, const LaunchShape& shape, cudaStream_t stream);
+// No quantization: q = mean of the M rows of g (fp64 sum in worker order), then the update of `rule`.
+int launch_mean_update(int rule, const float* g, uint64_t d, uint64_t ld, uint32_t M, float* x, float* h, float* z,
+                       const StepScalars& sc, unsigned int* status, const LaunchShape& shape, cudaStream_t stream);
 
 // margins_ws: device fp32 [M*B] scratch for the per-row coefficients.
-int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
+// status: the context's flag word; row ids >= n_rows and (CSR) broken rowptr pairs or columns outside
+// [0, d) are skipped and raise kFlagBadIndex.
+int launch_logreg_dense(const float* X, const float* y, uint64_t n_rows, uint64_t d, uint32_t M,
                         const uint64_t* shard_row0_host, const uint32_t* batch_rows, uint32_t B,
                         uint64_t t, const float* x, float* g, uint64_t ld_g, float* coef_ws,
-                        const LaunchShape& shape, cudaStream_t stream);
+                        unsigned int* status, const LaunchShape& shape, cudaStream_t stream);
 int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float* vals,
-                      const float* y, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
+                      const float* y, uint64_t n_rows, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
                       const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
-                      uint64_t ld_g, const LaunchShape& shape, cudaStream_t stream, uint32_t* touched = nullptr);
+                      uint64_t ld_g, unsigned int* status, const LaunchShape& shape, cudaStream_t stream,
+                      uint32_t* touched = nullptr);
 // With `touched` the launcher does not clear g: it adds into rows that are zero wherever the bits are zero
 // and sets the bit of every entry it adds to.  launch_touched_clear re-establishes that state from the
 // bits a previous gradient left: zeroes the marked entries of g, then the bits.
@@ -137,6 +162,15 @@ int launch_touched_codes(bool stochastic, const float* g, const Geometry& geo, u
 uint64_t optimal_scratch_bytes(uint64_t d);
 int launch_optimal_threshold(const float* row, uint64_t d, void* scratch, float* ws_threshold, float* threshold_out,
                              unsigned long long* kept_out, unsigned int* status, cudaStream_t stream);
+
+// Passes A and B in one cooperative launch (rows that fit L2); results as launch_abs_sum/abs_max followed
+// by launch_threshold_codes/stochastic_codes.  keep_codes: ordinary instead of streaming code stores.
+int launch_quantize_stream(bool stochastic, bool keep_codes, const float* g, const Geometry& geo,
+                           const StreamParams& sp, const Workspace& ws, StreamSync* sync, uint32_t* codes,
+                           float* scales_out, float* thresholds_out, unsigned long long* counts_out,
+                           const LaunchShape& shape, cudaStream_t stream);
+// One bounded wait on a word nothing sets: raises kFlagTimeout after max_polls polls.
+int launch_wait_selftest(StreamSync* sync, unsigned int* status, uint32_t max_polls, cudaStream_t stream);
 
 void query_launch_shape(LaunchShape* shape);
 

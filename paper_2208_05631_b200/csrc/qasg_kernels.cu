@@ -704,6 +704,86 @@ dense_update_kernel(const float* __restrict__ q, uint64_t d, float* __restrict__
   }
 }
 
+// ------------------------------------------------------------------ pass C without quantization
+// q_t = plain mean of the M fp32 gradients (32-bit CMD / RDA adagrad): per coordinate the M values
+// are read once, summed in fp64 in worker order, scaled by 1/M and rounded to fp32; then the same
+// accumulator and update as above.  A thread owns four coordinates; eight rows are in flight at a time.
+template <int kRule>
+__global__ void __launch_bounds__(kThreads)
+mean_update_kernel(const float* __restrict__ g, uint64_t d, uint64_t ld, uint32_t M, double inv_m,
+                   float* __restrict__ x, float* __restrict__ h, float* __restrict__ z, StepScalars sc,
+                   unsigned int* __restrict__ status) {
+  const uint64_t full = d >> 2;
+  const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+  const uint64_t first = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  bool nonfinite = false;
+  for (uint64_t grp = first; grp < full; grp += stride) {
+    float4 hv = *reinterpret_cast<const float4*>(h + 4 * grp);
+    float4 av = *reinterpret_cast<const float4*>((kRule == 0 ? x : z) + 4 * grp);
+    const float* p = g + 4 * grp;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    uint32_t m = 0;
+    for (; m + 8 <= M; m += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = load_f4(p + static_cast<uint64_t>(m + k) * ld);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        a0 += static_cast<double>(v[k].x);
+        a1 += static_cast<double>(v[k].y);
+        a2 += static_cast<double>(v[k].z);
+        a3 += static_cast<double>(v[k].w);
+      }
+    }
+    for (; m < M; ++m) {
+      const float4 v = load_f4(p + static_cast<uint64_t>(m) * ld);
+      a0 += static_cast<double>(v.x);
+      a1 += static_cast<double>(v.y);
+      a2 += static_cast<double>(v.z);
+      a3 += static_cast<double>(v.w);
+    }
+    const float4 q = make_float4(static_cast<float>(a0 * inv_m), static_cast<float>(a1 * inv_m),
+                                 static_cast<float>(a2 * inv_m), static_cast<float>(a3 * inv_m));
+    nonfinite |= !(fabsf(q.x) <= 3.402823466e38f) | !(fabsf(q.y) <= 3.402823466e38f) |
+                 !(fabsf(q.z) <= 3.402823466e38f) | !(fabsf(q.w) <= 3.402823466e38f);
+    if (kRule == 0) {
+      cmd_update(q.x, av.x, hv.x, sc);
+      cmd_update(q.y, av.y, hv.y, sc);
+      cmd_update(q.z, av.z, hv.z, sc);
+      cmd_update(q.w, av.w, hv.w, sc);
+      *reinterpret_cast<float4*>(x + 4 * grp) = av;
+    } else {
+      float4 xv;
+      rda_update(q.x, xv.x, hv.x, av.x, sc);
+      rda_update(q.y, xv.y, hv.y, av.y, sc);
+      rda_update(q.z, xv.z, hv.z, av.z, sc);
+      rda_update(q.w, xv.w, hv.w, av.w, sc);
+      *reinterpret_cast<float4*>(z + 4 * grp) = av;
+      *reinterpret_cast<float4*>(x + 4 * grp) = xv;
+    }
+    *reinterpret_cast<float4*>(h + 4 * grp) = hv;
+  }
+  if (first == 0) {  // ragged tail: d % 4 coordinates
+    for (uint64_t i = 4 * full; i < d; ++i) {
+      double acc = 0.0;
+      for (uint32_t m = 0; m < M; ++m) acc += static_cast<double>(g[static_cast<uint64_t>(m) * ld + i]);
+      const float q = static_cast<float>(acc * inv_m);
+      nonfinite |= !(fabsf(q) <= 3.402823466e38f);
+      float xi = (kRule == 0) ? x[i] : 0.f, hi = h[i];
+      if (kRule == 0) {
+        cmd_update(q, xi, hi, sc);
+      } else {
+        float zi = z[i];
+        rda_update(q, xi, hi, zi, sc);
+        z[i] = zi;
+      }
+      x[i] = xi;
+      h[i] = hi;
+    }
+  }
+  if (nonfinite) atomicOr(status, kFlagNonFinite);
+}
+
 // ------------------------------------------------------------------ server row: q = Q(average)
 // Double quantization (Algorithm 1, "Quantize the aggregated gradient"): the averaged gradient is
 // quantized again with the same Q.  The average is never stored: these kernels rebuild it from the
@@ -1390,6 +1470,17 @@ int launch_dense_update(int rule, const float* q, uint64_t d, float* x, float* h
   return 1;
 }
 
+
+int launch_mean_update(int rule, const float* g, uint64_t d, uint64_t ld, uint32_t M, float* x, float* h, float* z,
+                       const StepScalars& sc, unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
+  const unsigned grid = update_grid(d, shape);
+  const double inv_m = 1.0 / static_cast<double>(M);
+  if (rule == 0)
+    mean_update_kernel<0><<<grid, kThreads, 0, stream>>>(g, d, ld, M, inv_m, x, h, z, sc, status);
+  else
+    mean_update_kernel<1><<<grid, kThreads, 0, stream>>>(g, d, ld, M, inv_m, x, h, z, sc, status);
+  return 1;
+}
 
 static unsigned row_grid(const Geometry& geo, const LaunchShape& shape) {
   const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * shape.reduce_ctas_per_sm;

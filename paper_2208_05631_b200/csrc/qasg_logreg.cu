@@ -36,13 +36,22 @@ __device__ __forceinline__ float logistic_coef(float y, float s, float inv_b) {
 }
 
 __global__ void __launch_bounds__(kThreads)
-logreg_dense_coef_kernel(const float* __restrict__ X, const float* __restrict__ y, uint64_t d, uint32_t M,
-                         Shards sh, const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t,
-                         const float* __restrict__ x, float* __restrict__ coef, uint32_t* __restrict__ rows) {
+logreg_dense_coef_kernel(const float* __restrict__ X, const float* __restrict__ y, uint64_t n_rows, uint64_t d,
+                         uint32_t M, Shards sh, const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t,
+                         const float* __restrict__ x, float* __restrict__ coef, uint32_t* __restrict__ rows,
+                         unsigned int* __restrict__ status) {
   const uint32_t warp = (blockIdx.x * kThreads + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= M * B) return;
   const uint32_t m = warp / B, b = warp - m * B;
   const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
+  if (r >= n_rows) {  // a caller's row id outside the matrix: the row adds nothing
+    if (lane == 0) {
+      coef[warp] = 0.f;
+      rows[warp] = 0u;
+      atomicOr(status, kFlagBadIndex);
+    }
+    return;
+  }
   const float4* a = reinterpret_cast<const float4*>(X + r * d);
   const float4* xv = reinterpret_cast<const float4*>(x);
   float acc = 0.f;
@@ -108,9 +117,10 @@ constexpr uint32_t kHotCols = 4096;
 template <bool kTouched>
 __global__ void __launch_bounds__(kThreads)
 logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ colidx,
-                  const float* __restrict__ vals, const float* __restrict__ y, uint64_t d, Shards sh,
-                  const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t, const float* __restrict__ x,
-                  float* __restrict__ g, uint64_t ld_g, uint32_t* __restrict__ touched, uint64_t touched_words) {
+                  const float* __restrict__ vals, const float* __restrict__ y, uint64_t n_rows, uint64_t d,
+                  Shards sh, const uint32_t* __restrict__ batch_rows, uint32_t B, uint64_t t,
+                  const float* __restrict__ x, float* __restrict__ g, uint64_t ld_g, uint32_t* __restrict__ touched,
+                  uint64_t touched_words, unsigned int* __restrict__ status) {
   __shared__ float hot[kHotCols];
   __shared__ uint32_t hot_bits[kHotCols / 32];
   const uint32_t m = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -119,17 +129,40 @@ logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict_
   if (threadIdx.x < kHotCols / 32) hot_bits[threadIdx.x] = 0u;
   __syncthreads();
   float* row = g + static_cast<uint64_t>(m) * ld_g;
+  // Indices come from the caller's data: a row id, a rowptr pair or a column outside its range is
+  // skipped and reported, never used as an address.
+  bool bad_index = false;
+  const uint64_t r = b < B ? batch_row(sh, batch_rows, m, b, B, t) : 0;
+  int64_t lo = 0, hi = 0;
   if (b < B) {
-    const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
-    const int64_t lo = rowptr[r], hi = rowptr[r + 1];
+    if (r < n_rows) {
+      lo = rowptr[r];
+      hi = rowptr[r + 1];
+      if (lo < 0 || hi < lo || hi > rowptr[n_rows]) {
+        bad_index = true;
+        hi = lo = 0;
+      }
+    } else {
+      bad_index = true;
+    }
+  }
+  if (b < B && hi > lo) {
     float acc = 0.f;
-    for (int64_t k = lo + lane; k < hi; k += 32) acc = fmaf(__ldg(vals + k), __ldg(x + __ldg(colidx + k)), acc);
+    for (int64_t k = lo + lane; k < hi; k += 32) {
+      const int32_t col = __ldg(colidx + k);
+      if (col >= 0 && static_cast<uint64_t>(col) < d) acc = fmaf(__ldg(vals + k), __ldg(x + col), acc);
+    }
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
     const float c = logistic_coef(y[r], acc, 1.f / static_cast<float>(B));
     uint32_t* bits = kTouched ? touched + static_cast<uint64_t>(m) * touched_words : nullptr;
     for (int64_t k = lo + lane; k < hi; k += 32) {
-      const uint32_t col = static_cast<uint32_t>(__ldg(colidx + k));
+      const int32_t signed_col = __ldg(colidx + k);
+      if (signed_col < 0 || static_cast<uint64_t>(signed_col) >= d) {
+        bad_index = true;
+        continue;
+      }
+      const uint32_t col = static_cast<uint32_t>(signed_col);
       const float add = c * __ldg(vals + k);
       const uint32_t bit = 1u << (col & 31u);
       if (col < kHotCols) {
@@ -142,6 +175,7 @@ logreg_csr_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict_
       }
     }
   }
+  if (bad_index) atomicOr(status, kFlagBadIndex);
   __syncthreads();
   const uint32_t hot_cols = d < kHotCols ? static_cast<uint32_t>(d) : kHotCols;
   for (uint32_t c = threadIdx.x; c < hot_cols; c += kThreads) {
@@ -199,33 +233,35 @@ static Shards make_shards(const uint64_t* shard_row0_host, uint32_t M) {
   return sh;
 }
 
-int launch_logreg_dense(const float* X, const float* y, uint64_t d, uint32_t M,
+int launch_logreg_dense(const float* X, const float* y, uint64_t n_rows, uint64_t d, uint32_t M,
                         const uint64_t* shard_row0_host, const uint32_t* batch_rows, uint32_t B,
                         uint64_t t, const float* x, float* g, uint64_t ld_g, float* coef_ws,
-                        const LaunchShape&, cudaStream_t stream) {
+                        unsigned int* status, const LaunchShape&, cudaStream_t stream) {
   const Shards sh = make_shards(shard_row0_host, M);
   uint32_t* rows_ws = reinterpret_cast<uint32_t*>(coef_ws + static_cast<uint64_t>(M) * B);
   const uint64_t warps = static_cast<uint64_t>(M) * B;
   const unsigned grid1 = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
-  logreg_dense_coef_kernel<<<grid1, kThreads, 0, stream>>>(X, y, d, M, sh, batch_rows, B, t, x, coef_ws, rows_ws);
+  logreg_dense_coef_kernel<<<grid1, kThreads, 0, stream>>>(X, y, n_rows, d, M, sh, batch_rows, B, t, x, coef_ws,
+                                                           rows_ws, status);
   const dim3 grid2(static_cast<unsigned>((d + 127) / 128), M);
   logreg_dense_colsum_kernel<<<grid2, kColsumThreads, 0, stream>>>(X, d, B, coef_ws, rows_ws, g, ld_g);
   return 2;
 }
 
 int launch_logreg_csr(const int64_t* rowptr, const int32_t* colidx, const float* vals,
-                      const float* y, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
+                      const float* y, uint64_t n_rows, uint64_t d, uint32_t M, const uint64_t* shard_row0_host,
                       const uint32_t* batch_rows, uint32_t B, uint64_t t, const float* x, float* g,
-                      uint64_t ld_g, const LaunchShape&, cudaStream_t stream, uint32_t* touched) {
+                      uint64_t ld_g, unsigned int* status, const LaunchShape&, cudaStream_t stream,
+                      uint32_t* touched) {
   const Shards sh = make_shards(shard_row0_host, M);
   const dim3 grid((B + kThreads / 32 - 1) / (kThreads / 32), M);
   if (touched) {
-    logreg_csr_kernel<true><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, d, sh, batch_rows, B, t, x, g,
-                                                          ld_g, touched, (d + 31) >> 5);
+    logreg_csr_kernel<true><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, n_rows, d, sh, batch_rows, B, t, x,
+                                                          g, ld_g, touched, (d + 31) >> 5, status);
   } else {
     cudaMemset2DAsync(g, ld_g * sizeof(float), 0, d * sizeof(float), M, stream);
-    logreg_csr_kernel<false><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, d, sh, batch_rows, B, t, x, g,
-                                                           ld_g, nullptr, 0);
+    logreg_csr_kernel<false><<<grid, kThreads, 0, stream>>>(rowptr, colidx, vals, y, n_rows, d, sh, batch_rows, B, t, x,
+                                                           g, ld_g, nullptr, 0, status);
   }
   return 1;
 }

@@ -15,10 +15,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "lib", "libqasg.so")
 
 OK = 0
-ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_BAD_CODE = range(1, 8)
-Q_THRESHOLD, Q_TERNARY_STOCH = 0, 1
+(ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_BAD_CODE,
+ ERR_BAD_INDEX) = range(1, 9)
+Q_THRESHOLD, Q_TERNARY_STOCH, Q_NONE = 0, 1, 2
 RULE_CMD, RULE_RDA = 0, 1
 CREATE_NO_CODE_SCRATCH = 1
+OPT_STREAM_ROW_BYTES, OPT_STREAM_LAG, OPT_WAIT_POLLS = 0, 1, 2
+LAG_AUTO = 0xFFFFFFFF
 
 # Names every build of the library must export (checked by the CPU tests).
 EXPORTS = [
@@ -28,7 +31,7 @@ EXPORTS = [
     "qasg_profile_begin", "qasg_profile_end", "qasg_kernel_name", "qasg_quantize_pack_static", "qasg_requantize", "qasg_step_double",
     "qasg_select_quantize_pack", "qasg_indicator_or", "qasg_step_select",
     "qasg_logreg_grad_csr_touched", "qasg_quantize_pack_touched", "qasg_step_touched",
-    "qasg_optimal_scratch_bytes", "qasg_quantize_pack_optimal",
+    "qasg_optimal_scratch_bytes", "qasg_quantize_pack_optimal", "qasg_set_option", "qasg_wait_selftest",
 ]
 STATIC_MAX_WORKERS = 16
 KERNEL_COUNT = 24
@@ -92,6 +95,8 @@ def load():
     lib.qasg_optimal_scratch_bytes.argtypes = [u64]
     lib.qasg_optimal_scratch_bytes.restype = u64
     lib.qasg_quantize_pack_optimal.argtypes = [vp, vp, u64, u64, u32, pp, vp, vp, vp, vp, vp, u64, vp]
+    lib.qasg_set_option.argtypes = [vp, i32, u64]
+    lib.qasg_wait_selftest.argtypes = [vp, u32, vp]
     lib.qasg_last_async_status.argtypes = [vp, vp]
     lib.qasg_launch_count.argtypes = [vp]
     lib.qasg_launch_count.restype = u64
@@ -251,6 +256,12 @@ class Context:
                                                  _ptr(scales), _ptr(thresholds), _ptr(counts), _ptr(scratch),
                                                  scratch.numel() * scratch.element_size(), _stream(stream)),
                "qasg_quantize_pack_optimal")
+
+    def set_option(self, option, value):
+        _check(load().qasg_set_option(self._h, int(option), int(value)), "qasg_set_option")
+
+    def wait_selftest(self, max_polls, stream=None):
+        _check(load().qasg_wait_selftest(self._h, int(max_polls), _stream(stream)), "qasg_wait_selftest")
 
     def last_async_status(self, stream=None):
         return int(load().qasg_last_async_status(self._h, _stream(stream)))

@@ -65,3 +65,30 @@ def test_reference_arm_prints_one_json_line():
     res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--d", "65536",
                           "--steps", "1", "--warmup", "0"], capture_output=True, text=True, env=env, timeout=300)
     assert res.returncode == 0 and res.stdout.strip() == ""
+
+
+def test_all_cores_harness_gives_the_single_process_oracle_bit_for_bit():
+    """The benchmark's second CPU leg drives the oracle over several processes (workers in parallel for
+    the quantizer, coordinate ranges for the update).  It must be the same oracle: every output equals
+    `qasg_oracle.step` bit for bit."""
+    import numpy as np
+    from oracle import harness
+    from oracle import qasg_oracle as O
+    from paper_2208_05631_b200 import inputs
+    d, M, t = 20_001, 3, 5
+    lam, eta, delta = 1e-3, 0.1, 1e-8
+    g = inputs.optimizer_only_gradients(d, M, t, seed=4) * np.float32(0.05)
+    x0, h0, z0 = (v.numpy().astype(np.float64) for v in inputs.random_state(d, seed=4))
+    with harness.Harness(processes=3) as hs:
+        path_g = hs.put("g", g)
+        paths = [hs.put(n, v) for n, v in (("x", x0), ("h", h0), ("z", z0))]
+        for quantizer in (O.QUANT_THRESHOLD, O.QUANT_TERNARY_STOCH):
+            for rule in (O.RULE_CMD, O.RULE_RDA):
+                state = paths if rule == O.RULE_RDA else [paths[0], paths[1], None]
+                got = hs.step(rule, path_g, M, d, state, t, lam, eta, delta, quantizer=quantizer, seed=9,
+                              range_len=4096)
+                ref = O.step(rule, g, x0, h0, z0, t, lam, eta, delta, quantizer=quantizer, seed=9)
+                for key in ("x", "h", "a", "q") + (("z",) if rule == O.RULE_RDA else ()):
+                    assert np.array_equal(got[key].view(np.uint64), np.asarray(ref[key]).view(np.uint64)), key
+                assert np.array_equal(got["scales"].view(np.uint32), ref["quant"]["scales"].view(np.uint32))
+                assert np.array_equal(got["counts"], ref["quant"]["counts"])

@@ -101,7 +101,6 @@ def test_more_than_2_to_31_coordinates():
     ctx.quantize_pack(g, d, ld, 1, 1, libqasg.make_params(), codes, scales, thr, cnt)
     assert ctx.last_async_status() == libqasg.OK
     row = g[0, :d].cpu().numpy()
-    del g
     tern, s, delta, n = O.threshold_quantize(row)
     del row
     assert thr.cpu().numpy()[0].view(np.uint32) == np.float32(delta).view(np.uint32)
@@ -111,6 +110,44 @@ def test_more_than_2_to_31_coordinates():
     half = (tern.size // 32) * 16          # pack in two pieces to bound the oracle's temporaries
     assert np.array_equal(got[: half // 16], O.pack_codes(tern[:half]))
     assert np.array_equal(got[half // 16:], O.pack_codes(tern[half:]))
+    del got
+    # pass C over the same row: both rules read the oracle's own code words and scale (uploaded, not the
+    # kernel's), and the iterates are compared on sampled coordinates on both sides of 2^31 and at the ends
+    rng = np.random.default_rng(7)
+    idx = np.unique(np.concatenate([rng.integers(0, d, size=1 << 19), np.arange(0, 4100), np.arange(d - 4200, d),
+                                    (1 << 31) + np.arange(-4100, 4099), (1 << 30) + np.arange(-16, 16)]))
+    q = O.decode_average(tern[idx][None, :], np.array([s], dtype=np.float32))
+    codes[0, : half // 16].copy_(torch.from_numpy(O.pack_codes(tern[:half]).view(np.int32)))
+    codes[0, half // 16:].copy_(torch.from_numpy(O.pack_codes(tern[half:]).view(np.int32)))
+    del tern
+    scales.copy_(torch.from_numpy(np.array([s], dtype=np.float32)))
+    idx_t = torch.from_numpy(idx).to(dev)
+    x, h, z = inputs.random_state(d, seed=6, device=dev)
+    x0s, h0s, z0s = (v[idx_t].cpu().numpy() for v in (x, h, z))
+    gbar = torch.empty(d, dtype=torch.float32, device=dev)
+    ctx.decode_average(codes, scales, d, 1, gbar)
+    U.assert_close(gbar[idx_t], q, "decoded average")
+    params = libqasg.make_params(LAM, ETA, DELTA)
+    ctx.cmd_step(gbar, x, h, d, T_STEP, params)
+    x_ref, h_ref, a = O.cmd_step(q, x0s, h0s, LAM, ETA, DELTA)
+    U.assert_close(x[idx_t], x_ref, "x (QCMD, dense q)")
+    U.assert_close(h[idx_t], h_ref, "h (QCMD, dense q)")
+    U.assert_zero_pattern(x[idx_t], x_ref, a, LAM)
+    del gbar
+    # the fused form: quantize again (same codes, checked above) and update in pass C
+    x, h, z = inputs.random_state(d, seed=6, device=dev)
+    ctx.step(libqasg.RULE_CMD, g, d, ld, 1, T_STEP, params, x, h, None, codes_out=codes)
+    U.assert_close(x[idx_t], x_ref, "x (QCMD)")
+    U.assert_close(h[idx_t], h_ref, "h (QCMD)")
+    U.assert_zero_pattern(x[idx_t], x_ref, a, LAM)
+    x, h, z = inputs.random_state(d, seed=6, device=dev)
+    ctx.step(libqasg.RULE_RDA, g, d, ld, 1, T_STEP, params, x, h, z, codes_out=codes)
+    x_ref, h_ref, z_ref, a = O.rda_step(q, h0s, z0s, T_STEP, LAM, ETA, DELTA)
+    U.assert_close(x[idx_t], x_ref, "x (QRDA)")
+    U.assert_close(h[idx_t], h_ref, "h (QRDA)")
+    U.assert_close(z[idx_t], z_ref, "z (QRDA)", atol=U.ATOL + 2.0 ** -23 * (np.abs(z0s) + np.abs(q)))
+    U.assert_zero_pattern(x[idx_t], x_ref, a, LAM)
+    assert ctx.last_async_status() == libqasg.OK
     ctx.close()
 
 
@@ -174,4 +211,98 @@ def test_sparse_form_at_the_size_of_the_sparse_logistic_workload():
     U.assert_close(h[idx_t], h_ref, "h")
     U.assert_close(z[idx_t], z_ref, "z", atol=U.ATOL + 2.0 ** -23 * (np.abs(z0[idx]) + np.abs(q)))
     U.assert_zero_pattern(x[idx_t], x_ref, a, lam)
+    ctx.close()
+
+
+def test_stochastic_quantizer_at_2_to_26_coordinates(tmp_path):
+    """The unbiased ternary quantizer at d = 2^26, M = 8 (the largest size its timings are quoted at): every
+    worker's scale, count and complete code row against the oracle, whose Philox draws and comparisons
+    run one worker per host process, in slices; then the fused QCMD step on sampled coordinates."""
+    from tests import _oracle_pool as P
+    if not _enough_memory():
+        pytest.skip("needs 40 GB of device memory and 24 GB of host memory")
+    dev = U.dev()
+    d, m_workers, t, seed = 1 << 26, 8, T_STEP, (0xC0FFEE << 20) | 77
+    g = inputs.student_t_gradients(d, m_workers, seed=9, device=dev)
+    jobs = []
+    for m in range(m_workers):
+        path = str(tmp_path / ("row%d.npy" % m))
+        np.save(path, g[m].cpu().numpy())
+        jobs.append((path, m, t, seed, 1 << 22))
+    ctx = libqasg.Context(d, m_workers, device=0)
+    params = libqasg.make_params(LAM, ETA, DELTA, quantizer=libqasg.Q_TERNARY_STOCH, seed=seed)
+    codes = torch.zeros((m_workers, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+    scales = torch.zeros(m_workers, dtype=torch.float32, device=dev)
+    counts = torch.zeros(m_workers, dtype=torch.int64, device=dev)
+    x0, h0, _ = inputs.random_state(d, seed=9, device=dev)
+    x, h = x0.clone(), h0.clone()
+    ctx.quantize_pack(g, d, d, m_workers, t, params, codes, scales, None, counts)
+    codes2 = torch.zeros_like(codes)
+    ctx.step(libqasg.RULE_CMD, g, d, d, m_workers, t, params, x, h, None, codes_out=codes2)
+    assert ctx.last_async_status() == libqasg.OK
+    assert torch.equal(codes, codes2)
+    del codes2
+    got_codes, got_scales, got_counts = U.codes_np(codes), scales.cpu().numpy(), counts.cpu().numpy()
+    rng = np.random.default_rng(10)
+    idx = np.unique(np.concatenate([rng.integers(0, d, size=1 << 19), np.arange(0, 4100), np.arange(d - 4100, d)]))
+    terns = np.zeros((m_workers, idx.size), dtype=np.int8)
+    ref_scales = np.zeros(m_workers, dtype=np.float32)
+    for m, words, scale, count in P.run(P.stochastic_row, jobs):
+        assert np.array_equal(got_codes[m], words), "codes of worker %d" % m
+        assert np.float32(scale).view(np.uint32) == got_scales[m].view(np.uint32), "scale of worker %d" % m
+        assert count == int(got_counts[m]) and 0 < count < d
+        terns[m] = O.unpack_codes(words, d)[idx]
+        ref_scales[m] = scale
+    q = O.decode_average(terns, ref_scales)
+    idx_t = torch.from_numpy(idx).to(dev)
+    x_ref, h_ref, a = O.cmd_step(q, x0[idx_t].cpu().numpy(), h0[idx_t].cpu().numpy(), LAM, ETA, DELTA)
+    U.assert_close(x[idx_t], x_ref, "x (QCMD)")
+    U.assert_close(h[idx_t], h_ref, "h (QCMD)")
+    U.assert_zero_pattern(x[idx_t], x_ref, a, LAM)
+    ctx.close()
+
+
+def test_thirty_two_workers_at_2_to_26_coordinates():
+    """d = 2^26, M = 32 (the eight-coordinate decode of pass C at the size it is timed at): every worker's
+    threshold, scale and complete code row, then both rules' iterates on sampled coordinates."""
+    if not _enough_memory():
+        pytest.skip("needs 40 GB of device memory and 24 GB of host memory")
+    dev = U.dev()
+    d, m_workers = 1 << 26, 32
+    g = inputs.normal_gradients(d, m_workers, seed=4, device=dev)
+    x0, h0, z0 = inputs.random_state(d, seed=4, device=dev)
+    ctx = libqasg.Context(d, m_workers, device=0)
+    params = libqasg.make_params(LAM, ETA, DELTA)
+    codes = torch.zeros((m_workers, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+    scales = torch.zeros(m_workers, dtype=torch.float32, device=dev)
+    xc, hc = x0.clone(), h0.clone()
+    ctx.step(libqasg.RULE_CMD, g, d, d, m_workers, T_STEP, params, xc, hc, None, codes_out=codes, scales_out=scales)
+    xr, hr, zr = x0.clone(), h0.clone(), z0.clone()
+    ctx.step(libqasg.RULE_RDA, g, d, d, m_workers, T_STEP, params, xr, hr, zr)
+    assert ctx.last_async_status() == libqasg.OK
+    rng = np.random.default_rng(11)
+    # both ends, and both sides of the places where one CTA's share of the coordinates ends and the next begins
+    seams = ((8 * 512 * 296 * np.arange(1, 8))[:, None] + np.arange(-9, 9)[None, :]).ravel()
+    idx = np.unique(np.concatenate([rng.integers(0, d, size=1 << 19), np.arange(0, 4100), np.arange(d - 4100, d), seams]))
+    terns = np.zeros((m_workers, idx.size), dtype=np.int8)
+    ref_scales = np.zeros(m_workers, dtype=np.float32)
+    gpu_scales = scales.cpu().numpy()
+    for m in range(m_workers):
+        tern, s, delta, n = O.threshold_quantize(g[m].cpu().numpy())
+        assert n > 0 and delta > 0
+        assert np.array_equal(U.codes_np(codes[m]), O.pack_codes(tern)), "codes of worker %d" % m
+        assert np.float32(s).view(np.uint32) == gpu_scales[m].view(np.uint32), "scale of worker %d" % m
+        terns[m], ref_scales[m] = tern[idx], s
+    q = O.decode_average(terns, ref_scales)
+    idx_t = torch.from_numpy(idx).to(dev)
+    x0s, h0s, z0s = (v[idx_t].cpu().numpy() for v in (x0, h0, z0))
+    x_ref, h_ref, a = O.cmd_step(q, x0s, h0s, LAM, ETA, DELTA)
+    U.assert_close(xc[idx_t], x_ref, "x (QCMD)")
+    U.assert_close(hc[idx_t], h_ref, "h (QCMD)")
+    U.assert_zero_pattern(xc[idx_t], x_ref, a, LAM)
+    x_ref, h_ref, z_ref, a = O.rda_step(q, h0s, z0s, T_STEP, LAM, ETA, DELTA)
+    U.assert_close(xr[idx_t], x_ref, "x (QRDA)")
+    U.assert_close(hr[idx_t], h_ref, "h (QRDA)")
+    U.assert_close(zr[idx_t], z_ref, "z (QRDA)", atol=U.ATOL + 2.0 ** -23 * (np.abs(z0s) + np.abs(q)))
+    U.assert_zero_pattern(xr[idx_t], x_ref, a, LAM)
     ctx.close()

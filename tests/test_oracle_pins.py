@@ -233,6 +233,15 @@ def test_stochastic_quantizer_edges():
     u = np.array([0.999, 0.0, 0.5], dtype=np.float32)        # p = 1, 1, 0.5 ; u < p strict
     tern, s = O.ternary_stochastic_quantize(g, u)
     assert s == 2 and tern.tolist() == [1, -1, 0]
+    # a slice quantized with the whole vector's scaler gives that slice of the whole vector's codes
+    rng = np.random.default_rng(8)
+    v, uu = rng.standard_normal(1000).astype(np.float32), rng.random(1000).astype(np.float32)
+    whole, s = O.ternary_stochastic_quantize(v, uu)
+    assert s == np.abs(v).max()
+    parts = [O.ternary_stochastic_quantize(v[lo:lo + 300], uu[lo:lo + 300], scale=s)[0] for lo in range(0, 1000, 300)]
+    assert np.array_equal(np.concatenate(parts), whole)
+    assert not np.array_equal(np.concatenate([O.ternary_stochastic_quantize(v[lo:lo + 300], uu[lo:lo + 300])[0]
+                                              for lo in range(0, 1000, 300)]), whole)
 
 
 # ------------------------------------------------------------------ averaging
