@@ -91,21 +91,25 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
 /* Frees the workspace.  The caller must have synchronized the streams it used. */
 qasg_status qasg_destroy(qasg_ctx* ctx);
 
-/* Options of a context (qasg_set_option).  Defaults suit a B200 (126 MB of L2).
+/* Options of a context (qasg_set_option).
  *
  * qasg_quantize_pack and qasg_step read every gradient row twice: once for the threshold of
- * Section 3.5 (a sum over the whole row), once to cut the codes.  Rows of at most
- * QASG_OPT_STREAM_ROW_BYTES bytes (4*d) are quantized by ONE cooperative launch that codes a row
- * while it is still in the L2 cache, QASG_OPT_STREAM_LAG rows after it was summed, so that the
- * gradients cross device memory once; its CTAs wait for one another through words in the
+ * Section 3.5 (a sum over the whole row), once to cut the codes; by default in two launches (all
+ * sums, then all codes).
+ *
+ * QASG_OPT_STREAM_ROW_BYTES > 0 selects, for rows of at most that many bytes (4*d), ONE cooperative
+ * launch that codes a row QASG_OPT_STREAM_LAG rows after it was summed, while the row is still in L2:
+ * the gradients then cross device memory once.  Its CTAs wait for one another through words in the
  * context's workspace, every wait bounded by QASG_OPT_WAIT_POLLS polls (about 0.2 us each), after
  * which the call gives up and qasg_last_async_status reports QASG_ERR_TIMEOUT (the outputs of that
- * call are then incomplete).  Longer rows go through two launches (all sums, then all codes).  Both
- * ways give the same bits. */
+ * call are then incomplete, and further calls do nothing until the status has been read).  It is off
+ * by default: on a B200 it moves half the bytes but measured slower than the two launches.
+ *
+ * Every setting gives the same bits. */
 typedef enum {
-  QASG_OPT_STREAM_ROW_BYTES = 0, /* 0 = always two launches; default 64 MiB                    */
+  QASG_OPT_STREAM_ROW_BYTES = 0, /* 0 = never (default)                                          */
   QASG_OPT_STREAM_LAG = 1,       /* 0, 1, 2, ...; 0xFFFFFFFF = chosen from the row size (default) */
-  QASG_OPT_WAIT_POLLS = 2        /* 1 .. 2^31; default 2^22 (about a second)                   */
+  QASG_OPT_WAIT_POLLS = 2        /* 1 .. 2^31; default 2^22 (about a second)                      */
 } qasg_option;
 qasg_status qasg_set_option(qasg_ctx* ctx, qasg_option option, uint64_t value);
 

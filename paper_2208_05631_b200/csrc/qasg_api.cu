@@ -22,7 +22,8 @@ struct qasg_ctx {
   unsigned long long* ksyn; // [1] number of bits of the synchronous indicator
   float* logreg_ws;         // kLogregEntries coefficients followed by as many row ids
   StreamSync* sync;         // words the CTAs of the one-launch quantizer wait on
-  uint64_t stream_row_bytes;  // rows up to this size are quantized by the one-launch kernel
+  StreamSlots slots;        // and the slots their chunk partials travel through
+  uint64_t stream_row_bytes;  // rows up to this size are quantized by the one-launch kernel (0: never)
   uint32_t stream_lag;      // kAutoLag: chosen from the row size
   uint32_t wait_polls;
   uint64_t launches;
@@ -69,7 +70,7 @@ struct Launch {
 
 constexpr uint64_t kMaxD = 1ull << 34;
 constexpr uint32_t kAutoLag = 0xFFFFFFFFu;
-constexpr uint64_t kDefaultStreamRowBytes = 64ull << 20;
+constexpr uint64_t kDefaultStreamRowBytes = 0;         // the one-launch kernel is opt-in
 // A row is coded `lag` rows after it was summed; in between the rows summed and coded meanwhile pass
 // through L2.  One row of lag hides the wait for a worker's threshold; it is taken while three rows fit.
 constexpr uint64_t kLagOneRowBytes = 24ull << 20;
@@ -145,7 +146,10 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
     if (stochastic && thresholds) cudaMemsetAsync(thresholds, 0, M * sizeof(float), stream);
     return;
   }
-  if (d * sizeof(float) <= ctx->stream_row_bytes) {  // one launch, each row coded out of L2
+  // One launch, each row coded out of L2: items of a worker's row are dealt to the resident CTAs one row
+  // after the other, so a row is cut into about as many chunks as there are CTAs.
+  const Geometry sgeo = make_geometry(d, ld_g, M, static_cast<uint32_t>(ctx->shape.sm_count * ctx->shape.reduce_ctas_per_sm));
+  if (d * sizeof(float) <= ctx->stream_row_bytes && sgeo.group <= kStreamMaxGroup) {
     const bool stochastic = p->quantizer != QASG_Q_THRESHOLD;
     StreamParams sp;
     sp.coef = p->thr_coef;
@@ -157,7 +161,7 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
     sp.t = t;
     const bool keep_codes = static_cast<uint64_t>(M) * qasg_code_words(d) * 4 <= kKeepCodesBytes;
     Launch l(ctx, stochastic ? kStreamStochastic : kStreamThreshold, stream);
-    l += launch_quantize_stream(stochastic, keep_codes, g, geo, sp, ctx->ws, ctx->sync, codes, scales, thresholds,
+    l += launch_quantize_stream(stochastic, keep_codes, g, sgeo, sp, ctx->ws, ctx->slots, ctx->sync, codes, scales, thresholds,
                                 counts_out, ctx->shape, stream);
     return;
   }
@@ -299,6 +303,9 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ok &= cudaMalloc(&ctx->ws.status, 64) == cudaSuccess;
   ok &= cudaMalloc(&ctx->logreg_ws, kLogregEntries * 2 * sizeof(float)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->sync, sizeof(StreamSync)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->slots.sum_a, 3 * slots * sizeof(unsigned long long)) == cudaSuccess;
+  ctx->slots.sum_b = ctx->slots.sum_a ? ctx->slots.sum_a + slots : nullptr;
+  ctx->slots.cnt_b = ctx->slots.sum_a ? ctx->slots.sum_a + 2 * slots : nullptr;
   ok &= cudaMalloc(&ctx->wsq.part_sum, kRowChunks * sizeof(double)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.part_max, kRowChunks * sizeof(uint32_t)) == cudaSuccess;
   ok &= cudaMalloc(&ctx->wsq.part_cnt, kRowChunks * sizeof(unsigned long long)) == cudaSuccess;
@@ -318,6 +325,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
     ok &= cudaMemset(ctx->ws.ticket, 0, 64) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.status, 0, 64) == cudaSuccess;
     ok &= cudaMemset(ctx->sync, 0, sizeof(StreamSync)) == cudaSuccess;
+    ok &= cudaMemset(ctx->slots.sum_a, 0xFF, 3 * slots * sizeof(unsigned long long)) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.thresholds, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
     ok &= cudaMemset(ctx->ws.scales, 0, kMaxWorkers * sizeof(float)) == cudaSuccess;
     ok &= cudaMemset(ctx->wsq.thresholds, 0, 64) == cudaSuccess;
@@ -345,6 +353,7 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->ws.status);
   cudaFree(ctx->logreg_ws);
   cudaFree(ctx->sync);
+  cudaFree(ctx->slots.sum_a);
   cudaFree(ctx->code_scratch);
   cudaFree(ctx->qcode_scratch);
   cudaFree(ctx->gbar_scratch);
@@ -761,6 +770,7 @@ qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream) {
   }
   if (flags & kFlagTimeout) {  // a call gave up half-way: its tickets and abort word are left set
     cudaMemsetAsync(ctx->sync, 0, sizeof(StreamSync), s);
+    cudaMemsetAsync(ctx->slots.sum_a, 0xFF, 3 * static_cast<size_t>(ctx->M_max) * kMaxChunks * sizeof(unsigned long long), s);
     cudaStreamSynchronize(s);
     return QASG_ERR_TIMEOUT;
   }

@@ -49,15 +49,21 @@ struct Workspace {
   unsigned int* status;          // OR of kFlag*
 };
 
-// Words the CTAs of the one-launch quantizer (qasg_stream.cu) synchronise through.  All of them are back
-// at zero when a call completes (the CTA that ends a worker's last item resets that worker's words), so a
-// captured launch can be replayed; a call that gave up leaves them set and the host clears them.
+// What the CTAs of the one-launch quantizer (qasg_stream.cu) hand to one another.  Chunk partials travel
+// through 64-bit slots that hold kEmptySlot until their item has stored its value; the consumer empties
+// them again, so everything is back in its initial state when a call completes and a captured launch can
+// be replayed.  A call that gave up leaves them in an unknown state: `abort` stays set and the host clears
+// slots and words.  These arrays belong to that kernel alone.
+constexpr unsigned long long kEmptySlot = 0xFFFFFFFFFFFFFFFFull;  // not the bits of any sum, count or maximum
+struct StreamSlots {
+  unsigned long long* sum_a;  // [M_max][kMaxChunks] chunk sums of |g| (double bits), or chunk maxima (stochastic)
+  unsigned long long* sum_b;  // [M_max][kMaxChunks] chunk sums of the kept |g| (double bits)
+  unsigned long long* cnt_b;  // [M_max][kMaxChunks] chunk counts of non-zero codes
+};
 struct StreamSync {
-  unsigned int ticket_a[kMaxWorkers];  // sum items of worker m completed in this call
-  unsigned int ticket_b[kMaxWorkers];  // code items of worker m completed in this call
-  unsigned int ready[kMaxWorkers];     // 1 once worker m's threshold (or scaler) of this call is published
-  unsigned int abort;                  // non-zero once a wait ran out: every later wait returns at once
-  unsigned int probe, probe_abort;     // the wait self-test's own words (nothing ever sets probe)
+  unsigned int ready[kMaxWorkers];  // 1 once worker m's threshold (or scaler) of this call is published
+  unsigned int abort;               // non-zero once a wait ran out: every later wait returns at once
+  unsigned int probe, probe_abort;  // the wait self-test's own words (nothing ever sets probe)
 };
 
 struct StreamParams {
@@ -165,9 +171,11 @@ int launch_optimal_threshold(const float* row, uint64_t d, void* scratch, float*
 
 // Passes A and B in one cooperative launch (rows that fit L2); results as launch_abs_sum/abs_max followed
 // by launch_threshold_codes/stochastic_codes.  keep_codes: ordinary instead of streaming code stores.
+// geo.group must not exceed kStreamMaxGroup (an item's tiles are combined in one go).
+constexpr uint32_t kStreamMaxGroup = 32;
 int launch_quantize_stream(bool stochastic, bool keep_codes, const float* g, const Geometry& geo,
-                           const StreamParams& sp, const Workspace& ws, StreamSync* sync, uint32_t* codes,
-                           float* scales_out, float* thresholds_out, unsigned long long* counts_out,
+                           const StreamParams& sp, const Workspace& ws, const StreamSlots& slots, StreamSync* sync,
+                           uint32_t* codes, float* scales_out, float* thresholds_out, unsigned long long* counts_out,
                            const LaunchShape& shape, cudaStream_t stream);
 // One bounded wait on a word nothing sets: raises kFlagTimeout after max_polls polls.
 int launch_wait_selftest(StreamSync* sync, unsigned int* status, uint32_t max_polls, cudaStream_t stream);

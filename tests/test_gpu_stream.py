@@ -1,5 +1,5 @@
-"""The one-launch quantizer (a row coded out of L2 right after it was summed) against the oracle and
-against the two-launch path, over row counts, lags and chunk shapes; and its bounded waits."""
+"""The one-launch quantizer (an option: a row coded out of L2 right after it was summed) against the oracle
+and against the default two-launch path, over row counts, lags and chunk shapes; and its bounded waits."""
 import numpy as np
 import pytest
 import torch
@@ -17,8 +17,6 @@ LAM, ETA, DELTA = 1e-3, 0.1, 1e-8
 def ctx():
     c = libqasg.Context(1 << 23, 64, device=0)
     yield c
-    c.set_option(libqasg.OPT_STREAM_ROW_BYTES, 64 << 20)
-    c.set_option(libqasg.OPT_STREAM_LAG, libqasg.LAG_AUTO)
     c.close()
 
 
@@ -65,10 +63,12 @@ def test_one_launch_equals_two_launches_and_the_oracle(ctx, d, M, quantizer):
         assert launches == 1
         _same(one, ref)
     ctx.set_option(libqasg.OPT_STREAM_LAG, libqasg.LAG_AUTO)
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 0)
 
 
 def test_repeated_calls_reuse_the_synchronisation_words(ctx):
-    # tickets return to zero and the ready words carry the call's epoch: nothing is reset between calls
+    # every slot and word is back in its initial state when a call completes: nothing is reset between calls
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 64 << 20)
     d, M = 200_003, 8
     for rep in range(20):
         g = inputs.optimizer_only_gradients(d, M, rep + 1, seed=3)
@@ -76,9 +76,11 @@ def test_repeated_calls_reuse_the_synchronisation_words(ctx):
         got, launches = _quantize(ctx, g_dev, ld, M, d, libqasg.Q_THRESHOLD, rep + 1, 0)
         assert launches == 1
         _same(got, O.quantize_workers(g, O.QUANT_THRESHOLD))
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 0)
 
 
 def test_nonfinite_gradient_in_one_launch(ctx):
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 64 << 20)
     g = np.ones((3, 50_000), dtype=np.float32)
     g[1, 4321] = np.nan
     g_dev, ld = U.grad_to_dev(g)
@@ -87,6 +89,7 @@ def test_nonfinite_gradient_in_one_launch(ctx):
     assert ctx.last_async_status() == libqasg.ERR_NONFINITE
     ref = O.quantize_workers(g, O.QUANT_THRESHOLD)
     assert np.array_equal(U.codes_np(codes), ref["codes"]) and not U.codes_np(codes)[1].any()
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 0)
 
 
 @pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
@@ -110,6 +113,7 @@ def test_fused_step_through_both_quantizer_paths(ctx, rule):
     ref = O.step(rule, g, x0, h0, z0, t, LAM, ETA, DELTA)
     U.assert_close(out[1][0], ref["x"], "x"), U.assert_close(out[1][1], ref["h"], "h")
     U.assert_zero_pattern(out[1][0], ref["x"], ref["a"], LAM)
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 0)
 
 
 def test_a_wait_that_nothing_ends_gives_up(ctx):
@@ -122,8 +126,11 @@ def test_a_wait_that_nothing_ends_gives_up(ctx):
     d, M = 70_001, 4
     g = inputs.optimizer_only_gradients(d, M, 1, seed=1)
     g_dev, ld = U.grad_to_dev(g)
-    got, _ = _quantize(ctx, g_dev, ld, M, d, libqasg.Q_THRESHOLD, 1, 0)
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 64 << 20)
+    got, launches = _quantize(ctx, g_dev, ld, M, d, libqasg.Q_THRESHOLD, 1, 0)
+    assert launches == 1
     _same(got, O.quantize_workers(g, O.QUANT_THRESHOLD))
+    ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, 0)
     ctx.wait_selftest(1)
     assert ctx.last_async_status() == libqasg.ERR_TIMEOUT
 
