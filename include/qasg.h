@@ -80,6 +80,11 @@ typedef struct {
 
 /* Flags of qasg_create. */
 #define QASG_CREATE_NO_CODE_SCRATCH 1u /* qasg_step will always be given codes_out   */
+/* By default the kernels of a step are launched as programmatic dependents of one another: a
+ * kernel's CTAs are placed, and in pass B request their first gradient tile, while the kernel
+ * before it drains; each waits for that kernel's completion before it touches what it wrote.
+ * With this flag every kernel starts only after the one before it has completed.  Same bits. */
+#define QASG_CREATE_SERIAL_LAUNCHES 2u
 
 /* Creates a context on CUDA device `device` able to serve calls with d <= d_max and
  * M <= M_max.  Allocates the whole workspace here (a few hundred KB of statistics, and,

@@ -289,6 +289,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ctx->stream_lag = kAutoLag;
   ctx->wait_polls = 1u << 22;
   query_launch_shape(&ctx->shape);
+  ctx->shape.chained = !(flags & QASG_CREATE_SERIAL_LAUNCHES);
   const size_t slots = static_cast<size_t>(M_max) * kMaxChunks;
   bool ok = true;
   ok &= cudaMalloc(&ctx->ws.part_sum, slots * sizeof(double)) == cudaSuccess;

@@ -5,6 +5,35 @@
 
 namespace qasg {
 
+// ------------------------------------------------------------------ chained launches
+// Programmatic dependent launch: a kernel launched with the attribute below may start while its predecessor
+// in the stream is still running (once every CTA of the predecessor has passed chain_trigger or exited).  The
+// rules every chained kernel here keeps:
+//   - chain_wait() comes before the first access to anything a predecessor may have written; it returns once
+//     the predecessor grid has completed and its writes are visible;
+//   - chain_trigger() comes after chain_wait(), so when a dependent starts, everything older than its
+//     immediate predecessor is complete: a dependent may therefore read, ahead of its own chain_wait(),
+//     only data that its immediate predecessor does not write (the gradients, in pass B).
+// Both are no-ops in a kernel launched without the attribute.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                  cudaStream_t stream, bool chained, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = chained ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ float4 load_f4(const float* p) {
   return __ldg(reinterpret_cast<const float4*>(p));
@@ -227,11 +256,19 @@ __device__ __forceinline__ ItemPos item_pos(const Geometry& geo, uint32_t item) 
   return p;
 }
 
-template <bool kMasked, class Begin, class Body, class End>
+// kEarlyLoad: the first tile's loads go out before chain_wait() (the gradients are not written by the launch
+// this one is chained to); otherwise the caller has waited already.
+template <bool kMasked, bool kEarlyLoad = false, class Begin, class Body, class End>
 __device__ __forceinline__ void stream_items(const float* __restrict__ g, const uint32_t* __restrict__ indicators,
                                              const Geometry& geo, int j, Begin&& begin, Body&& body, End&& end) {
   const uint32_t n_items = geo.M * geo.chunks;
-  if (blockIdx.x >= n_items) return;
+  if (blockIdx.x >= n_items) {
+    if (kEarlyLoad) {
+      chain_wait();
+      chain_trigger();
+    }
+    return;
+  }
   const uint64_t ind_words = (geo.d + 31) >> 5;
   ItemPos cur = item_pos(geo, blockIdx.x);
   uint32_t k = cur.k0;
@@ -244,6 +281,10 @@ __device__ __forceinline__ void stream_items(const float* __restrict__ g, const 
       load_tile_mask(indicators + static_cast<uint64_t>(p.m) * ind_words, geo.d, kk, j, mk);
   };
   load(cur, k, a, ma);
+  if (kEarlyLoad) {
+    chain_wait();
+    chain_trigger();
+  }
   begin(cur.m, cur.c);
   auto step = [&](float4 (&cv)[kTileRows], TileMask& cm, float4 (&nv)[kTileRows], TileMask& nm) -> bool {
     ItemPos nxt = cur;

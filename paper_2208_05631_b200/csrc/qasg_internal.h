@@ -78,6 +78,7 @@ struct LaunchShape {
   int sm_count;
   int reduce_ctas_per_sm;  // resident CTAs per SM for the reduction kernels
   int update_ctas_per_sm;  // same for the coordinate-wise kernels
+  bool chained;            // launch the step's kernels as programmatic dependents of their predecessors
 };
 
 // Constants of the indicator test, rounded to fp32 on the host: lambda*eta, lambda*t.

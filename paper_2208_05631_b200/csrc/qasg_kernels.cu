@@ -52,6 +52,8 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
   __shared__ ChunkSumStorage sm_sum;
   __shared__ bool sm_last;
   const int j = threadIdx.x;
+  chain_wait();  // the gradients may come from the launch before this one
+  chain_trigger();
   ChunkSum chunk_sum(&sm_sum);
   auto begin = [](uint32_t, uint32_t) {};
   auto body = [&](const float4 (&v)[kTileRows], const TileMask&, uint32_t) {
@@ -92,6 +94,8 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
   __shared__ uint32_t sm_warp[kThreads / 32];
   __shared__ bool sm_last;
   const int j = threadIdx.x;
+  chain_wait();
+  chain_trigger();
   const uint32_t n_items = geo.M * geo.chunks;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
@@ -149,6 +153,10 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
   const int j = threadIdx.x;
   const uint64_t row_words = (geo.d + 15) >> 4;
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
+  if (kMasked) {  // the indicator words come from the launch before this one
+    chain_wait();
+    chain_trigger();
+  }
   ChunkSum chunk_sum(&sm_sum);
   uint8_t* codes8 = nullptr;  // per item: the worker's code row, its threshold, the kept count so far
   float delta = 0.f, ndelta = 0.f, cntf = 0.f;
@@ -196,7 +204,8 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
           ws.part_cnt[p] = total;
         }
       };
-  stream_items<kMasked>(g, indicators, geo, j, begin, body, end);
+  // unmasked: the first gradient tile is requested ahead of the wait for the thresholds
+  stream_items<kMasked, !kMasked>(g, indicators, geo, j, begin, body, end);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   finish_codes<true>(geo, ws, scales_out, counts_out);
   if (j == 0) *ws.ticket = 0u;
@@ -216,6 +225,8 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
   const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
   const uint32_t t_lo = static_cast<uint32_t>(t), t_hi = static_cast<uint32_t>(t >> 32);
+  chain_wait();
+  chain_trigger();
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
@@ -410,6 +421,8 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
                      uint32_t M, double inv_m, float* __restrict__ x, float* __restrict__ h,
                      float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
   extern __shared__ double sm_lut[];
+  chain_wait();  // scales and codes come from the launch before this one
+  chain_trigger();
   build_decode_lut<kLanes>(sm_lut, scales, M);
   const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
   const uint64_t row_bytes = ((d + 15) >> 4) * 4;
@@ -573,6 +586,8 @@ decode_update_wide_kernel(const uint32_t* __restrict__ codes, const float* __res
                           uint32_t M, double inv_m, float* __restrict__ x, float* __restrict__ h,
                           float* __restrict__ z, StepScalars sc, unsigned int* __restrict__ status) {
   extern __shared__ double sm_lut[];
+  chain_wait();  // scales and codes come from the launch before this one
+  chain_trigger();
   build_decode_lut3(sm_lut, scales, M);
   const uint32_t lut_lane =
       static_cast<uint32_t>(__cvta_generic_to_shared(sm_lut + (threadIdx.x & (kLut3Lanes - 1))));
@@ -1262,6 +1277,7 @@ void query_launch_shape(LaunchShape* shape) {
   int a = 0, b = 0;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, threshold_codes_kernel<false>, kThreads, 0);
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dense_update_kernel<1>, kThreads, 0);
+  shape->chained = false;
   shape->reduce_ctas_per_sm = a > 0 ? a : 1;
   shape->update_ctas_per_sm = b > 0 ? b : 1;
 }
@@ -1282,13 +1298,14 @@ static unsigned update_grid(uint64_t d, const LaunchShape& shape) {
 int launch_abs_sum(const float* g, const Geometry& geo, float coef, const Workspace& ws,
                    float* thresholds_out, const LaunchShape& shape, cudaStream_t stream,
                    const unsigned long long* denom) {
-  abs_sum_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, coef, ws, thresholds_out, denom);
+  launch_chained(abs_sum_kernel, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo, coef, ws,
+                 thresholds_out, denom);
   return 1;
 }
 
 int launch_abs_max(const float* g, const Geometry& geo, const Workspace& ws,
                    const LaunchShape& shape, cudaStream_t stream) {
-  abs_max_kernel<<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws);
+  launch_chained(abs_max_kernel, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo, ws);
   return 1;
 }
 
@@ -1296,11 +1313,11 @@ int launch_threshold_codes(const float* g, const Geometry& geo, const Workspace&
                            uint32_t* codes, float* scales_out, unsigned long long* counts_out,
                            const LaunchShape& shape, cudaStream_t stream, const uint32_t* indicators) {
   if (indicators)
-    threshold_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                                  counts_out, indicators);
+    launch_chained(threshold_codes_kernel<true>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo, ws,
+                   codes, scales_out, counts_out, indicators);
   else
-    threshold_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(g, geo, ws, codes, scales_out,
-                                                                                   counts_out, nullptr);
+    launch_chained(threshold_codes_kernel<false>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo, ws,
+                   codes, scales_out, counts_out, static_cast<const uint32_t*>(nullptr));
   return 1;
 }
 
@@ -1309,11 +1326,11 @@ int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, 
                             unsigned long long* counts_out, const LaunchShape& shape,
                             cudaStream_t stream, const uint32_t* indicators) {
   if (indicators)
-    stochastic_codes_kernel<true><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
-        g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, indicators);
+    launch_chained(stochastic_codes_kernel<true>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo, seed,
+                   t, stream_base, ws, codes, scales_out, counts_out, indicators);
   else
-    stochastic_codes_kernel<false><<<reduce_grid(geo, shape), kThreads, 0, stream>>>(
-        g, geo, seed, t, stream_base, ws, codes, scales_out, counts_out, nullptr);
+    launch_chained(stochastic_codes_kernel<false>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo,
+                   seed, t, stream_base, ws, codes, scales_out, counts_out, static_cast<const uint32_t*>(nullptr));
   return 1;
 }
 
@@ -1371,8 +1388,8 @@ static void launch_decode_update_as(const uint32_t* codes, const float* scales, 
   const uint64_t max_grid = static_cast<uint64_t>(shape.sm_count) * resident;
   if (grid > max_grid) grid = max_grid;
   const double inv_m = 1.0 / static_cast<double>(M);
-  kernel<<<static_cast<unsigned>(grid), kThreadsC, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc,
-                                                                        status);
+  launch_chained(kernel, static_cast<unsigned>(grid), kThreadsC, lut_bytes, stream, shape.chained, codes, scales, d, M,
+                 inv_m, x, h, z, sc, status);
 }
 
 template <int kRule, int kM4>
@@ -1395,8 +1412,8 @@ static void launch_decode_update_wide_as(const uint32_t* codes, const float* sca
   const uint64_t max_grid = static_cast<uint64_t>(shape.sm_count) * resident;
   if (grid > max_grid) grid = max_grid;
   const double inv_m = 1.0 / static_cast<double>(M);
-  kernel<<<static_cast<unsigned>(grid), kWideThreads, lut_bytes, stream>>>(codes, scales, d, M, inv_m, x, h, z, sc,
-                                                                           status);
+  launch_chained(kernel, static_cast<unsigned>(grid), kWideThreads, lut_bytes, stream, shape.chained, codes, scales, d, M,
+                 inv_m, x, h, z, sc, status);
 }
 
 template <int kRule>

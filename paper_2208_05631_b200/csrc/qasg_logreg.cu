@@ -6,7 +6,7 @@
 // CSR: one warp per minibatch row computes the margin and scatters with atomic adds.  The sparse form
 // keeps the dense rows of g zero between calls and a bit per entry that a minibatch touched, so a call
 // moves the touched sectors only (no clearing or re-reading of M*d floats).
-#include "qasg_internal.h"
+#include "qasg_device.cuh"
 
 namespace qasg {
 
@@ -41,6 +41,8 @@ logreg_dense_coef_kernel(const float* __restrict__ X, const float* __restrict__ 
                          const float* __restrict__ x, float* __restrict__ coef, uint32_t* __restrict__ rows,
                          unsigned int* __restrict__ status) {
   const uint32_t warp = (blockIdx.x * kThreads + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  chain_wait();  // x comes from the update of the iteration before
+  chain_trigger();
   if (warp >= M * B) return;
   const uint32_t m = warp / B, b = warp - m * B;
   const uint64_t r = batch_row(sh, batch_rows, m, b, B, t);
@@ -78,6 +80,8 @@ logreg_dense_colsum_kernel(const float* __restrict__ X, uint64_t d, uint32_t B, 
                            const uint32_t* __restrict__ rows, float* __restrict__ g, uint64_t ld_g) {
   constexpr int kRowLanes = kColsumThreads / 32;
   __shared__ float4 sm[kRowLanes][32];
+  chain_wait();  // the coefficients come from the launch before this one
+  chain_trigger();
   const uint32_t m = blockIdx.y, cq = threadIdx.x & 31, rl = threadIdx.x >> 5;
   const uint64_t col = (static_cast<uint64_t>(blockIdx.x) * 32 + cq) * 4;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -236,15 +240,24 @@ static Shards make_shards(const uint64_t* shard_row0_host, uint32_t M) {
 int launch_logreg_dense(const float* X, const float* y, uint64_t n_rows, uint64_t d, uint32_t M,
                         const uint64_t* shard_row0_host, const uint32_t* batch_rows, uint32_t B,
                         uint64_t t, const float* x, float* g, uint64_t ld_g, float* coef_ws,
-                        unsigned int* status, const LaunchShape&, cudaStream_t stream) {
+                        unsigned int* status, const LaunchShape& shape, cudaStream_t stream) {
   const Shards sh = make_shards(shard_row0_host, M);
   uint32_t* rows_ws = reinterpret_cast<uint32_t*>(coef_ws + static_cast<uint64_t>(M) * B);
   const uint64_t warps = static_cast<uint64_t>(M) * B;
   const unsigned grid1 = static_cast<unsigned>((warps * 32 + kThreads - 1) / kThreads);
-  logreg_dense_coef_kernel<<<grid1, kThreads, 0, stream>>>(X, y, n_rows, d, M, sh, batch_rows, B, t, x, coef_ws,
-                                                           rows_ws, status);
-  const dim3 grid2(static_cast<unsigned>((d + 127) / 128), M);
-  logreg_dense_colsum_kernel<<<grid2, kColsumThreads, 0, stream>>>(X, d, B, coef_ws, rows_ws, g, ld_g);
+  launch_chained(logreg_dense_coef_kernel, grid1, kThreads, 0, stream, shape.chained, X, y, n_rows, d, M, sh, batch_rows, B,
+                 t, x, coef_ws, rows_ws, status);
+  cudaLaunchConfig_t cfg = {};  // a two-dimensional grid: (column blocks, workers)
+  cfg.gridDim = dim3(static_cast<unsigned>((d + 127) / 128), M);
+  cfg.blockDim = dim3(kColsumThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = shape.chained ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, logreg_dense_colsum_kernel, X, d, B, static_cast<const float*>(coef_ws),
+                     static_cast<const uint32_t*>(rows_ws), g, ld_g);
   return 2;
 }
 

@@ -20,6 +20,7 @@ OK = 0
 Q_THRESHOLD, Q_TERNARY_STOCH, Q_NONE = 0, 1, 2
 RULE_CMD, RULE_RDA = 0, 1
 CREATE_NO_CODE_SCRATCH = 1
+CREATE_SERIAL_LAUNCHES = 2
 OPT_STREAM_ROW_BYTES, OPT_STREAM_LAG, OPT_WAIT_POLLS = 0, 1, 2
 LAG_AUTO = 0xFFFFFFFF
 

@@ -46,3 +46,35 @@ def test_fused_step_replayed_from_a_cuda_graph(rule):
         assert torch.equal(got, want)
     assert ctx.last_async_status() == libqasg.OK
     ctx.close()
+
+
+def test_chained_launches_give_the_bits_of_serial_launches():
+    """By default a step's kernels are launched as programmatic dependents of one another (a kernel is placed,
+    and pass B requests its first tile, while its predecessor drains).  The same iterations on a context
+    created with QASG_CREATE_SERIAL_LAUNCHES must give the same bits: gradient kernel + fused step, both
+    quantizers, state carried over ten iterations."""
+    dev = torch.device("cuda:0")
+    n, d, M, B = 4096, 1024, 8, 64
+    prob = inputs.logreg_dense_problem(n=n, d=d, M=M, seed=1)
+    X, y = torch.from_numpy(prob["X"]).to(dev), torch.from_numpy(prob["y"]).to(dev)
+    results = []
+    for flags in (0, libqasg.CREATE_SERIAL_LAUNCHES):
+        ctx = libqasg.Context(d, M, device=0, flags=flags)
+        out = []
+        for quantizer in (libqasg.Q_THRESHOLD, libqasg.Q_TERNARY_STOCH):
+            params = libqasg.make_params(1e-4, 0.1, 1e-8, quantizer=quantizer, seed=5)
+            for rule in (libqasg.RULE_CMD, libqasg.RULE_RDA):
+                x, h, z = (torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(3))
+                g = torch.empty((M, d), dtype=torch.float32, device=dev)
+                codes = torch.zeros((M, libqasg.code_words(d)), dtype=torch.int32, device=dev)
+                for t in range(1, 11):
+                    ctx.logreg_grad_dense(X, y, n, d, M, prob["shard_row0"], None, B, t, x, g, d)
+                    ctx.step(rule, g, d, d, M, t, params, x, h, z, codes_out=codes)
+                torch.cuda.synchronize()
+                out += [x.clone(), h.clone(), z.clone(), codes.clone()]
+        assert ctx.last_async_status() == libqasg.OK
+        ctx.close()
+        results.append(out)
+    for a, b in zip(*results):
+        assert torch.equal(a, b)
+    assert any(bool(t.any()) for t in results[0])
