@@ -445,7 +445,7 @@ def run_config3(rig, args):
     x0, h0, z0 = inputs.random_state(d, seed=SEED + rig.rank, device=dev)
     xc, hc = x0.clone(), h0.clone()                 # QCMD state
     xr, hr, zr = x0.clone(), h0.clone(), z0.clone()  # QRDA state
-    ctx = libqasg.Context(d, M, device=rig.local)
+    ctx = new_context(libqasg, rig, args, d, M)
     params = libqasg.make_params(LAM, ETA, DELTA, quantizer=quantizer_of(args, libqasg), seed=SEED)
 
     def restore():
@@ -482,7 +482,7 @@ def run_config3(rig, args):
     units = {k: v * d for k, v in bpc.items()}
     per_kernel = kernel_table(kernels, units)
     roofline = roofline_of(per_kernel, units, traffic=lambda k: ncu_traffic(k, d, M))
-    once = 4.0 * d <= ctx_stream_row_bytes()
+    once = 4.0 * d <= args.stream_row_bytes
     moved = (step_bytes(M, "qcmd", once) + step_bytes(M, "qrda", once)) * d
     minimal = (minimal_bytes(M, "qcmd") + minimal_bytes(M, "qrda")) * d
     peak, _ = measured_peak()
@@ -501,8 +501,11 @@ def run_config3(rig, args):
               "bytes_moved_frac_of_peak": moved / 1e9 / sec / peak})
 
 
-def ctx_stream_row_bytes():
-    return 64 << 20          # the library's default for the one-launch quantizer (QASG_OPT_STREAM_ROW_BYTES)
+def new_context(libqasg, rig, args, d, M):
+    ctx = libqasg.Context(d, M, device=rig.local)
+    if args.stream_row_bytes:
+        ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, args.stream_row_bytes)
+    return ctx
 
 
 def e2e_single_step(rig, args, ctx, params, g, x0, h0, z0):
@@ -786,7 +789,7 @@ def run_config5(rig, args):
             g = inputs.normal_gradients(d, M, seed=4, device=dev)
             x0, h0, z0 = inputs.random_state(d, seed=4, device=dev)
             x, h, z = x0.clone(), h0.clone(), z0.clone()
-            ctx = libqasg.Context(d, M, device=rig.local)
+            ctx = new_context(libqasg, rig, args, d, M)
             for rule, name in ((libqasg.RULE_CMD, "qcmd"), (libqasg.RULE_RDA, "qrda")):
                 def before():
                     x.copy_(x0), h.copy_(h0), z.copy_(z0)
@@ -801,7 +804,7 @@ def run_config5(rig, args):
                 one()
                 torch.cuda.synchronize()
                 kernel_ms = {k: v[0] / v[1] for k, v in ctx.profile_end().items()}
-                once = 4.0 * d <= ctx_stream_row_bytes() and args.variant == "step" and args.quantizer != "none"
+                once = 4.0 * d <= args.stream_row_bytes and args.variant == "step" and args.quantizer != "none"
                 moved = step_bytes(M, name, once) * d if args.quantizer != "none" else minimal_bytes(M, name) * d
                 grid.append({"d": d, "M": M, "rule": name, "ms_median": med, "ms_best": min(times),
                              "coord_workers_per_s": d * M / (med * 1e-3),
@@ -821,8 +824,9 @@ def run_config5(rig, args):
     emit(rig, args, value=rig.world * total_units / (total_ms * 1e-3), ms_per_step=total_ms,
          config={"workload": WORKLOAD_5, "quantizer": args.quantizer, "variant": args.variant,
                  "l2": "flushed (a 252 MiB buffer written) and the state restored before every timed step",
-                 "note": "gbs_moved: bytes the step must move through device memory (g twice above d=2^24, once where a "
-                         "row is coded out of L2); gbs_minimal: each gradient once + state once"},
+                 "one_launch_quantizer_row_bytes": args.stream_row_bytes,
+                 "note": "gbs_moved: bytes the step must move through device memory (g twice; once where the one-launch "
+                         "quantizer codes a row out of L2); gbs_minimal: each gradient once + state once"},
          clocks=clocks, gpu_launches=launches, e2e=None, roofline=None, cpu_baseline=None, grid=grid)
 
 
@@ -932,6 +936,8 @@ def main():
     ap.add_argument("--max-log2-d", type=int, default=28)
     ap.add_argument("--workers", default="2,4,8,16,32", help="workload 5 and optimal")
     ap.add_argument("--csr-rows", type=int, default=1_000_000, help="workload 4: rows of the CSR matrix")
+    ap.add_argument("--stream-row-bytes", type=int, default=0,
+                    help="workloads 3 and 5: quantize rows up to this size with the one-launch kernel (library option; 0 = default path)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
