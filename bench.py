@@ -2,7 +2,7 @@
 """Benchmark of the quantized adaptive-subgradient step (libqasg) on synthetic workloads.
 
   python bench.py [--config 1|2|3|4|5|optimal|touched] [--gpus N] [--steps K] [--warmup W]
-                  [--impl ours|reference] [--quantizer threshold|stochastic|none] [--variant step|double|select]
+                  [--impl ours|reference] [--quantizer threshold|stochastic|none] [--variant step|double|select] [--state-density P]
 
 Workloads (--config; default 3, the headline):
   1  optimizer-only QCMD run: d = 10,000, M = 4, g ~ N(0,1)(1+0.1m), 100 iterations from x = h = 0;
@@ -433,6 +433,7 @@ def workload_3(args, note):
                         "step + one fused QRDA step per bench step, each from the stated state (restored, "
                         "untimed, before every step)" % (args.d, args.M, T_STEP, LAM, ETA, DELTA, SEED),
             "d": args.d, "M": args.M, "quantizer": args.quantizer, "variant": args.variant, "rules": ["qcmd", "qrda"],
+            "state_density": args.state_density,
             "l2": "inputs (%.1f GiB of gradients) are larger than L2 and the state restore (%.1f GiB copied) "
                   "passes through it between steps" % (args.d * args.M * 4 / 2 ** 30, 5 * args.d * 4 / 2 ** 30),
             "parallelism": "replicas" if args.gpus > 1 else "single", "note": note}
@@ -443,6 +444,8 @@ def run_config3(rig, args):
     dev, d, M = rig.dev, args.d, args.M
     g = inputs.student_t_gradients(d, M, seed=SEED + rig.rank, device=dev)
     x0, h0, z0 = inputs.random_state(d, seed=SEED + rig.rank, device=dev)
+    if args.state_density < 1.0:   # a sparse iterate: the selection masks are then mixed in every tile
+        x0 *= inputs.bernoulli_mask(d, args.state_density, seed=SEED + rig.rank, device=dev)
     xc, hc = x0.clone(), h0.clone()                 # QCMD state
     xr, hr, zr = x0.clone(), h0.clone(), z0.clone()  # QRDA state
     ctx = new_context(libqasg, rig, args, d, M)
@@ -930,6 +933,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quantizer", default="threshold", choices=["threshold", "stochastic", "none"])
     ap.add_argument("--variant", default="step", choices=["step", "double", "select"])
+    ap.add_argument("--state-density", type=float, default=1.0,
+                    help="config 3: fraction of the iterate x that is non-zero (seeded Bernoulli mask)")
     ap.add_argument("--d", type=int, default=1 << 28, help="workload 3: coordinates")
     ap.add_argument("--M", type=int, default=8, help="workload 3: workers")
     ap.add_argument("--min-log2-d", type=int, default=20, help="workload 5 and optimal")

@@ -223,7 +223,9 @@ qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint
  *   indicators  device, uint32 [M][ceil(d/32)]: bit i&31 of word i>>5 of row m; unused bits 0.
  *   selected    device, uint64 [M] or NULL: k_m.  A worker's message is then 32 + d + 2*k_m bits
  *               (Section 3.5 "Encode").
- *   other arguments as for qasg_quantize_pack. */
+ *   other arguments as for qasg_quantize_pack.
+ * The comparisons are "greater or unordered": a NaN component (QRDA: a NaN z + g) is marked like an
+ * infinite one, enters the sums and is reported as QASG_ERR_NONFINITE; outputs are then unspecified. */
 qasg_status qasg_select_quantize_pack(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
                                       uint64_t ld_g, uint32_t M, uint64_t t, const qasg_params* params,
                                       const float* x, const float* h, const float* z, uint32_t* codes,

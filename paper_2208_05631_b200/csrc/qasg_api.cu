@@ -15,6 +15,7 @@ struct qasg_ctx {
   LaunchShape shape;
   Workspace ws;
   Workspace wsq;            // server row (the re-quantized average): kRowChunks partial slots, 1 statistic
+  Workspace wss;            // selection statistics: [M_max][kRowChunks] partial slots, the statistics of ws
   uint32_t* code_scratch;   // [M_max][code_words(d_max)] or NULL
   uint32_t* qcode_scratch;  // [code_words(d_max)] or NULL
   float* gbar_scratch;      // [d_max rounded up to 4] or NULL: the averaged gradient of the server row
@@ -27,6 +28,7 @@ struct qasg_ctx {
   uint32_t stream_lag;      // kAutoLag: chosen from the row size
   uint32_t wait_polls;
   uint64_t launches;
+  bool ticket_dirty;        // a launch failed since the completion counter was last known to be zero
   bool profiling;
   std::vector<cudaEvent_t> events;  // pairs (start, stop), reused between profiles
   std::vector<int> event_kernel;    // kernel id of each recorded pair
@@ -106,7 +108,19 @@ qasg_status enter(const qasg_ctx* ctx) {
   return cudaSetDevice(ctx->device) == cudaSuccess ? QASG_OK : QASG_ERR_CUDA;
 }
 
-qasg_status leave() { return cudaGetLastError() == cudaSuccess ? QASG_OK : QASG_ERR_CUDA; }
+// A launch that failed may have left the grid-completion counter of the reduction kernels non-zero (its
+// last CTA puts it back to zero): the next call that uses it clears it first.
+qasg_status leave(qasg_ctx* ctx) {
+  if (cudaGetLastError() == cudaSuccess) return QASG_OK;
+  ctx->ticket_dirty = true;
+  return QASG_ERR_CUDA;
+}
+
+void clear_ticket_if_dirty(qasg_ctx* ctx, cudaStream_t stream) {
+  if (!ctx->ticket_dirty) return;
+  cudaMemsetAsync(ctx->ws.ticket, 0, sizeof(unsigned int), stream);
+  ctx->ticket_dirty = false;
+}
 
 // About four rounds of resident CTAs: enough items to balance the launch.
 uint32_t target_items(const qasg_ctx* ctx) {
@@ -129,6 +143,7 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
                    uint64_t* counts, cudaStream_t stream, const uint32_t* touched = nullptr) {
   const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
+  clear_ticket_if_dirty(ctx, stream);
   if (touched) {  // rows held in sparse form: one warp per tile
     const bool stochastic = p->quantizer != QASG_Q_THRESHOLD;
     if (!stochastic) {
@@ -186,6 +201,7 @@ void requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint6
                 cudaStream_t stream, const unsigned long long* denom = nullptr) {
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
   unsigned long long* count_out = reinterpret_cast<unsigned long long*>(qcount);
+  clear_ticket_if_dirty(ctx, stream);
   if (ctx->gbar_scratch) {
     float* gbar = ctx->gbar_scratch;
     const uint64_t ld = ((d + 3) / 4) * 4;
@@ -221,16 +237,21 @@ void select_quantize_pack(qasg_ctx* ctx, int rule, const float* g, uint64_t d, u
                           const qasg_params* p, const float* x, const float* h, const float* z, uint32_t* codes,
                           float* scales, float* thresholds, uint64_t* counts, uint32_t* indicators,
                           uint64_t* selected, cudaStream_t stream) {
-  // the selection kernel's items are chunks (each for all M workers), not (worker, chunk) pairs
-  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx) * M);
+  // The selection kernel's items are chunks (each for all M workers), not (worker, chunk) pairs: it takes
+  // shorter chunks (up to kRowChunks of them, about sixteen rounds of its resident CTAs) so that the launch
+  // still balances; its partials have their own slots.
+  const Geometry geo_sel =
+      make_geometry(d, ld_g, M, kRowChunks, static_cast<uint32_t>(ctx->shape.sm_count) * kSelectCtasPerSm * 16u * M);
+  const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
   const bool stochastic = p->quantizer == QASG_Q_TERNARY_STOCH;
   SelectScalars sc;
   sc.lambda = p->lambda;
   sc.lambda_t = p->lambda * static_cast<float>(t);
   unsigned long long* counts_out = reinterpret_cast<unsigned long long*>(counts);
+  clear_ticket_if_dirty(ctx, stream);
   {
     Launch l(ctx, kSelectStats, stream);
-    l += launch_select_stats(rule, stochastic, g, geo, x, rule == QASG_RULE_CMD ? h : z, sc, p->thr_coef, ctx->ws,
+    l += launch_select_stats(rule, stochastic, g, geo_sel, x, rule == QASG_RULE_CMD ? h : z, sc, p->thr_coef, ctx->wss,
                              indicators, thresholds, reinterpret_cast<unsigned long long*>(selected), ctx->shape,
                              stream);
   }
@@ -284,6 +305,7 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ctx->d_max = d_max;
   ctx->M_max = M_max;
   ctx->launches = 0;
+  ctx->ticket_dirty = false;
   ctx->profiling = false;
   ctx->stream_row_bytes = kDefaultStreamRowBytes;
   ctx->stream_lag = kAutoLag;
@@ -316,6 +338,12 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ok &= cudaMalloc(&ctx->wsq.selected, 64) == cudaSuccess;
   ctx->wsq.ticket = ctx->ws.ticket;
   ctx->wsq.status = ctx->ws.status;
+  ctx->wss = ctx->ws;
+  const size_t sel_slots = static_cast<size_t>(M_max) * kRowChunks;
+  ctx->wss.part_sum = nullptr, ctx->wss.part_max = nullptr, ctx->wss.part_cnt = nullptr;
+  ok &= cudaMalloc(&ctx->wss.part_sum, sel_slots * sizeof(double)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wss.part_max, sel_slots * sizeof(uint32_t)) == cudaSuccess;
+  ok &= cudaMalloc(&ctx->wss.part_cnt, sel_slots * sizeof(unsigned long long)) == cudaSuccess;
   if (ok && !(flags & QASG_CREATE_NO_CODE_SCRATCH)) {
     ok &= cudaMalloc(&ctx->code_scratch, static_cast<size_t>(M_max) * qasg_code_words(d_max) * 4) == cudaSuccess;
     ok &= cudaMalloc(&ctx->qcode_scratch, qasg_code_words(d_max) * 4) == cudaSuccess;
@@ -362,6 +390,9 @@ qasg_status qasg_destroy(qasg_ctx* ctx) {
   cudaFree(ctx->ksyn);
   cudaFree(ctx->ws.selected);
   cudaFree(ctx->wsq.selected);
+  cudaFree(ctx->wss.part_sum);
+  cudaFree(ctx->wss.part_max);
+  cudaFree(ctx->wss.part_cnt);
   cudaFree(ctx->wsq.part_sum);
   cudaFree(ctx->wsq.part_max);
   cudaFree(ctx->wsq.part_cnt);
@@ -398,7 +429,7 @@ qasg_status qasg_wait_selftest(qasg_ctx* ctx, uint32_t max_polls, void* stream) 
   qasg_status st = enter(ctx);
   if (st != QASG_OK) return st;
   ctx->launches += launch_wait_selftest(ctx->sync, ctx->ws.status, max_polls, static_cast<cudaStream_t>(stream));
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
@@ -413,7 +444,7 @@ qasg_status qasg_quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64
   if ((st = enter(ctx)) != QASG_OK) return st;
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales, thresholds, counts,
                 static_cast<cudaStream_t>(stream));
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_decode_average(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d,
@@ -425,7 +456,7 @@ qasg_status qasg_decode_average(qasg_ctx* ctx, const uint32_t* codes, const floa
   if ((st = enter(ctx)) != QASG_OK) return st;
   { Launch l(ctx, kDecodeAverage, static_cast<cudaStream_t>(stream)); l += launch_decode_average(codes, scales, d, M, gbar, ctx->ws.status, ctx->shape,
                                          static_cast<cudaStream_t>(stream)); }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_cmd_step(qasg_ctx* ctx, const float* q, float* x, float* h, uint64_t d, uint64_t t,
@@ -438,7 +469,7 @@ qasg_status qasg_cmd_step(qasg_ctx* ctx, const float* q, float* x, float* h, uin
   if ((st = enter(ctx)) != QASG_OK) return st;
   { Launch l(ctx, kDenseUpdateCmd, static_cast<cudaStream_t>(stream)); l += launch_dense_update(QASG_RULE_CMD, q, d, x, h, nullptr, scalars(params, t), ctx->shape,
                                        static_cast<cudaStream_t>(stream)); }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, float* z, uint64_t d,
@@ -451,7 +482,7 @@ qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, flo
   if ((st = enter(ctx)) != QASG_OK) return st;
   { Launch l(ctx, kDenseUpdateRda, static_cast<cudaStream_t>(stream)); l += launch_dense_update(QASG_RULE_RDA, q, d, x, h, z, scalars(params, t), ctx->shape,
                                        static_cast<cudaStream_t>(stream)); }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
@@ -464,13 +495,13 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
   if (params->quantizer == QASG_Q_NONE) {
     Launch l(ctx, rule == QASG_RULE_CMD ? kMeanUpdateCmd : kMeanUpdateRda, s);
     l += launch_mean_update(rule, g, d, ld_g, M, x, h, z, scalars(params, t), ctx->ws.status, ctx->shape, s);
-    return leave();
+    return leave(ctx);
   }
   uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales_out, nullptr, nullptr, s);
   { Launch l(ctx, rule == QASG_RULE_CMD ? kDecodeUpdateCmd : kDecodeUpdateRda, s); l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t),
                                         ctx->ws.status, ctx->shape, s); }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_quantize_pack_touched(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
@@ -486,7 +517,7 @@ qasg_status qasg_quantize_pack_touched(qasg_ctx* ctx, const float* g, uint64_t d
   if ((st = enter(ctx)) != QASG_OK) return st;
   quantize_pack(ctx, g, d, ld_g, M, t, params, codes, scales, thresholds, counts, static_cast<cudaStream_t>(stream),
                 touched);
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_step_touched(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g, uint32_t M,
@@ -511,7 +542,7 @@ qasg_status qasg_step_touched(qasg_ctx* ctx, qasg_rule rule, const float* g, uin
     l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t), ctx->ws.status,
                               ctx->shape, s);
   }
-  return leave();
+  return leave(ctx);
 }
 
 uint64_t qasg_optimal_scratch_bytes(uint64_t d) { return (d >= 1 && d < (1ull << 31)) ? optimal_scratch_bytes(d) : 0; }
@@ -530,6 +561,7 @@ qasg_status qasg_quantize_pack_optimal(qasg_ctx* ctx, const float* g, uint64_t d
   if (scratch_bytes < optimal_scratch_bytes(d)) return QASG_ERR_WORKSPACE;
   if ((st = enter(ctx)) != QASG_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  clear_ticket_if_dirty(ctx, s);
   for (uint32_t m = 0; m < M; ++m) {  // one row after the other through the same scratch
     Launch l(ctx, kOptimalThreshold, s);
     l += launch_optimal_threshold(g + static_cast<uint64_t>(m) * ld_g, d, scratch, ctx->ws.thresholds + m,
@@ -541,7 +573,7 @@ qasg_status qasg_quantize_pack_optimal(qasg_ctx* ctx, const float* g, uint64_t d
     l += launch_threshold_codes(g, geo, ctx->ws, codes, scales, reinterpret_cast<unsigned long long*>(counts),
                                 ctx->shape, s);
   }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_requantize(qasg_ctx* ctx, const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,
@@ -555,7 +587,7 @@ qasg_status qasg_requantize(qasg_ctx* ctx, const uint32_t* codes, const float* s
   if ((st = enter(ctx)) != QASG_OK) return st;
   requantize(ctx, codes, scales, d, M, t, params, qcodes, qscale, qthreshold, qcount,
              static_cast<cudaStream_t>(stream));
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
@@ -584,7 +616,7 @@ qasg_status qasg_step_double(qasg_ctx* ctx, qasg_rule rule, const float* g, uint
     l += launch_decode_update(rule, qcodes, ctx->wsq.scales, d, 1, x, h, z, scalars(params, t), ctx->ws.status,
                               ctx->shape, s);
   }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_select_quantize_pack(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
@@ -604,7 +636,7 @@ qasg_status qasg_select_quantize_pack(qasg_ctx* ctx, qasg_rule rule, const float
   if ((st = enter(ctx)) != QASG_OK) return st;
   select_quantize_pack(ctx, rule, g, d, ld_g, M, t, params, x, h, z, codes, scales, thresholds, counts, indicators,
                        selected, static_cast<cudaStream_t>(stream));
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_indicator_or(qasg_ctx* ctx, const uint32_t* indicators, uint64_t d, uint32_t M, uint32_t* isyn,
@@ -618,7 +650,7 @@ qasg_status qasg_indicator_or(qasg_ctx* ctx, const uint32_t* indicators, uint64_
     l += launch_indicator_or(indicators, d, M, isyn, reinterpret_cast<unsigned long long*>(ksyn), ctx->shape,
                              static_cast<cudaStream_t>(stream));
   }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_step_select(qasg_ctx* ctx, qasg_rule rule, int double_quant, const float* g, uint64_t d,
@@ -659,7 +691,7 @@ qasg_status qasg_step_select(qasg_ctx* ctx, qasg_rule rule, int double_quant, co
     l += launch_decode_update(rule, codes, ctx->ws.scales, d, M, x, h, z, scalars(params, t), ctx->ws.status,
                               ctx->shape, s);
   }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_step_host(qasg_ctx* ctx, qasg_rule rule, const float* g_host, uint64_t d, uint64_t ld_g,
@@ -721,7 +753,7 @@ qasg_status qasg_logreg_grad_dense(qasg_ctx* ctx, const float* X, const float* y
   if ((st = enter(ctx)) != QASG_OK) return st;
   { Launch l(ctx, kLogregDense, static_cast<cudaStream_t>(stream)); l += launch_logreg_dense(X, y, n_rows, d, M, shard_row0, batch_rows, B, t, x, g, ld_g, ctx->logreg_ws,
                                        ctx->ws.status, ctx->shape, static_cast<cudaStream_t>(stream)); }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
@@ -734,7 +766,7 @@ qasg_status qasg_logreg_grad_csr(qasg_ctx* ctx, const int64_t* rowptr, const int
   if ((st = enter(ctx)) != QASG_OK) return st;
   { Launch l(ctx, kLogregCsr, static_cast<cudaStream_t>(stream)); l += launch_logreg_csr(rowptr, colidx, vals, y, n_rows, d, M, shard_row0, batch_rows, B, t, x, g, ld_g,
                                      ctx->ws.status, ctx->shape, static_cast<cudaStream_t>(stream)); }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_logreg_grad_csr_touched(qasg_ctx* ctx, const int64_t* rowptr, const int32_t* colidx,
@@ -755,7 +787,7 @@ qasg_status qasg_logreg_grad_csr_touched(qasg_ctx* ctx, const int64_t* rowptr, c
                            ctx->ws.status, ctx->shape, s,
                            touched);
   }
-  return leave();
+  return leave(ctx);
 }
 
 qasg_status qasg_last_async_status(qasg_ctx* ctx, void* stream) {

@@ -420,6 +420,83 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
   return c;
 }
 
+// The same block function with the key schedule (k0 + r*W0, k1 + r*W1), r = 0..9, worked out once on the host
+// and passed by value: the twenty words are then constant operands of the xors, and a round is two widening
+// multiplies and two three-input xors.
+struct PhiloxKeys {
+  uint32_t k0[10], k1[10];
+};
+inline PhiloxKeys philox_key_schedule(uint64_t seed) {
+  PhiloxKeys ks;
+  uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    ks.k0[r] = k0;
+    ks.k1[r] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return ks;
+}
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys& ks) {
+  constexpr uint64_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t p0 = kM0 * c.x, p1 = kM1 * c.z;
+    c = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ c.y ^ ks.k0[round], static_cast<uint32_t>(p1),
+                   static_cast<uint32_t>(p0 >> 32) ^ c.w ^ ks.k1[round], static_cast<uint32_t>(p0));
+  }
+  return c;
+}
+
+// The stochastic quantizer keeps a coordinate iff u < RN(a / s) (fp32 division), a = |v|, u = k 2^-24 with
+// k = word >> 8.  The division is avoided where its outcome is certain.  With r24 = RN(1/s) 2^24 and
+// q = RN(a r24), q is within 2^-22 q (at most 4 for q <= 2^24; + 2^-124 where the quotient is subnormal) of
+// RN(a / s) 2^24, and u < p is k < ceil(p 2^24) for the integer k; so with K = ceil(q), wherever k is more than
+// 9 away from K, k < K decides.  A row of four coordinates takes the divisions only if one of its four is
+// within 9 (about one row in 200,000).  `fast` is false where 1/s would not be a normal number accurate to
+// 2^-24 (s = 0, huge, tiny or not finite): then every row takes the divisions.  A NaN magnitude gives K = 0:
+// not kept on either path.
+struct KeepTest {
+  float s, r24;
+  bool fast;
+};
+__device__ __forceinline__ KeepTest keep_test(float s) {
+  KeepTest kt;
+  kt.s = s;
+  kt.fast = s >= 7.8886090522101181e-31f && s <= 1.2676506002282294e30f;  // 2^-100 <= s <= 2^100
+  kt.r24 = kt.fast ? __frcp_rn(s) * 16777216.f : 0.f;
+  return kt;
+}
+// k - K for one coordinate: negative iff the fast test keeps it; `nearest` collects min |k - K| + 9 as unsigned.
+__device__ __forceinline__ int32_t keep_margin(uint32_t word, float a, const KeepTest& kt, uint32_t& nearest) {
+  const int32_t t = static_cast<int32_t>(word >> 8) - __float2int_ru(__fmul_rn(a, kt.r24));  // a >= 0: K >= 0
+  nearest = min(nearest, static_cast<uint32_t>(t + 9));
+  return t;
+}
+__device__ __forceinline__ bool keeps_exact(uint32_t word, float a, float s) {
+  return static_cast<float>(word >> 8) * 5.9604644775390625e-08f < __fdiv_rn(a, s);
+}
+// 2-bit code (1 = +1, 2 = -1, 0 = dropped) from the keep mask (all ones or 0) and the sign bit of v; a kept
+// coordinate is never +-0.
+__device__ __forceinline__ uint32_t code_of(float v, uint32_t keep_mask) {
+  return keep_mask & (1u + (__float_as_uint(v) >> 31));
+}
+// The code byte of four coordinates that share the Philox block w.
+__device__ __forceinline__ uint32_t stochastic_code_byte(const float4& v, const uint4& w, const KeepTest& kt) {
+  uint32_t nearest = 0xffffffffu;
+  const int32_t tx = keep_margin(w.x, fabsf(v.x), kt, nearest), ty = keep_margin(w.y, fabsf(v.y), kt, nearest);
+  const int32_t tz = keep_margin(w.z, fabsf(v.z), kt, nearest), tw = keep_margin(w.w, fabsf(v.w), kt, nearest);
+  uint32_t mx = static_cast<uint32_t>(tx >> 31), my = static_cast<uint32_t>(ty >> 31);
+  uint32_t mz = static_cast<uint32_t>(tz >> 31), mw = static_cast<uint32_t>(tw >> 31);
+  if (!kt.fast || nearest <= 18u) {
+    mx = keeps_exact(w.x, fabsf(v.x), kt.s) ? 0xffffffffu : 0u;
+    my = keeps_exact(w.y, fabsf(v.y), kt.s) ? 0xffffffffu : 0u;
+    mz = keeps_exact(w.z, fabsf(v.z), kt.s) ? 0xffffffffu : 0u;
+    mw = keeps_exact(w.w, fabsf(v.w), kt.s) ? 0xffffffffu : 0u;
+  }
+  return code_of(v.x, mx) + 4u * code_of(v.y, my) + 16u * code_of(v.z, mz) + 64u * code_of(v.w, mw);
+}
+
 __device__ __forceinline__ float philox_uniform(uint32_t word) {
   return static_cast<float>(word >> 8) * 5.9604644775390625e-08f;  // 2^-24, exact
 }

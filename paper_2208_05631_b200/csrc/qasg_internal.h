@@ -20,6 +20,7 @@ constexpr int kMaxChunks = 1024;
 constexpr int kMaxWorkers = 64;
 // The server row (the averaged gradient, re-quantized) is one long row: it may use more chunks.
 constexpr int kRowChunks = 8 * kMaxChunks;
+constexpr int kSelectCtasPerSm = 3;  // resident CTAs of the selection-statistics kernel
 
 enum : unsigned { kFlagNonFinite = 1u, kFlagBadCode = 2u, kFlagBadIndex = 4u, kFlagTimeout = 8u };
 

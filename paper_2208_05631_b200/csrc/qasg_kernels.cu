@@ -169,29 +169,36 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
   auto body = [&](const float4 (&v)[kTileRows], const TileMask& mask, uint32_t k) {
         double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
         uint32_t bytes[kTileRows];
+        auto rows = [&](auto use_mask) {
 #pragma unroll
-        for (int r = 0; r < kTileRows; ++r) {
-          const float4 t = v[r];
-          // strict comparisons; a NaN threshold or value compares false and codes 0
-          float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
-          float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
-          float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
-          float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
-          if (kMasked) {
-            const uint32_t nib = mask.nibble(r, j);
-            const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
-            const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
-            px *= sx, nx *= sx, py *= sy, ny *= sy, pz *= sz, nz *= sz, pw *= sw, nw *= sw;
+          for (int r = 0; r < kTileRows; ++r) {
+            float4 t = v[r];
+            if (decltype(use_mask)::value) {  // a coordinate that is not selected is not sent: it enters as +0.0, which codes 0
+              const uint32_t nib = mask.nibble(r, j);
+              t.x = (nib & 1u) ? t.x : 0.f, t.y = (nib & 2u) ? t.y : 0.f;
+              t.z = (nib & 4u) ? t.z : 0.f, t.w = (nib & 8u) ? t.w : 0.f;
+            }
+            // strict comparisons; a NaN threshold or value compares false and codes 0
+            const float px = t.x > delta ? 1.f : 0.f, nx = t.x < ndelta ? 1.f : 0.f;
+            const float py = t.y > delta ? 1.f : 0.f, ny = t.y < ndelta ? 1.f : 0.f;
+            const float pz = t.z > delta ? 1.f : 0.f, nz = t.z < ndelta ? 1.f : 0.f;
+            const float pw = t.w > delta ? 1.f : 0.f, nw = t.w < ndelta ? 1.f : 0.f;
+            const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;  // 1.0f where kept
+            // |v| * 1 = |v| and |v| * 0 = +0: the kept magnitudes enter the sum unchanged
+            cx += static_cast<double>(fabsf(t.x) * kx);
+            cy += static_cast<double>(fabsf(t.y) * ky);
+            cz += static_cast<double>(fabsf(t.z) * kz);
+            cw += static_cast<double>(fabsf(t.w) * kw);
+            cntf += (kx + ky) + (kz + kw);  // exact: far below 2^24 per thread and chunk
+            bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
           }
-          const float kx = px + nx, ky = py + ny, kz = pz + nz, kw = pw + nw;  // 1.0f where kept
-          // |v| * 1 = |v| and |v| * 0 = +0: the kept magnitudes enter the sum unchanged
-          cx += static_cast<double>(fabsf(t.x) * kx);
-          cy += static_cast<double>(fabsf(t.y) * ky);
-          cz += static_cast<double>(fabsf(t.z) * kz);
-          cw += static_cast<double>(fabsf(t.w) * kw);
-          cntf += (kx + ky) + (kz + kw);  // exact: far below 2^24 per thread and chunk
-          bytes[r] = pack4({px, nx}, {py, ny}, {pz, nz}, {pw, nw});
-        }
+        };
+        // A warp whose 512 coordinates of this tile are all selected (its 16 indicator words are all ones)
+        // takes the unmasked arithmetic; the decision is the same in every lane.
+        if (kMasked && !__all_sync(0xffffffffu, (j & 31) >= 16 || mask.word == 0xffffffffu))
+          rows(std::true_type{});
+        else
+          rows(std::false_type{});
         store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
         chunk_sum.add_tile((cx + cy) + (cz + cw));
       };
@@ -214,7 +221,7 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
 // ------------------------------------------------------------------ pass B': stochastic codes
 template <bool kMasked>
 __global__ void __launch_bounds__(kThreads, 4)
-stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed, uint64_t t,
+stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, PhiloxKeys keys, uint64_t t,
                         uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
                         unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
   __shared__ uint32_t sm_cnt[kThreads / 32];
@@ -223,7 +230,6 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
   const uint32_t n_items = geo.M * geo.chunks;
   const uint64_t row_words = (geo.d + 15) >> 4;
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
-  const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
   const uint32_t t_lo = static_cast<uint32_t>(t), t_hi = static_cast<uint32_t>(t >> 32);
   chain_wait();
   chain_trigger();
@@ -231,7 +237,7 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
     uint8_t* codes8 = reinterpret_cast<uint8_t*>(codes + static_cast<uint64_t>(m) * row_words);
-    const float scale = ws.scales[m];
+    const KeepTest kt = keep_test(ws.scales[m]);
     const uint32_t* ind_row = kMasked ? indicators + static_cast<uint64_t>(m) * ((geo.d + 31) >> 5) : nullptr;
     const uint32_t k0 = c * geo.group;
     const uint32_t k1 = min(k0 + geo.group, geo.tiles);
@@ -243,17 +249,13 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, uint64_t seed
         const float4 v = tile[r];
         // coordinates 4*blk .. 4*blk+3 share one Philox block
         const uint32_t blk = k * (kTile / 4) + r * (kTileCols / 4) + j;
-        const uint4 w = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), key0, key1);
-        // |v|/s with IEEE division; s = 0 gives NaN and the comparison is false.
-        bool kx = philox_uniform(w.x) < __fdiv_rn(fabsf(v.x), scale);
-        bool ky = philox_uniform(w.y) < __fdiv_rn(fabsf(v.y), scale);
-        bool kz = philox_uniform(w.z) < __fdiv_rn(fabsf(v.z), scale);
-        bool kw = philox_uniform(w.w) < __fdiv_rn(fabsf(v.w), scale);
-        if (kMasked) {
+        const uint4 w = philox4x32_10(make_uint4(blk, stream_base + m, t_lo, t_hi), keys);
+        // u < |v|/s as the IEEE division decides it; s = 0 gives NaN and the comparison is false.
+        bytes[r] = stochastic_code_byte(v, w, kt);
+        if (kMasked) {  // unselected coordinates code 0: the nibble's bits spread to the byte's four fields
           const uint32_t nib = mask.nibble(r, j);
-          kx = kx && (nib & 1u), ky = ky && (nib & 2u), kz = kz && (nib & 4u), kw = kw && (nib & 8u);
+          bytes[r] &= ((nib & 1u) | ((nib & 2u) << 1) | ((nib & 4u) << 2) | ((nib & 8u) << 3)) * 3u;
         }
-        bytes[r] = pack4(split_code(v.x, kx), split_code(v.y, ky), split_code(v.z, kz), split_code(v.w, kw));
         cnt += nonzero_codes(bytes[r]);
       }
       store_code_bytes(codes8, k, j, k < full_tiles, row_words * 4, bytes);
@@ -575,6 +577,11 @@ __device__ __forceinline__ bool decode_batch(const uint8_t* __restrict__ codes8,
 
 __device__ __forceinline__ void prefetch_l2(const void* p) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+// One request for a run of bytes (16-byte aligned, a multiple of 16 long) to be brought into L2: it holds no
+// register and no shared memory while it is in flight.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
 // Two CTAs of kWideThreads threads per SM.  The workers are decoded in batches of 16 (their code bits
@@ -1084,9 +1091,8 @@ __host__ __device__ inline size_t select_smem_bytes(uint32_t M) {
   return static_cast<size_t>(M) * (kSelectDoublesPerWorker * sizeof(double) + 2 * sizeof(uint32_t));
 }
 
-// QRDA keeps two state tiles of z in registers next to the two gradient tiles: two CTAs per SM, not three.
 template <int kRule, bool kStochastic>
-__global__ void __launch_bounds__(kThreads, kRule == 0 ? 3 : 2)
+__global__ void __launch_bounds__(kThreads, kSelectCtasPerSm)
 select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __restrict__ x,
                     const float* __restrict__ hz, SelectScalars sc, float coef, Workspace ws,
                     uint32_t* __restrict__ indicators, float* __restrict__ thresholds_out,
@@ -1108,62 +1114,66 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
     __syncthreads();
     uint32_t pending = 0, pushed = 0;
     // The chunk is one stream of gradient tiles, (tile k, worker 0..M-1), (tile k+1, worker 0..M-1), ...:
-    // the next one is always in flight, and the state of tile k+1 is requested while the last worker of
-    // tile k is processed.  Of x only "non-zero" is kept (one bit per coordinate).
-    float4 ga[kTileRows], gb[kTileRows], xn[kTileRows], zc[kTileRows], zn[kTileRows];
+    // the next one is always in flight.  The state of a tile is read at its start.
+    // Of x only "non-zero" is kept, folded into the level each coordinate is compared with: -1 where
+    // x != 0 (every magnitude exceeds it), lambda (QRDA: lambda t) elsewhere.  The comparison is
+    // "greater or unordered": a NaN is marked, enters the sums and is reported.
+    float4 ga[kTileRows], gb[kTileRows], level[kTileRows], zc[kTileRows];
     bool a_cur = true;
     auto whole_tile = [&](uint32_t k) { return static_cast<uint64_t>(k + 1) * kTile <= geo.d; };
-    load_state_tile(x, geo.d, k0, j, whole_tile(k0), xn);
-    if (kRule == 1) load_state_tile(hz, geo.d, k0, j, whole_tile(k0), zn);
+    const float base_level = kRule == 0 ? sc.lambda : sc.lambda_t;
     load_tile(g, static_cast<uint64_t>(k0) * kTile, geo.d, j, ga);
     for (uint32_t k = k0; k < k1; ++k) {
       const uint64_t tile_base = static_cast<uint64_t>(k) * kTile;
-      uint32_t xmask = 0u;  // bit 4r + q: x != 0 at coordinate q of the thread's float4 of row r
+      const bool whole = whole_tile(k);
+      load_state_tile(x, geo.d, k, j, whole, level);
+      if (kRule == 1) load_state_tile(hz, geo.d, k, j, whole, zc);
 #pragma unroll
       for (int r = 0; r < kTileRows; ++r) {
-        xmask |= (xn[r].x != 0.f ? 1u : 0u) << (4 * r);
-        xmask |= (xn[r].y != 0.f ? 2u : 0u) << (4 * r);
-        xmask |= (xn[r].z != 0.f ? 4u : 0u) << (4 * r);
-        xmask |= (xn[r].w != 0.f ? 8u : 0u) << (4 * r);
-        if (kRule == 1) zc[r] = zn[r];
+        level[r].x = level[r].x != 0.f ? -1.f : base_level;
+        level[r].y = level[r].y != 0.f ? -1.f : base_level;
+        level[r].z = level[r].z != 0.f ? -1.f : base_level;
+        level[r].w = level[r].w != 0.f ? -1.f : base_level;
       }
+      // Two adjacent threads share an indicator byte and the even one writes it.  A tile that is not whole
+      // may reach past the row's last indicator word: those bytes are not written (the bits below d's word
+      // boundary that lie at or past d come out 0, since g, x and z read as +0.0 there).
+      const uint64_t byte0 = (tile_base >> 3) + (j >> 1);
+      uint32_t rows_written = kTileRows;
+      if (!whole) {
+        const uint64_t left = ind_words * 4 > byte0 ? (ind_words * 4 - byte0 + kTileCols / 8 - 1) / (kTileCols / 8) : 0;
+        rows_written = left < kTileRows ? static_cast<uint32_t>(left) : kTileRows;
+      }
+      if (j & 1) rows_written = 0u;
       // One worker's share of this tile: indicator bits, selected |g| into the fixed-order sum.
-      // Coordinates at or past d read as x = z = g = +0.0 and are never selected (lambda >= 0).
       auto worker_tile = [&](const float4 (&gv)[kTileRows], uint32_t m) {
-        uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words);
+        uint8_t* ind8 = reinterpret_cast<uint8_t*>(indicators + static_cast<uint64_t>(m) * ind_words) + byte0;
         double cx = 0.0, cy = 0.0, cz = 0.0, cw = 0.0;
-        float cntf = 0.f;
-        uint32_t best = 0u;
+        uint32_t cnt = 0u, best = 0u;
 #pragma unroll
         for (int r = 0; r < kTileRows; ++r) {
-          const uint64_t i0 = tile_base + r * kTileCols + 4 * j;
-          bool bx, by, bz, bw;
-          if (kRule == 0) {
-            bx = fabsf(gv[r].x) > sc.lambda, by = fabsf(gv[r].y) > sc.lambda;
-            bz = fabsf(gv[r].z) > sc.lambda, bw = fabsf(gv[r].w) > sc.lambda;
-          } else {
-            bx = fabsf(__fadd_rn(zc[r].x, gv[r].x)) > sc.lambda_t, by = fabsf(__fadd_rn(zc[r].y, gv[r].y)) > sc.lambda_t;
-            bz = fabsf(__fadd_rn(zc[r].z, gv[r].z)) > sc.lambda_t, bw = fabsf(__fadd_rn(zc[r].w, gv[r].w)) > sc.lambda_t;
+          const float4 gr = gv[r];
+          float dx = gr.x, dy = gr.y, dz = gr.z, dw = gr.w;
+          if (kRule == 1) {
+            dx = __fadd_rn(zc[r].x, gr.x), dy = __fadd_rn(zc[r].y, gr.y);
+            dz = __fadd_rn(zc[r].z, gr.z), dw = __fadd_rn(zc[r].w, gr.w);
           }
-          const uint32_t nib = ((xmask >> (4 * r)) & 15u) | static_cast<uint32_t>(bx) | (static_cast<uint32_t>(by) << 1) |
-                               (static_cast<uint32_t>(bz) << 2) | (static_cast<uint32_t>(bw) << 3);
-          const float sx = (nib & 1u) ? 1.f : 0.f, sy = (nib & 2u) ? 1.f : 0.f;
-          const float sz = (nib & 4u) ? 1.f : 0.f, sw = (nib & 8u) ? 1.f : 0.f;
+          const float px = !(fabsf(dx) <= level[r].x) ? 1.f : 0.f, py = !(fabsf(dy) <= level[r].y) ? 1.f : 0.f;
+          const float pz = !(fabsf(dz) <= level[r].z) ? 1.f : 0.f, pw = !(fabsf(dw) <= level[r].w) ? 1.f : 0.f;
+          const float sx = fabsf(gr.x) * px, sy = fabsf(gr.y) * py, sz = fabsf(gr.z) * pz, sw = fabsf(gr.w) * pw;
           if (!kStochastic) {
-            cx += static_cast<double>(fabsf(gv[r].x) * sx);
-            cy += static_cast<double>(fabsf(gv[r].y) * sy);
-            cz += static_cast<double>(fabsf(gv[r].z) * sz);
-            cw += static_cast<double>(fabsf(gv[r].w) * sw);
+            cx += static_cast<double>(sx);
+            cy += static_cast<double>(sy);
+            cz += static_cast<double>(sz);
+            cw += static_cast<double>(sw);
           } else {
-            best = max(best, __float_as_uint(fabsf(gv[r].x) * sx));
-            best = max(best, __float_as_uint(fabsf(gv[r].y) * sy));
-            best = max(best, __float_as_uint(fabsf(gv[r].z) * sz));
-            best = max(best, __float_as_uint(fabsf(gv[r].w) * sw));
+            best = max(max(best, __float_as_uint(sx)), __float_as_uint(sy));
+            best = max(max(best, __float_as_uint(sz)), __float_as_uint(sw));
           }
-          cntf += (sx + sy) + (sz + sw);
-          // two adjacent threads share an indicator byte; the even one writes it (zeros past d)
+          const uint32_t nib = static_cast<uint32_t>(fmaf(8.f, pw, fmaf(4.f, pz, fmaf(2.f, py, px))));
+          cnt += __popc(nib);
           const uint32_t upper = __shfl_down_sync(0xffffffffu, nib, 1);
-          if ((j & 1) == 0 && (i0 >> 3) < ind_words * 4) ind8[i0 >> 3] = static_cast<uint8_t>(nib | (upper << 4));
+          if (static_cast<uint32_t>(r) < rows_written) ind8[r * (kTileCols / 8)] = static_cast<uint8_t>(nib | (upper << 4));
         }
         if (!kStochastic) {
           const double v = warp_pair_tree((cx + cy) + (cz + cw));
@@ -1172,7 +1182,7 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
           best = __reduce_max_sync(0xffffffffu, best);
           if (lane == 0 && best) atomicMax(&sm_max[m], best);
         }
-        const uint32_t cnt = __reduce_add_sync(0xffffffffu, static_cast<uint32_t>(cntf));
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
         if (lane == 0 && cnt) atomicAdd(&sm_cnt[m], cnt);
       };
       for (uint32_t m = 0; m < M; ++m) {
@@ -1181,8 +1191,6 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
             load_tile(g + static_cast<uint64_t>(m + 1) * geo.ld, tile_base, geo.d, j, nxt);
           } else if (k + 1 < k1) {
             load_tile(g, tile_base + kTile, geo.d, j, nxt);
-            load_state_tile(x, geo.d, k + 1, j, whole_tile(k + 1), xn);
-            if (kRule == 1) load_state_tile(hz, geo.d, k + 1, j, whole_tile(k + 1), zn);
           }
         };
         if (a_cur) {
@@ -1211,7 +1219,7 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
     }
     __syncthreads();
     for (uint32_t wm = j; wm < M; wm += kThreads) {
-      const uint64_t p = static_cast<uint64_t>(wm) * kMaxChunks + c;
+      const uint64_t p = static_cast<uint64_t>(wm) * kRowChunks + c;
       ws.part_sum[p] = kStochastic ? 0.0 : tile_fold(stacks + wm * 32, pushed, geo.log2_group);
       ws.part_cnt[p] = sm_cnt[wm];
       ws.part_max[p] = sm_max[wm];
@@ -1225,13 +1233,22 @@ select_stats_kernel(const float* __restrict__ g, Geometry geo, const float* __re
     unsigned long long n = 0;
     uint32_t bmax = 0u;
     for (uint32_t idx = lane; idx < geo.chunks; idx += 32) {
-      n += __ldcg(ws.part_cnt + static_cast<uint64_t>(m) * kMaxChunks + idx);
-      if (kStochastic) bmax = max(bmax, __ldcg(ws.part_max + static_cast<uint64_t>(m) * kMaxChunks + idx));
+      n += __ldcg(ws.part_cnt + static_cast<uint64_t>(m) * kRowChunks + idx);
+      if (kStochastic) bmax = max(bmax, __ldcg(ws.part_max + static_cast<uint64_t>(m) * kRowChunks + idx));
     }
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
     double total = 0.0;
-    if (!kStochastic) total = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+    if (!kStochastic) {  // pairwise tree over the worker's up to kRowChunks = 8 * kMaxChunks partials
+      double blk[kRowChunks / kMaxChunks];
+#pragma unroll 1
+      for (uint32_t b = 0; b < kRowChunks / kMaxChunks; ++b) {
+        const uint32_t base = b * kMaxChunks;
+        blk[b] = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kRowChunks + base,
+                                 geo.chunks > base ? geo.chunks - base : 0u, lane);
+      }
+      total = ((blk[0] + blk[1]) + (blk[2] + blk[3])) + ((blk[4] + blk[5]) + (blk[6] + blk[7]));
+    }
     if (kStochastic) bmax = __reduce_max_sync(0xffffffffu, bmax);
     if (lane == 0) {
       ws.selected[m] = n;
@@ -1326,11 +1343,11 @@ int launch_stochastic_codes(const float* g, const Geometry& geo, uint64_t seed, 
                             unsigned long long* counts_out, const LaunchShape& shape,
                             cudaStream_t stream, const uint32_t* indicators) {
   if (indicators)
-    launch_chained(stochastic_codes_kernel<true>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo, seed,
-                   t, stream_base, ws, codes, scales_out, counts_out, indicators);
+    launch_chained(stochastic_codes_kernel<true>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo,
+                   philox_key_schedule(seed), t, stream_base, ws, codes, scales_out, counts_out, indicators);
   else
     launch_chained(stochastic_codes_kernel<false>, reduce_grid(geo, shape), kThreads, 0, stream, shape.chained, g, geo,
-                   seed, t, stream_base, ws, codes, scales_out, counts_out, static_cast<const uint32_t*>(nullptr));
+                   philox_key_schedule(seed), t, stream_base, ws, codes, scales_out, counts_out, static_cast<const uint32_t*>(nullptr));
   return 1;
 }
 
@@ -1339,7 +1356,7 @@ int launch_select_stats(int rule, bool stochastic, const float* g, const Geometr
                         uint32_t* indicators, float* thresholds_out, unsigned long long* selected_out,
                         const LaunchShape& shape, cudaStream_t stream) {
   const size_t smem = select_smem_bytes(geo.M);
-  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * (rule == 0 ? 3 : 2);
+  const uint64_t resident = static_cast<uint64_t>(shape.sm_count) * kSelectCtasPerSm;
   const unsigned grid = static_cast<unsigned>(geo.chunks < resident ? geo.chunks : resident);
 #define QASG_SELECT(R, S)                                                                                    \
   do {                                                                                                       \

@@ -73,6 +73,12 @@ def random_state(d, seed=2, device="cpu"):
     return x, h, z
 
 
+def bernoulli_mask(d, density, seed=2, device="cpu"):
+    """fp32 [d] of zeros and ones, one with probability `density` (for a sparse iterate)."""
+    gen = _torch_gen(int(seed) + 2000003, device)
+    return (torch.rand(d, generator=gen, device=device, dtype=torch.float32) < float(density)).to(torch.float32)
+
+
 # ------------------------------------------------------------------ logistic regression
 def shard_rows(n, M):
     """Row ranges of M equal contiguous shards: int64 [M+1]."""
