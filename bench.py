@@ -508,6 +508,8 @@ def new_context(libqasg, rig, args, d, M):
     ctx = libqasg.Context(d, M, device=rig.local)
     if args.stream_row_bytes:
         ctx.set_option(libqasg.OPT_STREAM_ROW_BYTES, args.stream_row_bytes)
+    if args.one_launch_step_bytes is not None:
+        ctx.set_option(libqasg.OPT_ONE_LAUNCH_STEP_BYTES, args.one_launch_step_bytes)
     return ctx
 
 
@@ -556,7 +558,7 @@ def run_config1(rig, args):
     ld = d
     gs = torch.stack([torch.from_numpy(inputs.optimizer_only_gradients(d, M, t, seed=0)) for t in range(1, T + 1)]).to(dev)
     x, h = (torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(2))
-    ctx = libqasg.Context(d, M, device=rig.local)
+    ctx = new_context(libqasg, rig, args, d, M)
     params = libqasg.make_params(1e-3, 0.1, 1e-8, quantizer=quantizer_of(args, libqasg), seed=0)
 
     def run():
@@ -646,7 +648,7 @@ def run_config2(rig, args):
     n, d, M, B = 65536, 4096, 8, 512
     prob = inputs.logreg_dense_problem(n=n, d=d, M=M, seed=1)
     X, y = torch.from_numpy(prob["X"]).to(dev), torch.from_numpy(prob["y"]).to(dev)
-    ctx = libqasg.Context(d, M, device=rig.local)
+    ctx = new_context(libqasg, rig, args, d, M)
     params = libqasg.make_params(1e-4, ETA, DELTA, quantizer=quantizer_of(args, libqasg), seed=1)
     state = {r: [torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(3)] for r in (0, 1)}
     g = torch.empty((M, d), dtype=torch.float32, device=dev)
@@ -716,7 +718,7 @@ def run_config4(rig, args):
     n, d, M, B = args.csr_rows, 1 << 24, 16, 1024
     prob = inputs.logreg_csr_problem(n=n, d=d, M=M, nnz_per_row=80, seed=3)
     dev_args = [torch.from_numpy(prob[k]).to(dev) for k in ("rowptr", "colidx", "vals", "y")]
-    ctx = libqasg.Context(d, M, device=rig.local)
+    ctx = new_context(libqasg, rig, args, d, M)
     params = libqasg.make_params(1e-5, ETA, DELTA, quantizer=quantizer_of(args, libqasg), seed=3)
     x, h, z = (torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(3))
     g = torch.zeros((M, d), dtype=torch.float32, device=dev)
@@ -828,6 +830,7 @@ def run_config5(rig, args):
          config={"workload": WORKLOAD_5, "quantizer": args.quantizer, "variant": args.variant,
                  "l2": "flushed (a 252 MiB buffer written) and the state restored before every timed step",
                  "one_launch_quantizer_row_bytes": args.stream_row_bytes,
+                 "one_launch_step_bytes": args.one_launch_step_bytes,
                  "note": "gbs_moved: bytes the step must move through device memory (g twice; once where the one-launch "
                          "quantizer codes a row out of L2); gbs_minimal: each gradient once + state once"},
          clocks=clocks, gpu_launches=launches, e2e=None, roofline=None, cpu_baseline=None, grid=grid)
@@ -842,7 +845,7 @@ def run_optimal(rig, args):
     M = int(args.workers.split(",")[0])
     for log2_d in range(args.min_log2_d, args.max_log2_d + 1, 2):
         d = 1 << log2_d
-        ctx = libqasg.Context(d, M, device=rig.local)
+        ctx = new_context(libqasg, rig, args, d, M)
         scratch = torch.empty(libqasg.optimal_scratch_bytes(d), dtype=torch.uint8, device=dev)
         params = libqasg.make_params(LAM, ETA, DELTA)
         for name, gen in (("normal", inputs.normal_gradients), ("student_t3", inputs.student_t_gradients)):
@@ -888,7 +891,7 @@ def run_touched(rig, args):
     from paper_2208_05631_b200 import libqasg
     dev = rig.dev
     d, M = 1 << 24, 16
-    ctx = libqasg.Context(d, M, device=rig.local)
+    ctx = new_context(libqasg, rig, args, d, M)
     params = libqasg.make_params(1e-5, ETA, DELTA)
     g = torch.randn((M, d), device=dev) * 0.01
     codes = torch.empty((M, libqasg.code_words(d)), dtype=torch.int32, device=dev)
@@ -941,6 +944,8 @@ def main():
     ap.add_argument("--max-log2-d", type=int, default=28)
     ap.add_argument("--workers", default="2,4,8,16,32", help="workload 5 and optimal")
     ap.add_argument("--csr-rows", type=int, default=1_000_000, help="workload 4: rows of the CSR matrix")
+    ap.add_argument("--one-launch-step-bytes", type=int, default=None,
+                    help="qasg_step as one launch up to this many bytes of gradients (default: the library's)")
     ap.add_argument("--stream-row-bytes", type=int, default=0,
                     help="workloads 3 and 5: quantize rows up to this size with the one-launch kernel (library option; 0 = default path)")
     ap.add_argument("--e2e-steps", type=int, default=2)

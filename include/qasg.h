@@ -110,11 +110,17 @@ qasg_status qasg_destroy(qasg_ctx* ctx);
  * call are then incomplete, and further calls do nothing until the status has been read).  It is off
  * by default: on a B200 it moves half the bytes but measured slower than the two launches.
  *
+ * QASG_OPT_ONE_LAUNCH_STEP_BYTES: qasg_step on at most that many bytes of gradients (4*d*M) runs its
+ * three passes as the phases of ONE launch (cooperative when it has more than one CTA) whose CTAs meet
+ * twice, with the same bounded waits and the same time-out behaviour: at such sizes a launch costs
+ * more than a pass (measured on a B200: 7 to 9 % faster up to 512 KB, slower from about 2 MB on).
+ *
  * Every setting gives the same bits. */
 typedef enum {
-  QASG_OPT_STREAM_ROW_BYTES = 0, /* 0 = never (default)                                          */
-  QASG_OPT_STREAM_LAG = 1,       /* 0, 1, 2, ...; 0xFFFFFFFF = chosen from the row size (default) */
-  QASG_OPT_WAIT_POLLS = 2        /* 1 .. 2^31; default 2^22 (about a second)                      */
+  QASG_OPT_STREAM_ROW_BYTES = 0,     /* 0 = never (default)                                          */
+  QASG_OPT_STREAM_LAG = 1,           /* 0, 1, 2, ...; 0xFFFFFFFF = chosen from the row size (default) */
+  QASG_OPT_WAIT_POLLS = 2,           /* 1 .. 2^31; default 2^22 (about a second)                      */
+  QASG_OPT_ONE_LAUNCH_STEP_BYTES = 3 /* 0 = never; default 524288 (faster there on a B200)           */
 } qasg_option;
 qasg_status qasg_set_option(qasg_ctx* ctx, qasg_option option, uint64_t value);
 
@@ -395,7 +401,7 @@ uint64_t qasg_launch_count(const qasg_ctx* ctx);
  * adds up, per kernel id (0 <= id < QASG_KERNEL_COUNT, names from qasg_kernel_name), the
  * elapsed milliseconds into ms[id] and the number of launches into launches[id] (both host
  * arrays of QASG_KERNEL_COUNT entries), then stops recording. */
-#define QASG_KERNEL_COUNT 24
+#define QASG_KERNEL_COUNT 26
 qasg_status qasg_profile_begin(qasg_ctx* ctx);
 qasg_status qasg_profile_end(qasg_ctx* ctx, double* ms, uint64_t* launches);
 const char* qasg_kernel_name(int id);

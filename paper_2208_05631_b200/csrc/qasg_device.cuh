@@ -172,6 +172,78 @@ __device__ __forceinline__ bool grid_last_cta(unsigned int* ticket, bool* sm_fla
   return last;
 }
 
+// ------------------------------------------------------------------ waits between CTAs (always bounded)
+__device__ __forceinline__ unsigned int load_acquire(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void store_release(unsigned int* p, unsigned int v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned int load_relaxed(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// One thread polls *flag until it holds `value`.  Gives up after max_polls polls (raising the abort
+// word and kFlagTimeout) or as soon as another CTA has given up.
+__device__ __forceinline__ bool wait_for_value(const unsigned int* flag, unsigned int value, unsigned int* abort_word,
+                                            unsigned int* status, uint32_t max_polls) {
+  for (uint32_t i = 0; i < max_polls; ++i) {
+    if (load_acquire(flag) == value) return true;
+    if (load_relaxed(abort_word) != 0u) break;
+    __nanosleep(i < 32 ? 20 : 200);
+  }
+  atomicExch(abort_word, 1u);
+  atomicOr(status, kFlagTimeout);
+  return false;
+}
+
+// One thread polls *counter until it holds at least `target` (a counter that only grows during the launch).
+__device__ __forceinline__ bool wait_until_at_least(const unsigned int* counter, unsigned int target,
+                                                    unsigned int* abort_word, unsigned int* status, uint32_t max_polls) {
+  for (uint32_t i = 0; i < max_polls; ++i) {
+    if (load_acquire(counter) >= target) return true;
+    if (load_relaxed(abort_word) != 0u) break;
+    if (i >= 64) __nanosleep(i < 1024 ? 40 : 400);
+  }
+  atomicExch(abort_word, 1u);
+  atomicOr(status, kFlagTimeout);
+  return false;
+}
+
+// All CTAs of a launch whose CTAs are resident together (a cooperative launch, or a single CTA) meet for the
+// `phase`-th time (1, 2, ...): what every thread wrote to global memory before the call is visible to every
+// thread of every CTA after it.  Returns false in every thread of the CTA if the wait ran out.
+__device__ __forceinline__ bool grid_meet(StreamSync* sync, uint32_t phase, uint32_t max_polls, unsigned int* status,
+                                          bool* sm_flag) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    bool ok = true;
+    if (gridDim.x > 1) {
+      atomicAdd(&sync->meet_count, 1u);
+      ok = wait_until_at_least(&sync->meet_count, phase * gridDim.x, &sync->abort, status, max_polls);
+    }
+    *sm_flag = ok;
+  }
+  __syncthreads();
+  const bool ok = *sm_flag;
+  __threadfence();
+  return ok;
+}
+// After the last meeting: the CTA that leaves last puts the counters back to zero for the next launch.
+__device__ __forceinline__ void grid_leave(StreamSync* sync) {
+  if (threadIdx.x == 0 && gridDim.x > 1) {
+    if (atomicAdd(&sync->meet_exit, 1u) == gridDim.x - 1) {
+      sync->meet_count = 0u;
+      sync->meet_exit = 0u;
+    }
+  }
+}
+
 // Calls body(tile_values, k) for the tiles k0 <= k < k1 of one worker row, keeping the loads
 // of tile k+1 in flight while tile k is processed (two register buffers, no copies).
 template <class Body>

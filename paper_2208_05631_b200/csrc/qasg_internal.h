@@ -65,6 +65,7 @@ struct StreamSync {
   unsigned int ready[kMaxWorkers];  // 1 once worker m's threshold (or scaler) of this call is published
   unsigned int abort;               // non-zero once a wait ran out: every later wait returns at once
   unsigned int probe, probe_abort;  // the wait self-test's own words (nothing ever sets probe)
+  unsigned int meet_count, meet_exit;  // the one-launch step: CTAs arrived at its meetings, CTAs that left
 };
 
 struct StreamParams {
@@ -181,6 +182,12 @@ int launch_quantize_stream(bool stochastic, bool keep_codes, const float* g, con
                            const LaunchShape& shape, cudaStream_t stream);
 // One bounded wait on a word nothing sets: raises kFlagTimeout after max_polls polls.
 int launch_wait_selftest(StreamSync* sync, unsigned int* status, uint32_t max_polls, cudaStream_t stream);
+// The whole fused step (passes A, B, C) as one launch whose CTAs meet twice; for small problems.
+// wsb: the statistics of ws with partial slots of its own (at least [M][kMaxChunks]) for pass B.
+int launch_fused_step(int rule, bool stochastic, const float* g, const Geometry& geo, float coef, uint64_t seed,
+                      uint64_t t, uint32_t stream_base, uint32_t max_polls, const Workspace& ws, const Workspace& wsb,
+                      StreamSync* sync, uint32_t* codes, float* scales_out, float* x, float* h, float* z,
+                      const StepScalars& sc, const LaunchShape& shape, cudaStream_t stream);
 
 void query_launch_shape(LaunchShape* shape);
 

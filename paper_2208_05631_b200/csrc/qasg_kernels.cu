@@ -46,15 +46,11 @@ Geometry make_geometry(uint64_t d, uint64_t ld, uint32_t M, uint32_t max_chunks,
 }
 
 // ------------------------------------------------------------------ pass A: sum |g|
-__global__ void __launch_bounds__(kThreads, 4)
-abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
-               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom) {
-  __shared__ ChunkSumStorage sm_sum;
-  __shared__ bool sm_last;
+// The CTA's share of the (worker, chunk) items: each chunk's fixed-order sum into its partial slot.
+__device__ __forceinline__ void abs_sum_partials(const float* __restrict__ g, const Geometry& geo, const Workspace& ws,
+                                                 ChunkSumStorage* sm_sum) {
   const int j = threadIdx.x;
-  chain_wait();  // the gradients may come from the launch before this one
-  chain_trigger();
-  ChunkSum chunk_sum(&sm_sum);
+  ChunkSum chunk_sum(sm_sum);
   auto begin = [](uint32_t, uint32_t) {};
   auto body = [&](const float4 (&v)[kTileRows], const TileMask&, uint32_t) {
         double cx = fabsf(v[0].x), cy = fabsf(v[0].y), cz = fabsf(v[0].z), cw = fabsf(v[0].w);
@@ -72,8 +68,13 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
         if (j == 0) ws.part_sum[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
       };
   stream_items<false>(g, nullptr, geo, j, begin, body, end);
-  if (!grid_last_cta(ws.ticket, &sm_last)) return;
-  const int warp = j >> 5, lane = j & 31;
+}
+
+// Delta_m of every worker from the chunk partials (all of them written and visible): one warp per worker.
+__device__ __forceinline__ void abs_sum_combine(const Geometry& geo, float coef, const Workspace& ws,
+                                                float* __restrict__ thresholds_out,
+                                                const unsigned long long* __restrict__ denom) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
     const double total = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
     if (lane == 0) {
@@ -85,17 +86,25 @@ abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace 
       if (!isfinite(total)) atomicOr(ws.status, kFlagNonFinite);
     }
   }
-  if (j == 0) *ws.ticket = 0u;
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+abs_sum_kernel(const float* __restrict__ g, Geometry geo, float coef, Workspace ws,
+               float* __restrict__ thresholds_out, const unsigned long long* __restrict__ denom) {
+  __shared__ ChunkSumStorage sm_sum;
+  __shared__ bool sm_last;
+  chain_wait();  // the gradients may come from the launch before this one
+  chain_trigger();
+  abs_sum_partials(g, geo, ws, &sm_sum);
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  abs_sum_combine(geo, coef, ws, thresholds_out, denom);
+  if (threadIdx.x == 0) *ws.ticket = 0u;
 }
 
 // ------------------------------------------------------------------ pass A': max |g|
-__global__ void __launch_bounds__(kThreads)
-abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
-  __shared__ uint32_t sm_warp[kThreads / 32];
-  __shared__ bool sm_last;
+__device__ __forceinline__ void abs_max_partials(const float* __restrict__ g, const Geometry& geo, const Workspace& ws,
+                                                 uint32_t* sm_warp) {
   const int j = threadIdx.x;
-  chain_wait();
-  chain_trigger();
   const uint32_t n_items = geo.M * geo.chunks;
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
@@ -124,8 +133,11 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
       ws.part_max[static_cast<uint64_t>(m) * kMaxChunks + c] = bmax;
     }
   }
-  if (!grid_last_cta(ws.ticket, &sm_last)) return;
-  const int warp = j >> 5, lane = j & 31;
+}
+
+// s_m = max |g_m| of every worker from the chunk maxima: one warp per worker.
+__device__ __forceinline__ void abs_max_combine(const Geometry& geo, const Workspace& ws) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
     uint32_t bmax = 0u;
     for (uint32_t idx = lane; idx < geo.chunks; idx += 32)
@@ -137,27 +149,33 @@ abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
       if (bmax >= 0x7f800000u) atomicOr(ws.status, kFlagNonFinite);
     }
   }
-  if (j == 0) *ws.ticket = 0u;
+}
+
+__global__ void __launch_bounds__(kThreads)
+abs_max_kernel(const float* __restrict__ g, Geometry geo, Workspace ws) {
+  __shared__ uint32_t sm_warp[kThreads / 32];
+  __shared__ bool sm_last;
+  chain_wait();
+  chain_trigger();
+  abs_max_partials(g, geo, ws, sm_warp);
+  if (!grid_last_cta(ws.ticket, &sm_last)) return;
+  abs_max_combine(geo, ws);
+  if (threadIdx.x == 0) *ws.ticket = 0u;
 }
 
 // ------------------------------------------------------------------ pass B: Q_Delta codes
 // kMasked: only coordinates whose indicator bit is set are candidates (sparse selection, Q(S(g, I))).
-template <bool kMasked>
-__global__ void __launch_bounds__(kThreads, 4)
-threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
-                       uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
-  __shared__ ChunkSumStorage sm_sum;
-  __shared__ uint32_t sm_cnt[kThreads / 32];
-  __shared__ bool sm_last;
+// The CTA's share of the (worker, chunk) items: code bytes, and each chunk's kept sum and count into its
+// partial slots.  kEarlyLoad: the first gradient tile is requested ahead of chain_wait().
+template <bool kMasked, bool kEarlyLoad>
+__device__ __forceinline__ void threshold_codes_partials(const float* __restrict__ g, const Geometry& geo,
+                                                         const Workspace& ws, uint32_t* __restrict__ codes,
+                                                         const uint32_t* __restrict__ indicators,
+                                                         ChunkSumStorage* sm_sum, uint32_t* sm_cnt) {
   const int j = threadIdx.x;
   const uint64_t row_words = (geo.d + 15) >> 4;
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
-  if (kMasked) {  // the indicator words come from the launch before this one
-    chain_wait();
-    chain_trigger();
-  }
-  ChunkSum chunk_sum(&sm_sum);
+  ChunkSum chunk_sum(sm_sum);
   uint8_t* codes8 = nullptr;  // per item: the worker's code row, its threshold, the kept count so far
   float delta = 0.f, ndelta = 0.f, cntf = 0.f;
   auto begin = [&](uint32_t m, uint32_t) {
@@ -211,28 +229,39 @@ threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
           ws.part_cnt[p] = total;
         }
       };
+  stream_items<kMasked, kEarlyLoad>(g, indicators, geo, j, begin, body, end);
+}
+
+template <bool kMasked>
+__global__ void __launch_bounds__(kThreads, 4)
+threshold_codes_kernel(const float* __restrict__ g, Geometry geo, Workspace ws,
+                       uint32_t* __restrict__ codes, float* __restrict__ scales_out,
+                       unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
+  __shared__ ChunkSumStorage sm_sum;
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ bool sm_last;
+  if (kMasked) {  // the indicator words come from the launch before this one
+    chain_wait();
+    chain_trigger();
+  }
   // unmasked: the first gradient tile is requested ahead of the wait for the thresholds
-  stream_items<kMasked, !kMasked>(g, indicators, geo, j, begin, body, end);
+  threshold_codes_partials<kMasked, !kMasked>(g, geo, ws, codes, indicators, &sm_sum, sm_cnt);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   finish_codes<true>(geo, ws, scales_out, counts_out);
-  if (j == 0) *ws.ticket = 0u;
+  if (threadIdx.x == 0) *ws.ticket = 0u;
 }
 
 // ------------------------------------------------------------------ pass B': stochastic codes
 template <bool kMasked>
-__global__ void __launch_bounds__(kThreads, 4)
-stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, PhiloxKeys keys, uint64_t t,
-                        uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
-                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
-  __shared__ uint32_t sm_cnt[kThreads / 32];
-  __shared__ bool sm_last;
+__device__ __forceinline__ void stochastic_codes_partials(const float* __restrict__ g, const Geometry& geo,
+                                                          const PhiloxKeys& keys, uint64_t t, uint32_t stream_base,
+                                                          const Workspace& ws, uint32_t* __restrict__ codes,
+                                                          const uint32_t* __restrict__ indicators, uint32_t* sm_cnt) {
   const int j = threadIdx.x;
   const uint32_t n_items = geo.M * geo.chunks;
   const uint64_t row_words = (geo.d + 15) >> 4;
   const uint32_t full_tiles = static_cast<uint32_t>(geo.d / kTile);
   const uint32_t t_lo = static_cast<uint32_t>(t), t_hi = static_cast<uint32_t>(t >> 32);
-  chain_wait();
-  chain_trigger();
   for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
     const uint32_t m = item / geo.chunks, c = item - m * geo.chunks;
     const float* row = g + static_cast<uint64_t>(m) * geo.ld;
@@ -265,9 +294,21 @@ stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, PhiloxKeys ke
     const unsigned long long total = block_count(cnt, sm_cnt);
     if (j == 0) ws.part_cnt[static_cast<uint64_t>(m) * kMaxChunks + c] = total;
   }
+}
+
+template <bool kMasked>
+__global__ void __launch_bounds__(kThreads, 4)
+stochastic_codes_kernel(const float* __restrict__ g, Geometry geo, PhiloxKeys keys, uint64_t t,
+                        uint32_t stream_base, Workspace ws, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
+                        unsigned long long* __restrict__ counts_out, const uint32_t* __restrict__ indicators) {
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ bool sm_last;
+  chain_wait();
+  chain_trigger();
+  stochastic_codes_partials<kMasked>(g, geo, keys, t, stream_base, ws, codes, indicators, sm_cnt);
   if (!grid_last_cta(ws.ticket, &sm_last)) return;
   finish_codes<false>(geo, ws, scales_out, counts_out);
-  if (j == 0) *ws.ticket = 0u;
+  if (threadIdx.x == 0) *ws.ticket = 0u;
 }
 
 // ------------------------------------------------------------------ pass C helpers
@@ -349,10 +390,13 @@ __device__ __forceinline__ uint32_t transpose_2bit_4x4(uint32_t w) {
 // Averaged decoded gradient of the four coordinates of group `grp` (Eq. SynQ_t).
 // kM4 > 0: the number of worker groups ceil(M/4) is a compile-time constant and the loop
 // unrolls; kM4 = 0: any M.
-template <int kM4, int kLanes>
+// kFresh: the codes were written earlier in this launch (by other CTAs): they are read from L2, not through
+// the read-only path.
+template <int kM4, int kLanes, bool kFresh = false>
 __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes8, uint64_t row_bytes,
                                                const double* lut, uint32_t M, double inv_m,
                                                uint64_t grp, uint32_t& bad) {
+  auto code_byte = [](const uint8_t* q) -> uint32_t { return kFresh ? __ldcg(q) : __ldg(q); };
   double q0 = 0.0, q1 = 0.0, q2 = 0.0, q3 = 0.0;
   const uint32_t m4 = kM4 > 0 ? static_cast<uint32_t>(kM4) : (M + 3) >> 2;
   if (kLanes > 1) lut += threadIdx.x & (kLanes - 1);  // kLanes copies: lanes l and l + kLanes share one
@@ -360,10 +404,10 @@ __device__ __forceinline__ float4 decode_group(const uint8_t* __restrict__ codes
   for (uint32_t G = 0; G < m4; ++G) {
     const uint8_t* p = codes8 + grp + static_cast<uint64_t>(4 * G) * row_bytes;
     const bool whole = (kM4 > 0 && G + 1 < m4);  // only the last group can be short of workers
-    uint32_t w = __ldg(p);
-    if (whole || 4 * G + 1 < M) w |= static_cast<uint32_t>(__ldg(p + row_bytes)) << 8;
-    if (whole || 4 * G + 2 < M) w |= static_cast<uint32_t>(__ldg(p + 2 * row_bytes)) << 16;
-    if (whole || 4 * G + 3 < M) w |= static_cast<uint32_t>(__ldg(p + 3 * row_bytes)) << 24;
+    uint32_t w = code_byte(p);
+    if (whole || 4 * G + 1 < M) w |= code_byte(p + row_bytes) << 8;
+    if (whole || 4 * G + 2 < M) w |= code_byte(p + 2 * row_bytes) << 16;
+    if (whole || 4 * G + 3 < M) w |= code_byte(p + 3 * row_bytes) << 24;
     bad |= w & (w >> 1) & 0x55555555u;
     w = transpose_2bit_4x4(w);
     const double* l = lut + static_cast<size_t>(G) * 256 * kLanes;
@@ -413,6 +457,30 @@ struct GroupState {
   }
 };
 
+// The last group of a vector whose length is not a multiple of 4: d % 4 coordinates, one by one.
+template <int kRule>
+__device__ __forceinline__ void update_ragged_group(float4 q, uint64_t grp, uint64_t d, float* __restrict__ x,
+                                                    float* __restrict__ h, float* __restrict__ z,
+                                                    const StepScalars& sc) {
+  const float qs[4] = {q.x, q.y, q.z, q.w};
+  for (uint64_t c = 4 * grp; c < d; ++c) {
+    if (kRule == 2) {
+      x[c] = qs[c - 4 * grp];
+      continue;
+    }
+    float xi = (kRule == 0) ? x[c] : 0.f, hi = h[c];
+    if (kRule == 0) {
+      cmd_update(qs[c - 4 * grp], xi, hi, sc);
+    } else {
+      float zi = z[c];
+      rda_update(qs[c - 4 * grp], xi, hi, zi, sc);
+      z[c] = zi;
+    }
+    x[c] = xi;
+    h[c] = hi;
+  }
+}
+
 // kThreadsC threads per CTA; a CTA takes kGroups * kThreadsC consecutive groups per round and a
 // thread owns kGroups of them, kThreadsC apart, with all their loads in flight before it decodes.
 // Up to 12 workers run with 16 copies of the tables (512 threads, two CTAs per SM); up to 52 with 16 or 8
@@ -453,28 +521,96 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
         GroupState<kRule> s0;
         s0.load(x, h, z, grp);
         s0.update_store(q, x, h, z, grp, sc);
-      } else {  // ragged tail: d % 4 coordinates
-        const float qs[4] = {q.x, q.y, q.z, q.w};
-        for (uint64_t c = 4 * grp; c < d; ++c) {
-          if (kRule == 2) {
-            x[c] = qs[c - 4 * grp];
-            continue;
-          }
-          float xi = (kRule == 0) ? x[c] : 0.f, hi = h[c];
-          if (kRule == 0) {
-            cmd_update(qs[c - 4 * grp], xi, hi, sc);
-          } else {
-            float zi = z[c];
-            rda_update(qs[c - 4 * grp], xi, hi, zi, sc);
-            z[c] = zi;
-          }
-          x[c] = xi;
-          h[c] = hi;
-        }
+      } else {
+        update_ragged_group<kRule>(q, grp, d, x, h, z, sc);
       }
     }
   }
   if (bad) atomicOr(status, kFlagBadCode);
+}
+
+// ------------------------------------------------------------------ the whole step in one launch
+// Passes A, B and C of a fused step as the phases of one launch, for sizes where three launches cost more
+// than the work: the CTAs (all resident: a cooperative launch, or one CTA) meet twice, after the chunk
+// partials of pass A and after those of pass B.  Behind a meeting every CTA works out all workers'
+// thresholds (scales) itself from the partials, the same arithmetic on the same numbers in every CTA, so
+// no third meeting is needed; CTA 0 writes the caller's copies.  The phases are the functions the three
+// kernels are made of: every output has the bits of the three-launch path.
+struct FusedParams {
+  float coef;            // threshold coefficient (0.75)
+  uint32_t max_polls;    // bound of the waits at the meetings
+  uint32_t stream_base;  // Philox counter word 1 = stream_base + worker
+  uint64_t t;
+};
+
+template <int kRule, bool kStochastic>
+__global__ void __launch_bounds__(kThreads, 2)
+fused_step_kernel(const float* __restrict__ g, Geometry geo, FusedParams fp, PhiloxKeys keys, Workspace ws,
+                  Workspace wsb, StreamSync* sync, uint32_t* __restrict__ codes, float* __restrict__ scales_out,
+                  float* __restrict__ x, float* __restrict__ h, float* __restrict__ z, StepScalars sc) {
+  extern __shared__ double sm_lut[];  // [ceil(M/4)][256]
+  __shared__ ChunkSumStorage sm_sum;
+  __shared__ uint32_t sm_cnt[kThreads / 32];
+  __shared__ float sm_scales[kMaxWorkers];
+  __shared__ bool sm_flag;
+  const int j = threadIdx.x;
+  chain_wait();  // the gradients may come from the launch before this one
+  chain_trigger();
+  // A launch that gave up leaves the meeting counters in an unknown state: until the host has cleared them
+  // (qasg_last_async_status does, when it reports the time-out) no further launch does anything.
+  if (j == 0) {
+    sm_flag = gridDim.x == 1 || load_relaxed(&sync->abort) == 0u;
+    if (!sm_flag) atomicOr(ws.status, kFlagTimeout);
+  }
+  __syncthreads();
+  if (!sm_flag) return;
+
+  // pass A: chunk partials, then every CTA the thresholds (or scalers) of all workers
+  if (kStochastic)
+    abs_max_partials(g, geo, ws, sm_cnt);
+  else
+    abs_sum_partials(g, geo, ws, &sm_sum);
+  if (!grid_meet(sync, 1u, fp.max_polls, ws.status, &sm_flag)) return;
+  if (kStochastic)
+    abs_max_combine(geo, ws);
+  else
+    abs_sum_combine(geo, fp.coef, ws, nullptr, nullptr);
+  __syncthreads();
+
+  // pass B: code bytes and chunk partials, then every CTA the scales of all workers.  Its partials go to
+  // slots of their own (wsb: the statistics of ws, other partial slots): a CTA that is still combining the
+  // partials of pass A must not find those of pass B in their place.
+  if (kStochastic)
+    stochastic_codes_partials<false>(g, geo, keys, fp.t, fp.stream_base, wsb, codes, nullptr, sm_cnt);
+  else
+    threshold_codes_partials<false, false>(g, geo, wsb, codes, nullptr, &sm_sum, sm_cnt);
+  if (!grid_meet(sync, 2u, fp.max_polls, ws.status, &sm_flag)) return;
+  finish_codes<!kStochastic>(geo, wsb, blockIdx.x == 0 ? scales_out : nullptr, nullptr);
+  __syncthreads();
+  if (j < static_cast<int>(geo.M)) sm_scales[j] = __ldcg(ws.scales + j);
+  __syncthreads();
+
+  // pass C: the CTA's share of the coordinates
+  build_decode_lut<1>(sm_lut, sm_scales, geo.M);
+  const uint8_t* codes8 = reinterpret_cast<const uint8_t*>(codes);
+  const uint64_t row_bytes = ((geo.d + 15) >> 4) * 4;
+  const uint64_t groups = (geo.d + 3) >> 2, full = geo.d >> 2;
+  const double inv_m = 1.0 / static_cast<double>(geo.M);
+  uint32_t bad = 0;
+  for (uint64_t grp = static_cast<uint64_t>(blockIdx.x) * kThreads + j; grp < groups;
+       grp += static_cast<uint64_t>(gridDim.x) * kThreads) {
+    if (grp < full) {
+      GroupState<kRule> s0;
+      s0.load(x, h, z, grp);
+      const float4 q = decode_group<0, 1, true>(codes8, row_bytes, sm_lut, geo.M, inv_m, grp, bad);
+      s0.update_store(q, x, h, z, grp, sc);
+    } else {
+      const float4 q = decode_group<0, 1, true>(codes8, row_bytes, sm_lut, geo.M, inv_m, grp, bad);
+      update_ragged_group<kRule>(q, grp, geo.d, x, h, z, sc);
+    }
+  }
+  if (bad) atomicOr(ws.status, kFlagBadCode);
+  grid_leave(sync);
 }
 
 // ------------------------------------------------------------------ pass C, eight coordinates per thread
@@ -1485,6 +1621,62 @@ int launch_decode_update(int rule, const uint32_t* codes, const float* scales, u
   else
     launch_decode_update_rule<2>(codes, scales, d, M, x, h, z, sc, status, shape, stream);
   return 1;
+}
+
+template <int kRule, bool kStochastic>
+static int launch_fused_step_as(const float* g, const Geometry& geo, const FusedParams& fp, const PhiloxKeys& keys,
+                                const Workspace& ws, const Workspace& wsb, StreamSync* sync, uint32_t* codes,
+                                float* scales_out, float* x, float* h, float* z, const StepScalars& sc,
+                                const LaunchShape& shape, cudaStream_t stream) {
+  auto kernel = fused_step_kernel<kRule, kStochastic>;
+  const size_t lut_bytes = static_cast<size_t>((geo.M + 3) / 4) * 256 * sizeof(double);
+  static thread_local int ctas_per_sm[64] = {0};  // per device, resolved on first use (the table is at most 32 KB)
+  int dev = 0;
+  cudaGetDevice(&dev);
+  int& resident = ctas_per_sm[dev & 63];
+  if (resident == 0) {
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kThreads, 32768);
+    if (resident < 1) resident = 1;
+  }
+  // enough CTAs for the (worker, chunk) items of passes A and B and for the coordinates of pass C,
+  // never more than are resident together
+  const uint64_t items = static_cast<uint64_t>(geo.M) * geo.chunks;
+  const uint64_t update_ctas = (((geo.d + 3) >> 2) + 2 * kThreads - 1) / (2 * kThreads);
+  uint64_t grid = items > update_ctas ? items : update_ctas;
+  const uint64_t max_grid = static_cast<uint64_t>(shape.sm_count) * resident;
+  if (grid > max_grid) grid = max_grid;
+  if (grid < 1) grid = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = lut_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = grid > 1 ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, g, geo, fp, keys, ws, wsb, sync, codes, scales_out, x, h, z, sc);
+  return 1;
+}
+
+int launch_fused_step(int rule, bool stochastic, const float* g, const Geometry& geo, float coef, uint64_t seed,
+                      uint64_t t, uint32_t stream_base, uint32_t max_polls, const Workspace& ws, const Workspace& wsb,
+                      StreamSync* sync, uint32_t* codes, float* scales_out, float* x, float* h, float* z,
+                      const StepScalars& sc, const LaunchShape& shape, cudaStream_t stream) {
+  FusedParams fp;
+  fp.coef = coef;
+  fp.max_polls = max_polls;
+  fp.stream_base = stream_base;
+  fp.t = t;
+  const PhiloxKeys keys = philox_key_schedule(seed);
+  if (rule == 0 && !stochastic)
+    return launch_fused_step_as<0, false>(g, geo, fp, keys, ws, wsb, sync, codes, scales_out, x, h, z, sc, shape, stream);
+  if (rule == 0)
+    return launch_fused_step_as<0, true>(g, geo, fp, keys, ws, wsb, sync, codes, scales_out, x, h, z, sc, shape, stream);
+  if (!stochastic)
+    return launch_fused_step_as<1, false>(g, geo, fp, keys, ws, wsb, sync, codes, scales_out, x, h, z, sc, shape, stream);
+  return launch_fused_step_as<1, true>(g, geo, fp, keys, ws, wsb, sync, codes, scales_out, x, h, z, sc, shape, stream);
 }
 
 int launch_decode_average(const uint32_t* codes, const float* scales, uint64_t d, uint32_t M,

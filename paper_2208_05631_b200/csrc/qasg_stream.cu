@@ -32,34 +32,6 @@
 
 namespace qasg {
 
-__device__ __forceinline__ unsigned int load_acquire(const unsigned int* p) {
-  unsigned int v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void store_release(unsigned int* p, unsigned int v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned int load_relaxed(const unsigned int* p) {
-  unsigned int v;
-  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-
-// One thread polls *flag until it holds `value`.  Gives up after max_polls polls (raising the abort
-// word and kFlagTimeout) or as soon as another CTA has given up.
-__device__ __forceinline__ bool wait_for_value(const unsigned int* flag, unsigned int value, unsigned int* abort_word,
-                                            unsigned int* status, uint32_t max_polls) {
-  for (uint32_t i = 0; i < max_polls; ++i) {
-    if (load_acquire(flag) == value) return true;
-    if (load_relaxed(abort_word) != 0u) break;
-    __nanosleep(i < 32 ? 20 : 200);
-  }
-  atomicExch(abort_word, 1u);
-  atomicOr(status, kFlagTimeout);
-  return false;
-}
-
 struct StreamItem {
   uint32_t index, kind, m, c, k0, k1;  // kind 0 = sum (A), 1 = codes (B), 2 = combine and publish (T); c = chunk
 };
@@ -521,12 +493,18 @@ quantize_stream_kernel(const float* __restrict__ g, Geometry geo, StreamParams s
     stream_publish_scale<kStochastic>(blockIdx.x, geo.chunks, sp.max_polls, ws, slots, sync, scales_out, counts_out);
 }
 
-// A wait that nothing ends: the bounded wait above on a word that no one sets.  The kernel returns after
-// max_polls polls with kFlagTimeout raised; nothing else is touched.
+// Waits that nothing ends: both bounded waits (for a value; for a counter to reach a target) on a word that
+// no one sets.  The kernel returns after 2 * max_polls polls with kFlagTimeout raised, only if both waits
+// gave up; nothing else is touched.
 __global__ void wait_selftest_kernel(StreamSync* sync, unsigned int* status, uint32_t max_polls) {
+  __shared__ unsigned int local_status;  // the waits raise their flag with an atomic: shared, not local, memory
   if (threadIdx.x == 0) {
+    local_status = 0u;
     sync->probe_abort = 0u;
-    wait_for_value(&sync->probe, 0xFFFFFFFFu, &sync->probe_abort, status, max_polls);
+    const bool a = wait_for_value(&sync->probe, 0xFFFFFFFFu, &sync->probe_abort, &local_status, max_polls);
+    sync->probe_abort = 0u;
+    const bool b = wait_until_at_least(&sync->probe, 1u, &sync->probe_abort, &local_status, max_polls);
+    if (!a && !b && local_status == kFlagTimeout) atomicOr(status, kFlagTimeout);
   }
 }
 

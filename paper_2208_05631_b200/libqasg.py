@@ -21,7 +21,7 @@ Q_THRESHOLD, Q_TERNARY_STOCH, Q_NONE = 0, 1, 2
 RULE_CMD, RULE_RDA = 0, 1
 CREATE_NO_CODE_SCRATCH = 1
 CREATE_SERIAL_LAUNCHES = 2
-OPT_STREAM_ROW_BYTES, OPT_STREAM_LAG, OPT_WAIT_POLLS = 0, 1, 2
+OPT_STREAM_ROW_BYTES, OPT_STREAM_LAG, OPT_WAIT_POLLS, OPT_ONE_LAUNCH_STEP_BYTES = 0, 1, 2, 3
 LAG_AUTO = 0xFFFFFFFF
 
 # Names every build of the library must export (checked by the CPU tests).
@@ -35,7 +35,7 @@ EXPORTS = [
     "qasg_optimal_scratch_bytes", "qasg_quantize_pack_optimal", "qasg_set_option", "qasg_wait_selftest",
 ]
 STATIC_MAX_WORKERS = 16
-KERNEL_COUNT = 24
+KERNEL_COUNT = 26
 
 
 class QasgError(RuntimeError):

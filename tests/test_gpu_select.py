@@ -102,3 +102,28 @@ def test_selected_run_40_steps(ctx, rule, double_quant):
         U.assert_zero_pattern(driven[0], xr, ref["a"], lam)
     assert ctx.last_async_status() == libqasg.OK
     assert 0 < ksum < T * d                                                 # the selection does select
+
+
+@pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
+@pytest.mark.parametrize("bad", [np.nan, np.inf])
+def test_non_finite_gradient_is_marked_and_reported(ctx, rule, bad):
+    """The selection compares "greater or unordered": a NaN or infinite component is marked where x = 0
+    too, and the call reports it; the other workers' indicators are those of the oracle."""
+    d, M, t, lam = 9001, 3, 4, 1e-2
+    g = inputs.normal_gradients(d, M, seed=8).numpy() * np.float32(0.02)
+    x, h, z = _state(d, 8)
+    x[4321] = 0.0
+    ref = O.select_quantize_workers(rule, g, x, h, z, t, lam, 0.1, 1e-8, libqasg.Q_THRESHOLD, seed=0)
+    g[1, 4321] = bad
+    g_dev, ld = U.grad_to_dev(g)
+    words = (d + 31) // 32
+    codes = U.new_codes(M, d)
+    ind = torch.zeros((M, words), dtype=torch.int32, device=U.dev())
+    scales = torch.zeros(M, dtype=torch.float32, device=U.dev())
+    ctx.select_quantize_pack(rule, g_dev, d, ld, M, t, libqasg.make_params(lam, 0.1, 1e-8), U.to_dev(x), U.to_dev(h),
+                             U.to_dev(z), codes, scales, None, None, ind, None)
+    assert ctx.last_async_status() == libqasg.ERR_NONFINITE
+    got = ind.cpu().numpy().view(np.uint32)
+    assert (got[1, 4321 >> 5] >> (4321 & 31)) & 1 == 1
+    assert np.array_equal(got[0], ref["ind_words"][0]) and np.array_equal(got[2], ref["ind_words"][2])
+    assert ctx.last_async_status() == libqasg.OK
