@@ -143,17 +143,24 @@ class ChunkSum {
 
 // Pairwise tree over a worker's kMaxChunks partial slots (slots >= chunks are +0.0),
 // computed by one warp: 32 adjacent slots per lane, then the lane butterfly.
+// kRounds: in how many rounds the lane's 32 slots are requested (4: eight at a time, few registers; 1: all
+// before the first is used, one round trip to L2 instead of four).  The sum is the same.
+template <int kRounds = 4>
 __device__ __forceinline__ double warp_chunk_tree(const double* part, uint32_t chunks, int lane) {
+  constexpr int kPer = 32 / kRounds;  // slots per round
   double top[4];
 #pragma unroll 1
-  for (int q = 0; q < 4; ++q) {  // 8 adjacent slots at a time keeps the register count low
-    double v[8];
+  for (int q0 = 0; q0 < 4; q0 += 4 / kRounds) {
+    double v[kPer];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const uint32_t idx = lane * 32 + q * 8 + k;
+    for (int k = 0; k < kPer; ++k) {
+      const uint32_t idx = lane * 32 + q0 * 8 + k;
       v[k] = idx < chunks ? __ldcg(part + idx) : 0.0;
     }
-    top[q] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+#pragma unroll
+    for (int q = 0; q < 4 / kRounds; ++q)
+      top[q0 + q] = ((v[8 * q] + v[8 * q + 1]) + (v[8 * q + 2] + v[8 * q + 3])) +
+                    ((v[8 * q + 4] + v[8 * q + 5]) + (v[8 * q + 6] + v[8 * q + 7]));
   }
   return warp_pair_tree((top[0] + top[1]) + (top[2] + top[3]));
 }
@@ -205,8 +212,10 @@ __device__ __forceinline__ bool wait_for_value(const unsigned int* flag, unsigne
 __device__ __forceinline__ bool wait_until_at_least(const unsigned int* counter, unsigned int target,
                                                     unsigned int* abort_word, unsigned int* status, uint32_t max_polls) {
   for (uint32_t i = 0; i < max_polls; ++i) {
-    if (load_acquire(counter) >= target) return true;
-    if (load_relaxed(abort_word) != 0u) break;
+    const unsigned int gave_up = load_relaxed(abort_word);  // both loads are in flight together
+    const unsigned int arrived = load_acquire(counter);
+    if (gave_up != 0u) break;  // first: after a launch that gave up the counter means nothing
+    if (arrived >= target) return true;
     if (i >= 64) __nanosleep(i < 1024 ? 40 : 400);
   }
   atomicExch(abort_word, 1u);
@@ -215,33 +224,70 @@ __device__ __forceinline__ bool wait_until_at_least(const unsigned int* counter,
 }
 
 // All CTAs of a launch whose CTAs are resident together (a cooperative launch, or a single CTA) meet for the
-// `phase`-th time (1, 2, ...): what every thread wrote to global memory before the call is visible to every
-// thread of every CTA after it.  Returns false in every thread of the CTA if the wait ran out.
+// `phase`-th time (1, 2, ...), and combine() (all threads of a CTA; it reads what the CTAs wrote to global
+// memory before they arrived and writes the same values whichever CTA runs it) has run before anyone goes on:
+//  * up to kMeetEveryone CTAs: everyone waits until all have arrived and then runs combine() itself (the
+//    shortest chain of round trips through L2);
+//  * more CTAs: the one that arrives last runs it and lets the others go (hundreds of CTAs reading the same
+//    few lines at once cost more than the extra hand-over).
+// What combine() wrote is visible to every thread of every CTA after the call (read it with loads that do
+// not go through L1 lines filled earlier in the launch).  Returns false in every thread of the CTA if the
+// wait ran out.
+// kLast: this is the launch's last meeting.  A CTA that has passed it says so; the one that says so last knows
+// that no CTA looks at the words any more and puts them back to zero for the next launch.
+// After a launch that gave up (the abort word is set until the host has cleared the words) every wait fails at
+// once: no further launch gets past its first meeting.
+constexpr unsigned int kMeetEveryone = 160;
+template <bool kLast, class Combine>
 __device__ __forceinline__ bool grid_meet(StreamSync* sync, uint32_t phase, uint32_t max_polls, unsigned int* status,
-                                          bool* sm_flag) {
+                                          uint32_t* sm_word, Combine&& combine) {
   __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) {
-    bool ok = true;
-    if (gridDim.x > 1) {
-      atomicAdd(&sync->meet_count, 1u);
-      ok = wait_until_at_least(&sync->meet_count, phase * gridDim.x, &sync->abort, status, max_polls);
-    }
-    *sm_flag = ok;
+  if (gridDim.x == 1) {
+    combine();
+    __syncthreads();
+    return true;
   }
-  __syncthreads();
-  const bool ok = *sm_flag;
-  __threadfence();
-  return ok;
-}
-// After the last meeting: the CTA that leaves last puts the counters back to zero for the next launch.
-__device__ __forceinline__ void grid_leave(StreamSync* sync) {
-  if (threadIdx.x == 0 && gridDim.x > 1) {
+  bool ok;
+  if (gridDim.x <= kMeetEveryone) {
+    if (threadIdx.x == 0) {
+      atomicAdd(&sync->meet_count, 1u);
+      *sm_word = wait_until_at_least(&sync->meet_count, phase * gridDim.x, &sync->abort, status, max_polls) ? 1u : 0u;
+    }
+    __syncthreads();
+    ok = *sm_word != 0u;
+    if (ok) combine();
+    __syncthreads();
+  } else {
+    if (threadIdx.x == 0) *sm_word = atomicAdd(&sync->meet_count, 1u) == phase * gridDim.x - 1 ? 1u : 0u;
+    __syncthreads();
+    const bool last = *sm_word != 0u;
+    if (last) {
+      __threadfence();
+      combine();
+      __threadfence();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      if (last) {
+        store_release(&sync->meet_go, phase);
+        *sm_word = 1u;
+      } else {
+        *sm_word = wait_until_at_least(&sync->meet_go, phase, &sync->abort, status, max_polls) ? 1u : 0u;
+      }
+    }
+    __syncthreads();
+    ok = *sm_word != 0u;
+  }
+  // said by a thread that the work right behind the meeting does not wait for
+  if (kLast && ok && threadIdx.x == blockDim.x - 1) {
     if (atomicAdd(&sync->meet_exit, 1u) == gridDim.x - 1) {
       sync->meet_count = 0u;
+      sync->meet_go = 0u;
       sync->meet_exit = 0u;
     }
   }
+  return ok;
 }
 
 // Calls body(tile_values, k) for the tiles k0 <= k < k1 of one worker row, keeping the loads
@@ -448,9 +494,11 @@ __device__ __forceinline__ unsigned long long block_count(uint32_t cnt, uint32_t
 
 // Last-CTA epilogue shared by both code kernels: per-worker totals of the counts, and for
 // the threshold quantizer the scale s_m = P_m / n_m.
-template <bool kThreshold>
+// sm_scales: if given, the CTA's shared copy of the M scales (valid after the CTA's next barrier).
+template <bool kThreshold, int kRounds = 4>
 __device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspace& ws,
-                                             float* scales_out, unsigned long long* counts_out) {
+                                             float* scales_out, unsigned long long* counts_out,
+                                             float* sm_scales = nullptr) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
     unsigned long long n = 0;
@@ -460,7 +508,8 @@ __device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspac
     for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
     float scale;
     if (kThreshold) {
-      const double picked = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+      const double picked =
+          warp_chunk_tree<kRounds>(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
       scale = n ? static_cast<float>(picked / static_cast<double>(n)) : 0.f;
     } else {
       scale = ws.scales[m];
@@ -470,6 +519,7 @@ __device__ __forceinline__ void finish_codes(const Geometry& geo, const Workspac
       if (kThreshold) ws.scales[m] = scale;
       if (scales_out) scales_out[m] = scale;
       if (counts_out) counts_out[m] = n;
+      if (sm_scales) sm_scales[m] = scale;
     }
   }
 }

@@ -65,7 +65,7 @@ struct StreamSync {
   unsigned int ready[kMaxWorkers];  // 1 once worker m's threshold (or scaler) of this call is published
   unsigned int abort;               // non-zero once a wait ran out: every later wait returns at once
   unsigned int probe, probe_abort;  // the wait self-test's own words (nothing ever sets probe)
-  unsigned int meet_count, meet_exit;  // the one-launch step: CTAs arrived at its meetings, CTAs that left
+  unsigned int meet_count, meet_go, meet_exit;  // the one-launch step: arrivals at its meetings, the meeting that is over, CTAs that left
 };
 
 struct StreamParams {

@@ -71,12 +71,14 @@ __device__ __forceinline__ void abs_sum_partials(const float* __restrict__ g, co
 }
 
 // Delta_m of every worker from the chunk partials (all of them written and visible): one warp per worker.
+template <int kRounds = 4>
 __device__ __forceinline__ void abs_sum_combine(const Geometry& geo, float coef, const Workspace& ws,
                                                 float* __restrict__ thresholds_out,
                                                 const unsigned long long* __restrict__ denom) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (uint32_t m = warp; m < geo.M; m += kThreads / 32) {
-    const double total = warp_chunk_tree(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
+    const double total =
+        warp_chunk_tree<kRounds>(ws.part_sum + static_cast<uint64_t>(m) * kMaxChunks, geo.chunks, lane);
     if (lane == 0) {
       // the mean is over all d coordinates, or over the selected ones when a count is given
       const unsigned long long n = denom ? denom[m] : geo.d;
@@ -532,10 +534,11 @@ decode_update_kernel(const uint32_t* __restrict__ codes, const float* __restrict
 // ------------------------------------------------------------------ the whole step in one launch
 // Passes A, B and C of a fused step as the phases of one launch, for sizes where three launches cost more
 // than the work: the CTAs (all resident: a cooperative launch, or one CTA) meet twice, after the chunk
-// partials of pass A and after those of pass B.  Behind a meeting every CTA works out all workers'
-// thresholds (scales) itself from the partials, the same arithmetic on the same numbers in every CTA, so
-// no third meeting is needed; CTA 0 writes the caller's copies.  The phases are the functions the three
-// kernels are made of: every output has the bits of the three-launch path.
+// partials of pass A and after those of pass B, and at each meeting all workers' thresholds (scales) are
+// worked out from the partials: by every CTA for itself when they are few, by the one that arrives last
+// when they are many (as the last CTA of the separate kernels does).  Same arithmetic on the same numbers
+// either way.  The phases are the functions the three kernels are made of: every output has the bits of
+// the three-launch path.
 struct FusedParams {
   float coef;            // threshold coefficient (0.75)
   uint32_t max_polls;    // bound of the waits at the meetings
@@ -543,6 +546,40 @@ struct FusedParams {
   uint64_t t;
 };
 
+template <bool kStochastic>
+__device__ __forceinline__ void fused_phase_a(const float* __restrict__ g, const Geometry& geo, const Workspace& ws,
+                                           ChunkSumStorage* sm_sum, uint32_t* sm_cnt) {
+  if (kStochastic)
+    abs_max_partials(g, geo, ws, sm_cnt);
+  else
+    abs_sum_partials(g, geo, ws, sm_sum);
+}
+// kRounds: 1 where one CTA combines for all (it reads up to 1024 partials per worker: one round trip to L2
+// instead of four); 4 where every CTA combines for itself (few partials; the small cases measured faster).
+template <bool kStochastic, int kRounds>
+__device__ __forceinline__ void fused_combine_a(const Geometry& geo, float coef, const Workspace& ws) {
+  if (kStochastic)
+    abs_max_combine(geo, ws);
+  else
+    abs_sum_combine<kRounds>(geo, coef, ws, nullptr, nullptr);
+}
+template <bool kStochastic>
+__device__ __forceinline__ void fused_phase_b(const float* __restrict__ g, const Geometry& geo, const PhiloxKeys& keys,
+                                           uint64_t t, uint32_t stream_base, const Workspace& wsb,
+                                           uint32_t* __restrict__ codes, ChunkSumStorage* sm_sum, uint32_t* sm_cnt) {
+  if (kStochastic)
+    stochastic_codes_partials<false>(g, geo, keys, t, stream_base, wsb, codes, nullptr, sm_cnt);
+  else
+    threshold_codes_partials<false, false>(g, geo, wsb, codes, nullptr, sm_sum, sm_cnt);
+}
+template <bool kStochastic, int kRounds>
+__device__ __forceinline__ void fused_combine_b(const Geometry& geo, const Workspace& wsb, float* scales_out,
+                                             float* sm_scales) {
+  finish_codes<!kStochastic, kRounds>(geo, wsb, scales_out, nullptr, sm_scales);
+}
+
+// Two CTAs per SM: the launch is for problems that do not fill the machine, and the phases keep their
+// registers (called instead of inlined, or squeezed into 64 registers, the small cases measured 20 % slower).
 template <int kRule, bool kStochastic>
 __global__ void __launch_bounds__(kThreads, 2)
 fused_step_kernel(const float* __restrict__ g, Geometry geo, FusedParams fp, PhiloxKeys keys, Workspace ws,
@@ -552,43 +589,38 @@ fused_step_kernel(const float* __restrict__ g, Geometry geo, FusedParams fp, Phi
   __shared__ ChunkSumStorage sm_sum;
   __shared__ uint32_t sm_cnt[kThreads / 32];
   __shared__ float sm_scales[kMaxWorkers];
-  __shared__ bool sm_flag;
+  __shared__ uint32_t sm_word;
   const int j = threadIdx.x;
   chain_wait();  // the gradients may come from the launch before this one
   chain_trigger();
-  // A launch that gave up leaves the meeting counters in an unknown state: until the host has cleared them
-  // (qasg_last_async_status does, when it reports the time-out) no further launch does anything.
-  if (j == 0) {
-    sm_flag = gridDim.x == 1 || load_relaxed(&sync->abort) == 0u;
-    if (!sm_flag) atomicOr(ws.status, kFlagTimeout);
+  // pass A: chunk partials, then the thresholds (or scalers) of all workers.  (After a launch that gave up
+  // no further launch gets past this meeting until the host has cleared the words: qasg_last_async_status
+  // does, when it reports the time-out.)
+  const bool everyone = gridDim.x <= kMeetEveryone;  // every CTA combines for itself
+  fused_phase_a<kStochastic>(g, geo, ws, &sm_sum, sm_cnt);
+  if (!grid_meet<false>(sync, 1u, fp.max_polls, ws.status, &sm_word, [&]() {
+        if (everyone)
+          fused_combine_a<kStochastic, 4>(geo, fp.coef, ws);
+        else
+          fused_combine_a<kStochastic, 1>(geo, fp.coef, ws);
+      }))
+    return;
+
+  // pass B: code bytes and chunk partials, then the scales of all workers.  Its partials go to slots of
+  // their own (wsb: the statistics of ws, other partial slots).
+  fused_phase_b<kStochastic>(g, geo, keys, fp.t, fp.stream_base, wsb, codes, &sm_sum, sm_cnt);
+  // where every CTA combines for itself the scales go straight into its shared copy
+  if (!grid_meet<true>(sync, 2u, fp.max_polls, ws.status, &sm_word, [&]() {
+        if (everyone)
+          fused_combine_b<kStochastic, 4>(geo, wsb, blockIdx.x == 0 ? scales_out : nullptr, sm_scales);
+        else
+          fused_combine_b<kStochastic, 1>(geo, wsb, scales_out, nullptr);
+      }))
+    return;
+  if (!everyone) {
+    if (j < static_cast<int>(geo.M)) sm_scales[j] = __ldcg(ws.scales + j);
+    __syncthreads();
   }
-  __syncthreads();
-  if (!sm_flag) return;
-
-  // pass A: chunk partials, then every CTA the thresholds (or scalers) of all workers
-  if (kStochastic)
-    abs_max_partials(g, geo, ws, sm_cnt);
-  else
-    abs_sum_partials(g, geo, ws, &sm_sum);
-  if (!grid_meet(sync, 1u, fp.max_polls, ws.status, &sm_flag)) return;
-  if (kStochastic)
-    abs_max_combine(geo, ws);
-  else
-    abs_sum_combine(geo, fp.coef, ws, nullptr, nullptr);
-  __syncthreads();
-
-  // pass B: code bytes and chunk partials, then every CTA the scales of all workers.  Its partials go to
-  // slots of their own (wsb: the statistics of ws, other partial slots): a CTA that is still combining the
-  // partials of pass A must not find those of pass B in their place.
-  if (kStochastic)
-    stochastic_codes_partials<false>(g, geo, keys, fp.t, fp.stream_base, wsb, codes, nullptr, sm_cnt);
-  else
-    threshold_codes_partials<false, false>(g, geo, wsb, codes, nullptr, &sm_sum, sm_cnt);
-  if (!grid_meet(sync, 2u, fp.max_polls, ws.status, &sm_flag)) return;
-  finish_codes<!kStochastic>(geo, wsb, blockIdx.x == 0 ? scales_out : nullptr, nullptr);
-  __syncthreads();
-  if (j < static_cast<int>(geo.M)) sm_scales[j] = __ldcg(ws.scales + j);
-  __syncthreads();
 
   // pass C: the CTA's share of the coordinates
   build_decode_lut<1>(sm_lut, sm_scales, geo.M);
@@ -610,7 +642,6 @@ fused_step_kernel(const float* __restrict__ g, Geometry geo, FusedParams fp, Phi
     }
   }
   if (bad) atomicOr(ws.status, kFlagBadCode);
-  grid_leave(sync);
 }
 
 // ------------------------------------------------------------------ pass C, eight coordinates per thread
