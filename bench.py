@@ -81,9 +81,9 @@ def minimal_bytes(M, rule):
 # quantizer's kernels, from one ncu capture at d = 2^24 (both kernels stream, so their traffic grows in
 # proportion to d).  Valid only for the kernel source it was taken from (checked by hash).
 NCU_TRAFFIC = {
-    "kernels_sha256": "15c39fbd299dd161025ec37617c0e0ae9bcdeef5e5b886510ff02a86c5f49841",
+    "kernels_sha256": "2ebc5709d2881f5bed57fd1081e966af7f0a286b30b60fde63c8990b17142613",
     "M": 8,
-    "bytes_per_coord": {"abs_sum": 541067520 / 2 ** 24, "threshold_codes": 568647424 / 2 ** 24},
+    "bytes_per_coord": {"abs_sum": 540856320 / 2 ** 24, "threshold_codes": 567921664 / 2 ** 24},
 }
 
 
