@@ -28,9 +28,11 @@ def ctx():
     c.close()
 
 
-@pytest.mark.parametrize("d,B,explicit", [(4096, 512, False), (260, 7, True), (4, 1, False)])
+# wide rows, a column count that is not a multiple of 128, more minibatch rows than row lanes
+@pytest.mark.parametrize("d,B,explicit", [(4096, 512, False), (260, 7, True), (4, 1, False), (8192, 33, True),
+                                          (8196, 9, False), (12000, 5, True), (1028, 300, True)])
 def test_dense_gradient(ctx, d, B, explicit):
-    M, n = 8, 8192 if d == 4096 else 256
+    M, n = 8, 8192 if d == 4096 else (1024 if d == 1028 else 256)
     prob = inputs.logreg_dense_problem(n=n, d=d, M=M, seed=1)
     rng = np.random.default_rng(2)
     x = (rng.standard_normal(d) * 0.05).astype(np.float32)
