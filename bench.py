@@ -81,7 +81,7 @@ def minimal_bytes(M, rule):
 # quantizer's kernels, from one ncu capture at d = 2^24 (both kernels stream, so their traffic grows in
 # proportion to d).  Valid only for the kernel source it was taken from (checked by hash).
 NCU_TRAFFIC = {
-    "kernels_sha256": "2ebc5709d2881f5bed57fd1081e966af7f0a286b30b60fde63c8990b17142613",
+    "kernels_sha256": "afcae0653967ed52d457675782f346e923cf18e16314d94894f1e1a64c4b6d06",
     "M": 8,
     "bytes_per_coord": {"abs_sum": 540856320 / 2 ** 24, "threshold_codes": 567921664 / 2 ** 24},
 }

@@ -589,34 +589,42 @@ __device__ __forceinline__ KeepTest keep_test(float s) {
   kt.r24 = kt.fast ? __frcp_rn(s) * 16777216.f : 0.f;
   return kt;
 }
-// k - K for one coordinate: negative iff the fast test keeps it; `nearest` collects min |k - K| + 9 as unsigned.
-__device__ __forceinline__ int32_t keep_margin(uint32_t word, float a, const KeepTest& kt, uint32_t& nearest) {
-  const int32_t t = static_cast<int32_t>(word >> 8) - __float2int_ru(__fmul_rn(a, kt.r24));  // a >= 0: K >= 0
-  nearest = min(nearest, static_cast<uint32_t>(t + 9));
+// hi32(a * b) + c as one multiply-add (the multiply pipe, not the integer pipe that the Philox xors keep busy).
+__device__ __forceinline__ uint32_t mad_hi(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+// k - K for one coordinate (k = word >> 8 = hi32(word * 2^24)): negative iff the fast test keeps it;
+// `nearest` collects min |k - K| + 9 as unsigned.
+__device__ __forceinline__ uint32_t keep_margin(uint32_t word, float a, const KeepTest& kt, uint32_t& nearest) {
+  const uint32_t K = static_cast<uint32_t>(__float2int_ru(__fmul_rn(a, kt.r24)));  // a >= 0: K >= 0
+  const uint32_t t = mad_hi(word, 1u << 24, 0u - K);
+  nearest = min(nearest, t + 9u);
   return t;
 }
 __device__ __forceinline__ bool keeps_exact(uint32_t word, float a, float s) {
   return static_cast<float>(word >> 8) * 5.9604644775390625e-08f < __fdiv_rn(a, s);
 }
-// 2-bit code (1 = +1, 2 = -1, 0 = dropped) from the keep mask (all ones or 0) and the sign bit of v; a kept
+// 2-bit code (1 = +1, 2 = -1, 0 = dropped) from the keep bit (1 or 0) and the sign bit of v; a kept
 // coordinate is never +-0.
-__device__ __forceinline__ uint32_t code_of(float v, uint32_t keep_mask) {
-  return keep_mask & (1u + (__float_as_uint(v) >> 31));
+__device__ __forceinline__ uint32_t code_of(float v, uint32_t keep01) {
+  return keep01 * mad_hi(__float_as_uint(v), 2u, 0u) + keep01;
 }
 // The code byte of four coordinates that share the Philox block w.
 __device__ __forceinline__ uint32_t stochastic_code_byte(const float4& v, const uint4& w, const KeepTest& kt) {
   uint32_t nearest = 0xffffffffu;
-  const int32_t tx = keep_margin(w.x, fabsf(v.x), kt, nearest), ty = keep_margin(w.y, fabsf(v.y), kt, nearest);
-  const int32_t tz = keep_margin(w.z, fabsf(v.z), kt, nearest), tw = keep_margin(w.w, fabsf(v.w), kt, nearest);
-  uint32_t mx = static_cast<uint32_t>(tx >> 31), my = static_cast<uint32_t>(ty >> 31);
-  uint32_t mz = static_cast<uint32_t>(tz >> 31), mw = static_cast<uint32_t>(tw >> 31);
+  const uint32_t tx = keep_margin(w.x, fabsf(v.x), kt, nearest), ty = keep_margin(w.y, fabsf(v.y), kt, nearest);
+  const uint32_t tz = keep_margin(w.z, fabsf(v.z), kt, nearest), tw = keep_margin(w.w, fabsf(v.w), kt, nearest);
+  uint32_t kx = mad_hi(tx, 2u, 0u), ky = mad_hi(ty, 2u, 0u);  // the sign bit of k - K
+  uint32_t kz = mad_hi(tz, 2u, 0u), kw = mad_hi(tw, 2u, 0u);
   if (!kt.fast || nearest <= 18u) {
-    mx = keeps_exact(w.x, fabsf(v.x), kt.s) ? 0xffffffffu : 0u;
-    my = keeps_exact(w.y, fabsf(v.y), kt.s) ? 0xffffffffu : 0u;
-    mz = keeps_exact(w.z, fabsf(v.z), kt.s) ? 0xffffffffu : 0u;
-    mw = keeps_exact(w.w, fabsf(v.w), kt.s) ? 0xffffffffu : 0u;
+    kx = keeps_exact(w.x, fabsf(v.x), kt.s) ? 1u : 0u;
+    ky = keeps_exact(w.y, fabsf(v.y), kt.s) ? 1u : 0u;
+    kz = keeps_exact(w.z, fabsf(v.z), kt.s) ? 1u : 0u;
+    kw = keeps_exact(w.w, fabsf(v.w), kt.s) ? 1u : 0u;
   }
-  return code_of(v.x, mx) + 4u * code_of(v.y, my) + 16u * code_of(v.z, mz) + 64u * code_of(v.w, mw);
+  return code_of(v.x, kx) + 4u * code_of(v.y, ky) + 16u * code_of(v.z, kz) + 64u * code_of(v.w, kw);
 }
 
 __device__ __forceinline__ float philox_uniform(uint32_t word) {
