@@ -113,14 +113,14 @@ qasg_status qasg_destroy(qasg_ctx* ctx);
  * QASG_OPT_ONE_LAUNCH_STEP_BYTES: qasg_step on at most that many bytes of gradients (4*d*M) runs its
  * three passes as the phases of ONE launch (cooperative when it has more than one CTA) whose CTAs meet
  * twice, with the same bounded waits and the same time-out behaviour: at such sizes a launch costs
- * more than a pass (measured on a B200: 7 to 9 % faster up to 512 KB, slower from about 2 MB on).
+ * more than a pass (measured on a B200: 5 to 20 % faster up to 8 MB, level to 32 MB, slower beyond).
  *
  * Every setting gives the same bits. */
 typedef enum {
   QASG_OPT_STREAM_ROW_BYTES = 0,     /* 0 = never (default)                                          */
   QASG_OPT_STREAM_LAG = 1,           /* 0, 1, 2, ...; 0xFFFFFFFF = chosen from the row size (default) */
   QASG_OPT_WAIT_POLLS = 2,           /* 1 .. 2^31; default 2^22 (about a second)                      */
-  QASG_OPT_ONE_LAUNCH_STEP_BYTES = 3 /* 0 = never; default 524288 (faster there on a B200)           */
+  QASG_OPT_ONE_LAUNCH_STEP_BYTES = 3 /* 0 = never; default 16 MiB (faster or level there on a B200)   */
 } qasg_option;
 qasg_status qasg_set_option(qasg_ctx* ctx, qasg_option option, uint64_t value);
 

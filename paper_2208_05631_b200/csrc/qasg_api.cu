@@ -75,9 +75,10 @@ struct Launch {
 constexpr uint64_t kMaxD = 1ull << 34;
 constexpr uint32_t kAutoLag = 0xFFFFFFFFu;
 constexpr uint64_t kDefaultStreamRowBytes = 0;         // the one-launch kernel is opt-in
-// Up to half a megabyte of gradients the one-launch step measured faster than three chained launches
-// (d = 10,000, M = 4: 11.1 against 11.9 us replayed from a graph); from about 2 MB on it is slower.
-constexpr uint64_t kDefaultOneLaunchStepBytes = 512ull << 10;
+// Up to 16 MB of gradients the one-launch step measured faster than three chained launches or level with them
+// (single cold steps: 5 to 20 % up to 2^18 coordinates x 32 workers, level at 2^20 x 2 and 2^20 x 8; replayed
+// from a graph d = 10,000, M = 4: 9.6 against 11.9 us); beyond that its two meetings cost more than two launches.
+constexpr uint64_t kDefaultOneLaunchStepBytes = 16ull << 20;
 // A row is coded `lag` rows after it was summed; in between the rows summed and coded meanwhile pass
 // through L2.  One row of lag hides the wait for a worker's threshold; it is taken while three rows fit.
 constexpr uint64_t kLagOneRowBytes = 24ull << 20;

@@ -10,8 +10,10 @@ from paper_2208_05631_b200 import inputs, libqasg
 pytestmark = pytest.mark.gpu
 
 
+# the step as three chained launches (option 0) and as the default picks it (one launch at this size)
+@pytest.mark.parametrize("one_launch_bytes", [0, None])
 @pytest.mark.parametrize("rule", [libqasg.RULE_CMD, libqasg.RULE_RDA])
-def test_fused_step_replayed_from_a_cuda_graph(rule):
+def test_fused_step_replayed_from_a_cuda_graph(rule, one_launch_bytes):
     dev = torch.device("cuda:0")
     d, M, t = 40_003, 8, 5
     ld = (d + 3) // 4 * 4
@@ -19,6 +21,8 @@ def test_fused_step_replayed_from_a_cuda_graph(rule):
     g[:, :d] = torch.from_numpy(inputs.optimizer_only_gradients(d, M, t, seed=2) * np.float32(0.01)).to(dev)
     x0, h0, z0 = inputs.random_state(d, seed=2, device=dev)
     ctx = libqasg.Context(d, M, device=0)
+    if one_launch_bytes is not None:
+        ctx.set_option(libqasg.OPT_ONE_LAUNCH_STEP_BYTES, one_launch_bytes)
     params = libqasg.make_params(1e-3, 0.1, 1e-8)
 
     eager = [v.clone() for v in (x0, h0, z0)]
@@ -48,7 +52,8 @@ def test_fused_step_replayed_from_a_cuda_graph(rule):
     ctx.close()
 
 
-def test_chained_launches_give_the_bits_of_serial_launches():
+@pytest.mark.parametrize("one_launch_bytes", [0, None])
+def test_chained_launches_give_the_bits_of_serial_launches(one_launch_bytes):
     """By default a step's kernels are launched as programmatic dependents of one another (a kernel is placed,
     and pass B requests its first tile, while its predecessor drains).  The same iterations on a context
     created with QASG_CREATE_SERIAL_LAUNCHES must give the same bits: gradient kernel + fused step, both
@@ -60,6 +65,8 @@ def test_chained_launches_give_the_bits_of_serial_launches():
     results = []
     for flags in (0, libqasg.CREATE_SERIAL_LAUNCHES):
         ctx = libqasg.Context(d, M, device=0, flags=flags)
+        if one_launch_bytes is not None:
+            ctx.set_option(libqasg.OPT_ONE_LAUNCH_STEP_BYTES, one_launch_bytes)
         out = []
         for quantizer in (libqasg.Q_THRESHOLD, libqasg.Q_TERNARY_STOCH):
             params = libqasg.make_params(1e-4, 0.1, 1e-8, quantizer=quantizer, seed=5)

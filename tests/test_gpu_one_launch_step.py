@@ -123,7 +123,7 @@ def test_non_finite_gradient_in_one_launch(ctx):
 def test_default_takes_one_launch_for_small_problems_only():
     c = libqasg.Context(1 << 20, 8, device=0)
     params = libqasg.make_params(LAM, ETA, DELTA)
-    for d, M, want in ((10_000, 4, 1), (131_072, 1, 1), (70_001, 8, 3)):
+    for d, M, want in ((10_000, 4, 1), (70_001, 8, 1), (1 << 19, 8, 1), ((1 << 19) + 4, 8, 3), (1 << 20, 8, 3)):
         g_dev, ld = U.grad_to_dev(inputs.normal_gradients(d, M, seed=1).numpy())
         x, h = (torch.zeros(d, dtype=torch.float32, device=U.dev()) for _ in range(2))
         before = c.launch_count()
