@@ -29,6 +29,7 @@ struct qasg_ctx {
   uint32_t wait_polls;
   uint64_t launches;
   uint64_t one_launch_step_bytes;  // qasg_step runs as one launch up to this many bytes of gradients
+  bool cooperative;                // the device can run cooperative launches (else the one-launch paths stay off)
   bool ticket_dirty;        // a launch failed since the completion counter was last known to be zero
   bool profiling;
   std::vector<cudaEvent_t> events;  // pairs (start, stop), reused between profiles
@@ -170,7 +171,7 @@ void quantize_pack(qasg_ctx* ctx, const float* g, uint64_t d, uint64_t ld_g, uin
   // One launch, each row coded out of L2: items of a worker's row are dealt to the resident CTAs one row
   // after the other, so a row is cut into about as many chunks as there are CTAs.
   const Geometry sgeo = make_geometry(d, ld_g, M, static_cast<uint32_t>(ctx->shape.sm_count * ctx->shape.reduce_ctas_per_sm));
-  if (d * sizeof(float) <= ctx->stream_row_bytes && sgeo.group <= kStreamMaxGroup) {
+  if (ctx->cooperative && d * sizeof(float) <= ctx->stream_row_bytes && sgeo.group <= kStreamMaxGroup) {
     const bool stochastic = p->quantizer != QASG_Q_THRESHOLD;
     StreamParams sp;
     sp.coef = p->thr_coef;
@@ -317,6 +318,9 @@ qasg_status qasg_create(qasg_ctx** out, int device, uint64_t d_max, uint32_t M_m
   ctx->stream_lag = kAutoLag;
   ctx->wait_polls = 1u << 22;
   ctx->one_launch_step_bytes = kDefaultOneLaunchStepBytes;
+  int cooperative = 0;  // the one-launch paths need all their CTAs resident together
+  cudaDeviceGetAttribute(&cooperative, cudaDevAttrCooperativeLaunch, device);
+  ctx->cooperative = cooperative != 0;
   query_launch_shape(&ctx->shape);
   ctx->shape.chained = !(flags & QASG_CREATE_SERIAL_LAUNCHES);
   const size_t slots = static_cast<size_t>(M_max) * kMaxChunks;
@@ -508,7 +512,7 @@ qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d,
     return leave(ctx);
   }
   uint32_t* codes = codes_out ? codes_out : ctx->code_scratch;
-  if (static_cast<uint64_t>(M) * d * 4 <= ctx->one_launch_step_bytes) {  // small: the three passes as one launch
+  if (ctx->cooperative && static_cast<uint64_t>(M) * d * 4 <= ctx->one_launch_step_bytes) {  // small: the three passes as one launch
     const Geometry geo = make_geometry(d, ld_g, M, kMaxChunks, target_items(ctx));
     Launch l(ctx, rule == QASG_RULE_CMD ? kFusedStepCmd : kFusedStepRda, s);
     l += launch_fused_step(rule, params->quantizer == QASG_Q_TERNARY_STOCH, g, geo, params->thr_coef, params->seed, t,
