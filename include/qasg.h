@@ -183,7 +183,9 @@ qasg_status qasg_rda_step(qasg_ctx* ctx, const float* q, float* x, float* h, flo
  * of a coordinate once, sums them in fp64 in worker order, q_i = fp32(sum * (1/M)), and applies
  * the same accumulator and update (4M + 16 or 20 bytes per coordinate); codes_out and
  * scales_out are not touched, thr_coef and seed are not used.  A non-finite mean is reported
- * as QASG_ERR_NONFINITE and still enters the state, as it would in plain AdaGrad. */
+ * as QASG_ERR_NONFINITE and still enters the state, as it would in plain AdaGrad.
+ * Three launches (sums, codes, decode + update), or one launch with the same three phases for up to
+ * QASG_OPT_ONE_LAUNCH_STEP_BYTES of gradients; the results have the same bits either way. */
 qasg_status qasg_step(qasg_ctx* ctx, qasg_rule rule, const float* g, uint64_t d, uint64_t ld_g,
                       uint32_t M, uint64_t t, const qasg_params* params, float* x, float* h,
                       float* z, uint32_t* codes_out, float* scales_out, void* stream);
